@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the SpecSteer verify + recover round on B200.
+
+One step = specsteer_verify_round + specsteer_recover_sample over one batch of synthetic logits
+(default: B=256, K=4, V=151936, float32 - the batched serving shape).  Prints ONE JSON line:
+verified draft positions/s with inputs resident in HBM (`value`), the same through the host-buffer
+entry point with the copies inside the timed region (`e2e`), the roofline of the streaming kernel,
+the CPU oracle timed on this machine's cores, and the clocks seen while timing.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 0..4] [--impl reference]
+
+Under torchrun every rank runs its own batch (requests shard with no collective on the data path).
+"""
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "verified_draft_positions_per_sec"
+UNIT = "positions/s"
+FALLBACK_HBM_GBS = 6650.0
+NOMINAL_HBM_GBS = 8000.0
+# DRAM bytes per launch of the streaming kernel from ncu (profiles/), keyed by configuration; None = not captured
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Reads SM clock and throttle reasons (read-only NVML queries) every ~10 ms while timing runs."""
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.samples, self.windows, self._stop_evt = [], [], threading.Event()
+        self.max_mhz = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if self.nv is None:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                self.samples.append((time.perf_counter(), mhz, int(reasons)))
+            except Exception:
+                pass
+            time.sleep(0.01)
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def window(self, t0, t1):
+        self.windows.append((t0, t1))
+
+    def summary(self):
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap",
+                 0x80: "hw_power_brake_slowdown"}
+        ins = [s for s in self.samples if any(a <= s[0] <= b for a, b in self.windows)]
+        scope = "timed regions"
+        if not ins:
+            ins, scope = self.samples, "whole run (timed regions shorter than the sampling period)"
+        if not ins:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0, "scope": "nvml unavailable"}
+        mhz = sorted(s[1] for s in ins)
+        bits = 0
+        for s in ins:
+            bits |= s[2]
+        return {"sm_mhz": mhz[len(mhz) // 2], "sm_max_mhz": self.max_mhz,
+                "reasons": [n for b, n in names.items() if bits & b], "samples": len(ins), "scope": scope}
+
+
+def _sample_requests(spec, n):
+    """Indices of a bounded sample that keeps the workload's mix: spread evenly over the sigma blocks."""
+    import numpy as np
+    n = max(1, min(n, spec.B))
+    return np.unique(np.linspace(0, spec.B - 1, n).round().astype(int))
+
+
+def _oracle_time(oracle, synth, inputs, sel, flags, nthreads):
+    import torch
+    idx = torch.as_tensor(sel, device=inputs["h_llm"].device)
+    npin = {k: (synth.to_numpy_bits(v[idx]) if k.startswith("h_") else v[idx].cpu().numpy()) for k, v in inputs.items()}
+    t0 = time.perf_counter()
+    out = oracle.verify_recover_round(
+        npin["h_llm"], npin["h_slm_plus"], npin["h_slm_minus"], npin["draft_tokens"], npin["draft_len"],
+        npin["lam"], npin["beta"], npin["temperature"], npin["u_accept"], npin["u_recover"],
+        flags=flags, nthreads=nthreads)
+    dt = time.perf_counter() - t0
+    return dt, int(npin["draft_len"].sum()), out
+
+
+def run_reference(args, rank, world):
+    """The reference arm: the CPU oracle, as it stands, on this machine's host cores (rank 0 only)."""
+    if rank != 0:
+        return
+    import torch
+    import oracle
+    from paper_2603_16219_b200 import synth
+    oracle.build()
+    spec = synth.CONFIGS[args.config]
+    cores = oracle.max_threads()
+    # inputs for the sample only: generate a reduced batch of the same recipe on the CPU
+    probe_B = min(spec.B, 8)
+    small = synth.RoundSpec(spec.name + "_sample", probe_B, spec.K, spec.V, spec.dtype, sigma_plus=spec.sigma_plus,
+                            heavy_tail=spec.heavy_tail, ragged=spec.ragged, beta_choices=spec.beta_choices,
+                            beta_uniform=spec.beta_uniform, temp_choices=spec.temp_choices, lam=spec.lam)
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    inputs = synth.make_round(small, device=dev, seed=0)
+    flags = oracle.FLAG_BONUS
+    dt, _, _ = _oracle_time(oracle, synth, inputs, list(range(min(2, probe_B))), flags, cores)
+    per_req = dt / min(2, probe_B)
+    budget = 120.0 / max(1, args.steps + args.warmup)
+    n_req = int(max(1, min(probe_B, budget / max(per_req, 1e-6))))
+    ends = [i // 2 if i % 2 == 0 else probe_B - 1 - i // 2 for i in range(probe_B)]   # alternate both regimes
+    sel = sorted(ends[:n_req])
+    for _ in range(args.warmup):
+        _oracle_time(oracle, synth, inputs, sel, flags, cores)
+    tot, pos = 0.0, 0
+    for _ in range(args.steps):
+        dt, p, _ = _oracle_time(oracle, synth, inputs, sel, flags, cores)
+        tot += dt
+        pos += p
+    value = pos / tot
+    sample = "%d of %d requests of %s per step (same recipe, seed 0), all %d rows each" % (n_req, spec.B, spec.name, spec.K + 1)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * tot / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": spec.name, "B": spec.B, "K": spec.K, "V": spec.V, "logit_dtype": spec.dtype,
+                   "accept_mode": "ratio", "recover_mode": "steer", "bonus_row": True, "lambda": spec.lam},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_cuda(args, rank, world, local_rank):
+    import torch
+    from paper_2603_16219_b200 import binding, build, synth
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+
+    spec = synth.CONFIGS[args.config]
+    flags = binding.FLAG_BONUS
+    inputs = synth.make_round(spec, device=dev, seed=rank)     # every rank owns its own requests
+    rows = synth.used_rows(spec, inputs["draft_len"], bonus=True)
+    positions = int(inputs["draft_len"].sum().item())
+    logit_bytes = spec.logit_bytes(rows)
+    ctx = binding.Context(spec.B, spec.K, spec.V, device=local_rank)
+    outs = binding.alloc_outputs(spec.B, spec.K, dev)
+    desc = binding.make_desc(inputs, outs, flags=flags)
+    stream = torch.cuda.current_stream(dev)
+
+    # When the batch fits in L2 (126 MB) rotate over enough copies to exceed it; otherwise the batch itself does.
+    l2_bytes = 126 << 20
+    n_sets = 1 if 3 * spec.rows * spec.V * spec.elem_bytes > 2 * l2_bytes else \
+        int((4 * l2_bytes) // max(1, 3 * spec.rows * spec.V * spec.elem_bytes)) + 1
+    sets = [(inputs, desc)]
+    for i in range(1, n_sets):
+        cp = {k: v.clone() for k, v in inputs.items()}
+        sets.append((cp, binding.make_desc(cp, outs, flags=flags)))
+
+    def step(i):
+        d = sets[i % n_sets][1]
+        ctx.verify_round(d, stream)
+        ctx.recover_sample(d, stream)
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    barrier()
+    # ---- timed region 1: K whole steps, events on the launching stream
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count
+    barrier()
+    w0 = time.perf_counter()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    barrier()
+    w1 = time.perf_counter()
+    sampler.window(w0, w1)
+    gpu_launches = ctx.launch_count - launches0
+    total_ms = e0.elapsed_time(e1)
+    # ---- timed region 2: the streaming kernel alone, one event pair per launch (same warm state)
+    ksteps = min(args.steps, 200)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    w0 = time.perf_counter()
+    for i in range(ksteps):
+        d = sets[i % n_sets][1]
+        evs[i][0].record(stream)
+        ctx.verify_round(d, stream)
+        evs[i][1].record(stream)
+        ctx.recover_sample(d, stream)
+    barrier()
+    sampler.window(w0, time.perf_counter())
+    kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / ksteps
+    assert ctx.device_error() == 0
+
+    if dist is not None:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * positions / (ms_per_step * 1e-3)
+
+    # ---- end to end: pinned host buffers in, pinned host results out, copies inside the timed region
+    host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
+    host_out = binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True)
+    hdesc = binding.make_desc(host_in, host_out, flags=flags)
+    h2d = sum(v.numel() * v.element_size() for v in host_in.values())
+    d2h = sum(v.numel() * v.element_size() for v in host_out.values())
+    e2e_steps = max(3, min(args.steps, 10))
+    for _ in range(2):
+        ctx.round_host(hdesc, stream)
+    barrier()
+    w0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        ctx.round_host(hdesc, stream)
+    torch.cuda.synchronize(dev)
+    w1 = time.perf_counter()
+    sampler.window(w0, w1)
+    e2e_s = (w1 - w0) / e2e_steps
+    if dist is not None:
+        t = torch.tensor([e2e_s], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_value = world * positions / e2e_s
+    assert torch.equal(host_out["accept_len"], outs["accept_len"].cpu())
+    sampler.stop()
+
+    if rank != 0:
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peaks()
+    achieved = logit_bytes / (kernel_ms * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": "verify_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+        "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+        "algorithmic_bytes_per_launch": logit_bytes, "kernel_ms": kernel_ms,
+        "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+        "whole_step_gbs": logit_bytes / (ms_per_step * 1e-3) / 1e9,
+    }
+    cpu = None
+    if world == 1:
+        import oracle
+        oracle.build()
+        cores = oracle.max_threads()
+        sel = _sample_requests(spec, 2 * cores if spec.B > 2 * cores else spec.B)
+        dt, pos, ora = _oracle_time(oracle, synth, inputs, sel, oracle.FLAG_BONUS, cores)
+        got = outs["accept_len"].cpu().numpy()[sel]
+        agree = int((got == ora["accept_len"]).sum())
+        cpu = {"value": pos / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": "%d of %d requests (evenly spaced over the batch), %.1f s of CPU wall time; "
+                         "accept_len equal to the GPU's on %d of them" % (len(sel), spec.B, dt, agree)}
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": spec.name, "B": spec.B, "K": spec.K, "V": spec.V, "logit_dtype": spec.dtype,
+                   "requests_per_gpu": spec.B, "rows_read_per_gpu": rows, "positions_per_step_per_gpu": positions,
+                   "accept_mode": "ratio", "recover_mode": "steer", "bonus_row": True, "lambda": spec.lam,
+                   "acceptance_rate": float(outs["accept_len"].sum().item()) / max(1, positions),
+                   "l2": ("inputs %.2f GB per step exceed L2" % (logit_bytes / 1e9)) if n_sets == 1 else
+                         ("rotating %d input sets (%.2f GB) to exceed L2" % (n_sets, n_sets * logit_bytes / 1e9)),
+                   "parallelism": "requests sharded over %d GPU(s), no collective" % world},
+        "roofline": roofline,
+        "cpu_baseline": cpu,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "api": "specsteer_round_host (pinned host buffers)"},
+        "gpu_launches": int(gpu_launches),
+        "clocks": sampler.summary(),
+    }
+    print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--config", type=int, default=3, help="index into the five benchmark configurations")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if world == 1 and args.gpus > 1:
+        # launched without torchrun: re-launch one process per GPU
+        import subprocess
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+               "--master-addr", "127.0.0.1", "--master-port", str(29500 + os.getpid() % 1000), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
+    if args.impl == "reference":
+        run_reference(args, rank, world)
+    else:
+        run_cuda(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

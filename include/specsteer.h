@@ -1,0 +1,156 @@
+/*
+ * specsteer.h - C ABI of the B200 (sm_100a) verify + recover step of SpecSteer's
+ * Draft-Verify-Recover loop (arXiv 2603.16219).
+ *
+ * One "round" takes, for B requests and K+1 positions each, three logit tensors over
+ * the full vocabulary V:
+ *     h_llm        h_LLM   the cloud Generalist                         (Algorithm 1, "Compute logits")
+ *     h_slm_plus   h_SLM+  the Specialist with private context           (Eq. 5, the drafter Q)
+ *     h_slm_minus  h_SLM-  the Specialist without private context        (Eq. 3 baseline)
+ * plus the K drafted token ids per request, and produces per request the number of
+ * accepted drafts and one token sampled at the first rejection.
+ *
+ * Conventions for every entry point
+ *   - Pointers inside specsteer_round_desc are DEVICE pointers unless the entry point
+ *     says otherwise; all tensors are caller-owned and never freed or retained.
+ *   - Logit tensors are [B][K+1][V], V contiguous; row t of request b starts at element
+ *     b*ld_req + t*ld_row.  The fast path needs 16-byte aligned rows (base pointers,
+ *     ld_row and ld_req all multiples of 16 bytes); otherwise a slower generic kernel runs.
+ *   - Calls only enqueue work on the given CUDA stream (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream).  They never synchronise and never copy to host.
+ *   - Host-checkable mistakes return an error code and launch nothing.  Problems only the
+ *     device can see set bits in req_status[b] and give the defined result stated below;
+ *     no kernel traps or reads out of bounds because of input values.
+ *   - Same inputs give bit-identical outputs from run to run.
+ *   - One round may be in flight per context; contexts are independent.
+ */
+#ifndef SPECSTEER_H
+#define SPECSTEER_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct specsteer_ctx specsteer_ctx; /* opaque, library-owned */
+
+typedef enum {
+  SPECSTEER_OK = 0,
+  SPECSTEER_ERR_INVALID_ARG = 1, /* NULL required pointer, negative size, stride < V, unknown enum */
+  SPECSTEER_ERR_UNSUPPORTED = 2, /* B, K or V beyond the maxima given to specsteer_ctx_create */
+  SPECSTEER_ERR_WORKSPACE = 3,   /* device allocation failed */
+  SPECSTEER_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, wrong device) */
+  SPECSTEER_ERR_ORDER = 5,       /* recover_sample without a preceding verify_round of the same shape */
+  SPECSTEER_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (reported by specsteer_ctx_device_error) */
+} specsteer_status;
+
+typedef enum { SPECSTEER_F32 = 0, SPECSTEER_BF16 = 1 } specsteer_dtype;
+
+/* How alpha_t is formed for drafted token y at position t.
+ *   RATIO    alpha = min(1, P_LLM(y) / (lambda * P_SLM-(y)))                (Eq. 7; Algorithm 1)
+ *   EXACT_Z  alpha = min(1, P*(y) / P_SLM+(y)) with the true partition Z_t  (Eq. 6) */
+typedef enum { SPECSTEER_ACCEPT_RATIO = 0, SPECSTEER_ACCEPT_EXACT_Z = 1 } specsteer_accept_mode;
+
+/* What is sampled at the first rejection.
+ *   STEER     y ~ Softmax(h_LLM + beta (h_SLM+ - h_SLM-))                   (Eq. 8; Algorithm 1 Phase 3)
+ *   RESIDUAL  y ~ normalise(max(0, Softmax(h_rec) - P_SLM+)), the speculative-sampling residual of the
+ *             fused target; not in the paper, offered so that EXACT_Z + RESIDUAL emits exactly P*. */
+typedef enum { SPECSTEER_RECOVER_STEER = 0, SPECSTEER_RECOVER_RESIDUAL = 1 } specsteer_recover_mode;
+
+enum {
+  SPECSTEER_FLAG_BONUS = 1u /* when all drafts are accepted, also sample one token (STEER) from row draft_len */
+};
+
+/* bits of req_status[b] */
+enum {
+  SPECSTEER_REQ_BAD_TOKEN = 1,      /* a reached draft token outside [0,V): that position is a rejection, alpha 0 */
+  SPECSTEER_REQ_BAD_LEN = 2,        /* draft_len outside [0,K]: treated as 0 */
+  SPECSTEER_REQ_NONFINITE = 4,      /* a reached row has a NaN/inf normaliser: accept_len = that row, no token */
+  SPECSTEER_REQ_RESIDUAL_EMPTY = 8, /* RESIDUAL had zero mass: STEER weights were used */
+  SPECSTEER_REQ_BAD_PARAM = 16      /* lambda <= 0, temperature <= 0 or a non-finite parameter: nothing accepted */
+};
+
+typedef struct {
+  int32_t B, K, V;        /* requests, maximum drafts per request, vocabulary size */
+  int64_t ld_row, ld_req; /* strides in ELEMENTS: ld_row >= V, ld_req >= (K+1)*ld_row */
+  int32_t dtype;          /* specsteer_dtype of the three logit tensors */
+  int32_t accept_mode;    /* specsteer_accept_mode */
+  int32_t recover_mode;   /* specsteer_recover_mode */
+  uint32_t flags;         /* SPECSTEER_FLAG_* */
+
+  /* ---- inputs ---- */
+  const void *h_llm, *h_slm_plus, *h_slm_minus; /* [B][K+1][V] logits */
+  const int32_t *draft_tokens;                  /* [B][K]   drafted ids y_hat (Eq. 5) */
+  const int32_t *draft_len;                     /* [B]      drafts actually made, 0..K; rows > draft_len unread */
+  const float *lambda;                          /* [B]      lambda of Eq. 7, > 0 */
+  const float *beta;                            /* [B]      beta of Eq. 8 */
+  const float *temperature;                     /* [B]      > 0; every logit is divided by it before any softmax */
+  const float *u_accept;                        /* [B][K]   uniforms in [0,1) for "Uniform(0,1) <= alpha_t" */
+  const float *u_recover;                       /* [B]      uniform in [0,1) for the recovery sample */
+
+  /* ---- outputs (caller-allocated; any may be NULL except accept_len) ---- */
+  int32_t *accept_len;   /* [B]      drafts accepted before the first rejection */
+  uint8_t *accept_flags; /* [B][K]   1 where u <= alpha (every drafted position, also after the first rejection) */
+  float *alpha;          /* [B][K]   acceptance probability; 0 beyond draft_len */
+  float *logp_llm;       /* [B][K]   log P_LLM(y_hat)      NaN beyond draft_len or for a bad token */
+  float *logp_minus;     /* [B][K]   log P_SLM-(y_hat) */
+  float *logp_plus;      /* [B][K]   log P_SLM+(y_hat) */
+  float *logp_star;      /* [B][K]   log Softmax(h_rec)(y_hat) = log P*(y_hat) at beta = 1 (Eq. 4) */
+  float *log_z;          /* [B][K+1] log sum_v P_LLM (P+/P-)^beta = log Z_t at beta = 1 (Eq. 2); NaN for unread rows */
+  int32_t *rec_token;    /* [B]      sampled token, -1 if none was sampled */
+  float *rec_logprob;    /* [B]      log of its probability under the sampled distribution */
+  int32_t *out_tokens;   /* [B][K+1] accepted drafts followed by rec_token, padded with -1 */
+  int32_t *n_out;        /* [B]      number of valid entries in out_tokens */
+  int32_t *req_status;   /* [B]      SPECSTEER_REQ_* bits */
+} specsteer_round_desc;
+
+/* Create a context on CUDA device `device` able to run rounds up to the given maxima.  Allocates the
+ * workspace (row normalisers, per-chunk partial sums, counters; about
+ * max_B*(max_K+1)*(64 + 32*ceil(max_V/2048)) bytes) once; no later call allocates.
+ * Errors: INVALID_ARG (NULL out, non-positive maxima), CUDA, WORKSPACE. */
+specsteer_status specsteer_ctx_create(specsteer_ctx **out, int device, int32_t max_B, int32_t max_K, int32_t max_V);
+
+/* Free the context and its workspace.  The caller must have synchronised any stream still using it. */
+specsteer_status specsteer_ctx_destroy(specsteer_ctx *ctx);
+
+/* Verification (Algorithm 1 Phase 2; Eq. 6/7): one pass over the three logit streams of every used row
+ * computes the four log-normalisers, then per position the log-probabilities, alpha and the accept flag,
+ * and per request accept_len = the first t with u_accept > alpha (or draft_len).  Writes every output of
+ * the descriptor except rec_token, rec_logprob, out_tokens, n_out (req_status is written here and may gain
+ * bits in specsteer_recover_sample).  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+specsteer_status specsteer_verify_round(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
+
+/* Recovery (Algorithm 1 Phase 3; Eq. 8): for each request whose accept_len < draft_len (or always, with
+ * FLAG_BONUS) samples one token from row accept_len by inverse CDF in vocabulary order:
+ * the smallest v with sum_{j<=v} w(j) > u_recover * sum_j w(j).  Must follow specsteer_verify_round with
+ * the same descriptor on the same stream (ERR_ORDER otherwise).  Writes rec_token, rec_logprob,
+ * out_tokens, n_out.  Errors: INVALID_ARG, ORDER, CUDA. */
+specsteer_status specsteer_recover_sample(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
+
+/* Whole round from HOST memory: every pointer in `desc` is a HOST pointer (pinned memory makes the copies
+ * asynchronous).  Copies inputs to device staging buffers owned by the context (allocated on the first
+ * call, sized for the context's maxima: 3*max_B*(max_K+1)*max_V elements of 4 bytes), runs verification and
+ * recovery, copies every non-NULL output back, and returns after the stream has drained.  Requests are
+ * processed in slabs so that the copy of one slab overlaps the kernels of the previous one.
+ * Errors: as the two calls above, plus WORKSPACE. */
+specsteer_status specsteer_round_host(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
+
+/* Synchronise the context's device and report whether any kernel of this context gave up a bounded wait:
+ * SPECSTEER_OK or SPECSTEER_ERR_TIMEOUT (sticky until the context is destroyed). */
+specsteer_status specsteer_ctx_device_error(specsteer_ctx *ctx);
+
+/* Bytes of device workspace owned by the context. */
+size_t specsteer_ctx_workspace_bytes(const specsteer_ctx *ctx);
+
+/* Number of kernels the context has launched since creation (for launch accounting in benchmarks). */
+uint64_t specsteer_ctx_launch_count(const specsteer_ctx *ctx);
+
+const char *specsteer_status_string(specsteer_status s);
+uint32_t specsteer_version(void); /* major<<16 | minor<<8 | patch */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPECSTEER_H */

@@ -220,6 +220,12 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
 
   for (int t = 0; t < n; ++t) if (a->out_tokens) a->out_tokens[(int64_t)b * (K + 1) + t] = yhat[t];
   n_out = n;
+  /* diagnostic: with FLAG_BONUS row `len` belongs to the round, so its log Z_t is reported whatever n is */
+  if ((a->flags & ORACLE_FLAG_BONUS) && a->log_z) {
+    row_load(w, V, a->dtype, a->h_llm, a->h_slm_plus, a->h_slm_minus,
+             (int64_t)b * a->ld_req + (int64_t)len * a->ld_row, beta, T);
+    if (row_finite(w)) a->log_z[(int64_t)b * (K + 1) + len] = w->lseR - w->lseL - beta * (w->lseP - w->lseM);
+  }
   if (stop_nonfinite) goto done;
 
   /* Phase 3: recovery at the first rejection; with FLAG_BONUS also one token from row len when all were accepted. */
@@ -227,8 +233,6 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
     int64_t off = (int64_t)b * a->ld_req + (int64_t)n * a->ld_row;
     row_load(w, V, a->dtype, a->h_llm, a->h_slm_plus, a->h_slm_minus, off, beta, T);
     if (!row_finite(w)) { status |= ORACLE_REQ_NONFINITE; goto done; }
-    if (n == len && a->log_z)
-      a->log_z[(int64_t)b * (K + 1) + n] = w->lseR - w->lseL - beta * (w->lseP - w->lseM);
     int mode = (n < len) ? a->recover_mode : ORACLE_RECOVER_STEER;
     double W = recovery_weights(w, V, mode, wgt);
     if (mode == ORACLE_RECOVER_RESIDUAL && !(W > 0.0)) {

@@ -1,0 +1,215 @@
+"""Thin ctypes binding over ``libspecsteer.so`` (the C ABI declared in ``include/specsteer.h``).
+
+Only argument marshalling lives here: torch tensors give device (or pinned-host) pointers and the
+current CUDA stream; every step of the round runs inside the library's kernels.  There is no CPU
+fallback: if the library has not been built, or no CUDA device is present, calls raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+from . import build as _build
+
+OK = 0
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_ORDER, ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
+F32, BF16 = 0, 1
+ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
+RECOVER_STEER, RECOVER_RESIDUAL = 0, 1
+FLAG_BONUS = 1
+REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1, 2, 4, 8, 16
+
+EXPORTS = (
+    "specsteer_ctx_create", "specsteer_ctx_destroy", "specsteer_verify_round", "specsteer_recover_sample",
+    "specsteer_round_host", "specsteer_ctx_device_error", "specsteer_ctx_workspace_bytes",
+    "specsteer_ctx_launch_count", "specsteer_status_string", "specsteer_version",
+)
+
+
+class RoundDesc(C.Structure):
+    """Mirror of ``specsteer_round_desc``."""
+    _fields_ = [
+        ("B", C.c_int32), ("K", C.c_int32), ("V", C.c_int32),
+        ("ld_row", C.c_int64), ("ld_req", C.c_int64),
+        ("dtype", C.c_int32), ("accept_mode", C.c_int32), ("recover_mode", C.c_int32), ("flags", C.c_uint32),
+        ("h_llm", C.c_void_p), ("h_slm_plus", C.c_void_p), ("h_slm_minus", C.c_void_p),
+        ("draft_tokens", C.c_void_p), ("draft_len", C.c_void_p),
+        ("lam", C.c_void_p), ("beta", C.c_void_p), ("temperature", C.c_void_p),
+        ("u_accept", C.c_void_p), ("u_recover", C.c_void_p),
+        ("accept_len", C.c_void_p), ("accept_flags", C.c_void_p), ("alpha", C.c_void_p),
+        ("logp_llm", C.c_void_p), ("logp_minus", C.c_void_p), ("logp_plus", C.c_void_p),
+        ("logp_star", C.c_void_p), ("log_z", C.c_void_p),
+        ("rec_token", C.c_void_p), ("rec_logprob", C.c_void_p), ("out_tokens", C.c_void_p),
+        ("n_out", C.c_void_p), ("req_status", C.c_void_p),
+    ]
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None):
+    """dlopen the CUDA library (no CUDA call is made by loading it)."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    path = path or _build.LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(
+            "libspecsteer.so is missing (%s): build it with `python -m paper_2603_16219_b200.build`; "
+            "there is no CPU fallback" % path)
+    lib = C.CDLL(path)
+    lib.specsteer_ctx_create.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_int32, C.c_int32, C.c_int32]
+    lib.specsteer_ctx_create.restype = C.c_int
+    lib.specsteer_ctx_destroy.argtypes = [C.c_void_p]
+    lib.specsteer_ctx_destroy.restype = C.c_int
+    for name in ("specsteer_verify_round", "specsteer_recover_sample", "specsteer_round_host"):
+        fn = getattr(lib, name)
+        fn.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_void_p]
+        fn.restype = C.c_int
+    lib.specsteer_ctx_device_error.argtypes = [C.c_void_p]
+    lib.specsteer_ctx_device_error.restype = C.c_int
+    lib.specsteer_ctx_workspace_bytes.argtypes = [C.c_void_p]
+    lib.specsteer_ctx_workspace_bytes.restype = C.c_size_t
+    lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
+    lib.specsteer_ctx_launch_count.restype = C.c_uint64
+    lib.specsteer_status_string.argtypes = [C.c_int]
+    lib.specsteer_status_string.restype = C.c_char_p
+    lib.specsteer_version.restype = C.c_uint32
+    _lib = lib
+    return lib
+
+
+class SpecSteerError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = load_library().specsteer_status_string(code).decode()
+        super().__init__("%s failed: %s (%d)" % (where, msg, code))
+
+
+def _check(code: int, where: str):
+    if code != OK:
+        raise SpecSteerError(code, where)
+
+
+_OUT_SPECS = {
+    # name: (dtype, per-request shape builder)
+    "accept_len": (torch.int32, lambda K: ()), "accept_flags": (torch.uint8, lambda K: (K,)),
+    "alpha": (torch.float32, lambda K: (K,)), "logp_llm": (torch.float32, lambda K: (K,)),
+    "logp_minus": (torch.float32, lambda K: (K,)), "logp_plus": (torch.float32, lambda K: (K,)),
+    "logp_star": (torch.float32, lambda K: (K,)), "log_z": (torch.float32, lambda K: (K + 1,)),
+    "rec_token": (torch.int32, lambda K: ()), "rec_logprob": (torch.float32, lambda K: ()),
+    "out_tokens": (torch.int32, lambda K: (K + 1,)), "n_out": (torch.int32, lambda K: ()),
+    "req_status": (torch.int32, lambda K: ()),
+}
+
+
+def alloc_outputs(B: int, K: int, device, pin: bool = False) -> Dict[str, torch.Tensor]:
+    """Caller-owned output tensors for one round (torch is only the allocator)."""
+    out = {}
+    for name, (dt, shp) in _OUT_SPECS.items():
+        t = torch.empty((B,) + shp(K), dtype=dt, device=device)
+        out[name] = t.pin_memory() if pin else t
+    return out
+
+
+def make_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor], *, accept_mode=ACCEPT_RATIO,
+              recover_mode=RECOVER_STEER, flags=0, V: Optional[int] = None) -> RoundDesc:
+    """Fill a descriptor from tensors.  Logits: [B, K+1, ld_row] (last dim contiguous); pass V if ld_row > V."""
+    hl, hp, hm = inputs["h_llm"], inputs["h_slm_plus"], inputs["h_slm_minus"]
+    if hl.dim() != 3 or hl.shape != hp.shape or hl.shape != hm.shape or hl.dtype != hp.dtype or hl.dtype != hm.dtype:
+        raise ValueError("logit tensors must share shape [B, K+1, V] and dtype")
+    if hl.dtype not in (torch.float32, torch.bfloat16):
+        raise ValueError("logits must be float32 or bfloat16")
+    for t in (hl, hp, hm):
+        if t.stride(2) != 1 or t.stride() != hl.stride():
+            raise ValueError("logit tensors need a contiguous vocabulary axis and equal strides")
+    B, K1, ld = hl.shape
+    d = RoundDesc()
+    d.B, d.K, d.V = B, K1 - 1, int(V if V is not None else ld)
+    d.ld_row = hl.stride(1) if K1 > 1 else ld          # strides of size-1 axes carry no information
+    d.ld_req = hl.stride(0) if B > 1 else K1 * d.ld_row
+    d.dtype = F32 if hl.dtype == torch.float32 else BF16
+    d.accept_mode, d.recover_mode, d.flags = int(accept_mode), int(recover_mode), int(flags)
+    d.h_llm, d.h_slm_plus, d.h_slm_minus = hl.data_ptr(), hp.data_ptr(), hm.data_ptr()
+
+    def ptr(t, dt, n):
+        if t.dtype != dt or not t.is_contiguous() or t.numel() != n:
+            raise ValueError("bad auxiliary tensor: dtype %s, numel %d (want %s, %d)" % (t.dtype, t.numel(), dt, n))
+        return t.data_ptr() if n else None
+
+    K = K1 - 1
+    d.draft_tokens = ptr(inputs["draft_tokens"], torch.int32, B * K)
+    d.draft_len = ptr(inputs["draft_len"], torch.int32, B)
+    d.lam = ptr(inputs["lam"], torch.float32, B)
+    d.beta = ptr(inputs["beta"], torch.float32, B)
+    d.temperature = ptr(inputs["temperature"], torch.float32, B)
+    d.u_accept = ptr(inputs["u_accept"], torch.float32, B * K)
+    d.u_recover = ptr(inputs["u_recover"], torch.float32, B)
+    for name, (dt, shp) in _OUT_SPECS.items():
+        t = outputs.get(name)
+        n = B
+        for s in shp(K):
+            n *= s
+        setattr(d, name, ptr(t, dt, n) if t is not None else None)
+    return d
+
+
+class Context:
+    """Owns one ``specsteer_ctx`` (device workspace sized for the given maxima)."""
+
+    def __init__(self, max_B: int, max_K: int, max_V: int, device: int = 0):
+        if not torch.cuda.is_available():
+            raise RuntimeError("specsteer needs a CUDA device; there is no CPU fallback")
+        self._lib = load_library()
+        h = C.c_void_p()
+        _check(self._lib.specsteer_ctx_create(C.byref(h), int(device), int(max_B), int(max_K), int(max_V)),
+               "specsteer_ctx_create")
+        self._h = h
+        self.device = int(device)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.specsteer_ctx_destroy(self._h)
+            self._h = None
+
+    __del__ = close
+
+    def _stream(self, stream):
+        s = stream if stream is not None else torch.cuda.current_stream(self.device)
+        return C.c_void_p(s.cuda_stream)
+
+    def verify_round(self, desc: RoundDesc, stream=None):
+        _check(self._lib.specsteer_verify_round(self._h, C.byref(desc), self._stream(stream)), "specsteer_verify_round")
+
+    def recover_sample(self, desc: RoundDesc, stream=None):
+        _check(self._lib.specsteer_recover_sample(self._h, C.byref(desc), self._stream(stream)),
+               "specsteer_recover_sample")
+
+    def round_host(self, desc: RoundDesc, stream=None):
+        _check(self._lib.specsteer_round_host(self._h, C.byref(desc), self._stream(stream)), "specsteer_round_host")
+
+    def device_error(self) -> int:
+        return int(self._lib.specsteer_ctx_device_error(self._h))
+
+    @property
+    def workspace_bytes(self) -> int:
+        return int(self._lib.specsteer_ctx_workspace_bytes(self._h))
+
+    @property
+    def launch_count(self) -> int:
+        return int(self._lib.specsteer_ctx_launch_count(self._h))
+
+
+def verify_recover_round(ctx: Context, inputs, *, accept_mode=ACCEPT_RATIO, recover_mode=RECOVER_STEER, flags=0,
+                         V=None, outputs=None, stream=None) -> Dict[str, torch.Tensor]:
+    """Convenience: allocate outputs if needed, run verification then recovery on the current stream."""
+    hl = inputs["h_llm"]
+    if outputs is None:
+        outputs = alloc_outputs(hl.shape[0], hl.shape[1] - 1, hl.device)
+    desc = make_desc(inputs, outputs, accept_mode=accept_mode, recover_mode=recover_mode, flags=flags, V=V)
+    ctx.verify_round(desc, stream)
+    ctx.recover_sample(desc, stream)
+    return outputs

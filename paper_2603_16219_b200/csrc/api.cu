@@ -1,0 +1,360 @@
+// C ABI: context, argument checks, launches, and the host-buffer round.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "internal.h"
+#include "specsteer.h"
+
+using namespace specsteer;
+
+struct specsteer_ctx {
+  int device;
+  int max_B, max_K, max_V;
+  LaunchInfo li;
+  // workspace (one allocation)
+  void* ws;
+  size_t ws_bytes;
+  float* part;
+  float* lse2;
+  unsigned* counter;
+  int* status_ws;
+  int* dev_error;
+  // last verified round, for the order check
+  bool verified;
+  int v_B, v_K, v_V, v_dtype;
+  const void* v_h_llm;
+  uint64_t launches;
+  bool poisoned;
+  // host-round staging
+  void* stage;
+  size_t stage_bytes;
+  cudaStream_t copy_stream;
+  cudaEvent_t ev_copied[2], ev_done[2];
+  bool host_ready;
+};
+
+static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
+
+namespace {
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct DeviceGuard {
+  int prev;
+  bool ok;
+  explicit DeviceGuard(int dev) : prev(-1), ok(false) {
+    if (cudaGetDevice(&prev) != cudaSuccess) return;
+    ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+  }
+  ~DeviceGuard() {
+    int cur = -1;
+    if (prev >= 0 && cudaGetDevice(&cur) == cudaSuccess && cur != prev) cudaSetDevice(prev);
+  }
+};
+
+specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
+  if (!ctx || !d) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->ld_row < d->V || d->ld_req < (int64_t)(d->K + 1) * d->ld_row) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->dtype != SPECSTEER_F32 && d->dtype != SPECSTEER_BF16) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z)
+    return SPECSTEER_ERR_INVALID_ARG;
+  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL)
+    return SPECSTEER_ERR_INVALID_ARG;
+  if (d->flags & ~(uint32_t)SPECSTEER_FLAG_BONUS) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->B > 0) {
+    if (!d->h_llm || !d->h_slm_plus || !d->h_slm_minus || !d->draft_len || !d->lambda || !d->beta ||
+        !d->temperature || !d->u_recover || !d->accept_len)
+      return SPECSTEER_ERR_INVALID_ARG;
+    if (d->K > 0 && (!d->draft_tokens || !d->u_accept)) return SPECSTEER_ERR_INVALID_ARG;
+  }
+  if (d->B > ctx->max_B || d->K > ctx->max_K || d->V > ctx->max_V) return SPECSTEER_ERR_UNSUPPORTED;
+  return SPECSTEER_OK;
+}
+
+int n_chunks_of(int V) { return (V + kTile - 1) / kTile; }
+
+// Parameters for the slab of requests [b0, b0 + nb).
+RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d, int b0, int nb) {
+  RoundParams p;
+  memset(&p, 0, sizeof p);
+  const size_t es = d->dtype == SPECSTEER_F32 ? 4 : 2;
+  const int K = d->K, K1 = K + 1;
+  p.B = nb; p.K = K; p.V = d->V;
+  p.ld_row = d->ld_row; p.ld_req = d->ld_req;
+  p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
+  p.n_chunks = n_chunks_of(d->V);
+  auto lg = [&](const void* base) { return (const void*)((const char*)base + (size_t)b0 * d->ld_req * es); };
+  p.h_llm = lg(d->h_llm); p.h_plus = lg(d->h_slm_plus); p.h_minus = lg(d->h_slm_minus);
+#define OFF(ptr, stride) ((ptr) ? (ptr) + (size_t)b0 * (stride) : nullptr)
+  p.draft_tokens = OFF(d->draft_tokens, K);
+  p.draft_len = OFF(d->draft_len, 1);
+  p.lambda = OFF(d->lambda, 1); p.beta = OFF(d->beta, 1); p.temperature = OFF(d->temperature, 1);
+  p.u_accept = OFF(d->u_accept, K); p.u_recover = OFF(d->u_recover, 1);
+  p.accept_len = OFF(d->accept_len, 1); p.accept_flags = OFF(d->accept_flags, K);
+  p.alpha = OFF(d->alpha, K); p.logp_llm = OFF(d->logp_llm, K); p.logp_minus = OFF(d->logp_minus, K);
+  p.logp_plus = OFF(d->logp_plus, K); p.logp_star = OFF(d->logp_star, K); p.log_z = OFF(d->log_z, K1);
+  p.rec_token = OFF(d->rec_token, 1); p.rec_logprob = OFF(d->rec_logprob, 1);
+  p.out_tokens = OFF(d->out_tokens, K1); p.n_out = OFF(d->n_out, 1); p.req_status = OFF(d->req_status, 1);
+  p.part = ctx->part + (size_t)b0 * K1 * p.n_chunks * 8;
+  p.lse2 = ctx->lse2 + (size_t)b0 * K1 * 4;
+  p.counter = ctx->counter + b0;
+  p.status_ws = ctx->status_ws + b0;
+#undef OFF
+  p.dev_error = ctx->dev_error;
+  return p;
+}
+
+bool rows_aligned(const specsteer_round_desc* d) {
+  const size_t es = d->dtype == SPECSTEER_F32 ? 4 : 2;
+  auto a16 = [](const void* p) { return ((uintptr_t)p & 15u) == 0; };
+  return a16(d->h_llm) && a16(d->h_slm_plus) && a16(d->h_slm_minus) && ((size_t)d->ld_row * es) % 16 == 0 &&
+         ((size_t)d->ld_req * es) % 16 == 0;
+}
+
+specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
+  const bool aligned = rows_aligned(d);
+  for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
+    const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
+    RoundParams p = slab_params(ctx, d, b0, nb);
+    int nl = 0;
+    if (launch_verify(p, d->dtype, aligned, ctx->li, s, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    ctx->launches += nl;
+  }
+  return SPECSTEER_OK;
+}
+
+specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
+  for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
+    const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
+    RoundParams p = slab_params(ctx, d, b0, nb);
+    int nl = 0;
+    if (launch_recover(p, d->dtype, ctx->li, s, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    ctx->launches += nl;
+  }
+  return SPECSTEER_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t max_B, int32_t max_K, int32_t max_V) {
+  if (!out) return SPECSTEER_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (max_B <= 0 || max_K < 0 || max_V <= 0 || device < 0) return SPECSTEER_ERR_INVALID_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || device >= ndev) return SPECSTEER_ERR_CUDA;
+  DeviceGuard g(device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  specsteer_ctx* c = new (std::nothrow) specsteer_ctx();
+  if (!c) return SPECSTEER_ERR_WORKSPACE;
+  memset(c, 0, sizeof *c);
+  c->device = device; c->max_B = max_B; c->max_K = max_K; c->max_V = max_V;
+  if (cudaDeviceGetAttribute(&c->li.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&c->li.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
+    delete c;
+    return SPECSTEER_ERR_CUDA;
+  }
+  const size_t rows = (size_t)max_B * (max_K + 1);
+  const size_t nch = (size_t)n_chunks_of(max_V);
+  const size_t b_part = align_up(rows * nch * 8 * sizeof(float), 256);
+  const size_t b_lse = align_up(rows * 4 * sizeof(float), 256);
+  const size_t b_cnt = align_up((size_t)max_B * sizeof(unsigned), 256);
+  const size_t b_st = align_up((size_t)max_B * sizeof(int), 256);
+  c->ws_bytes = b_part + b_lse + b_cnt + b_st + 256;
+  if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
+    cudaGetLastError();
+    delete c;
+    return SPECSTEER_ERR_WORKSPACE;
+  }
+  char* w = (char*)c->ws;
+  c->part = (float*)w; w += b_part;
+  c->lse2 = (float*)w; w += b_lse;
+  c->counter = (unsigned*)w; w += b_cnt;
+  c->status_ws = (int*)w; w += b_st;
+  c->dev_error = (int*)w;
+  if (cudaMemset(c->ws, 0, c->ws_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
+    cudaFree(c->ws);
+    delete c;
+    return SPECSTEER_ERR_CUDA;
+  }
+  *out = c;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_ctx_destroy(specsteer_ctx* ctx) {
+  if (!ctx) return SPECSTEER_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (ctx->host_ready) {
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(ctx->ev_copied[i]); cudaEventDestroy(ctx->ev_done[i]); }
+    cudaStreamDestroy(ctx->copy_stream);
+  }
+  if (ctx->stage) cudaFree(ctx->stage);
+  if (ctx->ws) cudaFree(ctx->ws);
+  delete ctx;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_verify_round(specsteer_ctx* ctx, const specsteer_round_desc* d, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  ctx->verified = false;
+  if (d->B == 0) { ctx->verified = true; ctx->v_B = 0; ctx->v_K = d->K; ctx->v_V = d->V; ctx->v_dtype = d->dtype; ctx->v_h_llm = d->h_llm; return SPECSTEER_OK; }
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  st = do_verify(ctx, d, (cudaStream_t)cuda_stream);
+  if (st != SPECSTEER_OK) return st;
+  ctx->verified = true;
+  ctx->v_B = d->B; ctx->v_K = d->K; ctx->v_V = d->V; ctx->v_dtype = d->dtype; ctx->v_h_llm = d->h_llm;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_recover_sample(specsteer_ctx* ctx, const specsteer_round_desc* d, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (!ctx->verified || ctx->v_B != d->B || ctx->v_K != d->K || ctx->v_V != d->V || ctx->v_dtype != d->dtype ||
+      ctx->v_h_llm != d->h_llm)
+    return SPECSTEER_ERR_ORDER;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  return do_recover(ctx, d, (cudaStream_t)cuda_stream);
+}
+
+specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_desc* h, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, h);
+  if (st != SPECSTEER_OK) return st;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (h->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int B = h->B, K = h->K, K1 = K + 1;
+  const size_t es = h->dtype == SPECSTEER_F32 ? 4 : 2;
+  if (!ctx->host_ready) {
+    if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    for (int i = 0; i < 2; ++i) {
+      if (cudaEventCreateWithFlags(&ctx->ev_copied[i], cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming) != cudaSuccess)
+        return SPECSTEER_ERR_CUDA;
+    }
+    ctx->host_ready = true;
+  }
+  // device staging: the three logit tensors (as strided as the caller's) + the small per-request arrays
+  const size_t logit_bytes = align_up((size_t)B * h->ld_req * es, 256);
+  const size_t small = align_up((size_t)B * (size_t)(K1 * 64 + 128) + 1024, 256);
+  const size_t need = 3 * logit_bytes + small;
+  if (need > ctx->stage_bytes) {
+    if (ctx->stage) { cudaStreamSynchronize(s); cudaFree(ctx->stage); ctx->stage = nullptr; ctx->stage_bytes = 0; }
+    if (cudaMalloc(&ctx->stage, need) != cudaSuccess) { cudaGetLastError(); return SPECSTEER_ERR_WORKSPACE; }
+    ctx->stage_bytes = need;
+  }
+  char* base = (char*)ctx->stage;
+  specsteer_round_desc d = *h;
+  d.h_llm = base; d.h_slm_plus = base + logit_bytes; d.h_slm_minus = base + 2 * logit_bytes;
+  char* w = base + 3 * logit_bytes;
+  auto carve = [&](size_t bytes) { char* r = w; w += align_up(bytes, 16); return r; };
+  int32_t* tok = (int32_t*)carve((size_t)B * K * 4); int32_t* len = (int32_t*)carve((size_t)B * 4);
+  float* lam = (float*)carve((size_t)B * 4); float* beta = (float*)carve((size_t)B * 4);
+  float* tmp = (float*)carve((size_t)B * 4); float* ua = (float*)carve((size_t)B * K * 4);
+  float* ur = (float*)carve((size_t)B * 4);
+  d.draft_tokens = tok; d.draft_len = len; d.lambda = lam; d.beta = beta; d.temperature = tmp;
+  d.u_accept = ua; d.u_recover = ur;
+  d.accept_len = (int32_t*)carve((size_t)B * 4);
+  d.accept_flags = h->accept_flags ? (uint8_t*)carve((size_t)B * K) : nullptr;
+  d.alpha = h->alpha ? (float*)carve((size_t)B * K * 4) : nullptr;
+  d.logp_llm = h->logp_llm ? (float*)carve((size_t)B * K * 4) : nullptr;
+  d.logp_minus = h->logp_minus ? (float*)carve((size_t)B * K * 4) : nullptr;
+  d.logp_plus = h->logp_plus ? (float*)carve((size_t)B * K * 4) : nullptr;
+  d.logp_star = h->logp_star ? (float*)carve((size_t)B * K * 4) : nullptr;
+  d.log_z = h->log_z ? (float*)carve((size_t)B * K1 * 4) : nullptr;
+  d.rec_token = h->rec_token ? (int32_t*)carve((size_t)B * 4) : nullptr;
+  d.rec_logprob = h->rec_logprob ? (float*)carve((size_t)B * 4) : nullptr;
+  d.out_tokens = h->out_tokens ? (int32_t*)carve((size_t)B * K1 * 4) : nullptr;
+  d.n_out = h->n_out ? (int32_t*)carve((size_t)B * 4) : nullptr;
+  d.req_status = h->req_status ? (int32_t*)carve((size_t)B * 4) : nullptr;
+
+  bool fail = false;
+#define CK(x) do { if ((x) != cudaSuccess) fail = true; } while (0)
+  // small inputs first, on the compute stream
+  if (K > 0) { CK(cudaMemcpyAsync(tok, h->draft_tokens, (size_t)B * K * 4, cudaMemcpyHostToDevice, s));
+               CK(cudaMemcpyAsync(ua, h->u_accept, (size_t)B * K * 4, cudaMemcpyHostToDevice, s)); }
+  CK(cudaMemcpyAsync(len, h->draft_len, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+  CK(cudaMemcpyAsync(lam, h->lambda, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+  CK(cudaMemcpyAsync(beta, h->beta, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+  CK(cudaMemcpyAsync(tmp, h->temperature, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+  CK(cudaMemcpyAsync(ur, h->u_recover, (size_t)B * 4, cudaMemcpyHostToDevice, s));
+  // the copy stream must not overwrite staging still in use by work queued earlier on `s`
+  CK(cudaEventRecord(ctx->ev_done[0], s));
+  CK(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[0], 0));
+
+  // slabs of requests: copy slab i+1 on the copy stream while slab i computes on `s`
+  const size_t req_bytes = (size_t)h->ld_req * es;
+  size_t per = (size_t)(96u << 20) / (3 * req_bytes);
+  int slab = (int)(per < 1 ? 1 : (per > (size_t)kMaxSlabB ? (size_t)kMaxSlabB : per));
+  int idx = 0;
+  for (int b0 = 0; b0 < B && !fail; b0 += slab, idx ^= 1) {
+    const int nb = B - b0 < slab ? B - b0 : slab;
+    const size_t o = (size_t)b0 * req_bytes, nbytes = (size_t)nb * req_bytes;
+    CK(cudaMemcpyAsync((char*)d.h_llm + o, (const char*)h->h_llm + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+    CK(cudaMemcpyAsync((char*)d.h_slm_plus + o, (const char*)h->h_slm_plus + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+    CK(cudaMemcpyAsync((char*)d.h_slm_minus + o, (const char*)h->h_slm_minus + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+    CK(cudaEventRecord(ctx->ev_copied[idx], ctx->copy_stream));
+    CK(cudaStreamWaitEvent(s, ctx->ev_copied[idx], 0));
+    RoundParams p = slab_params(ctx, &d, b0, nb);
+    int nl = 0;
+    CK(launch_verify(p, d.dtype, rows_aligned(&d), ctx->li, s, &nl)); ctx->launches += nl;
+    CK(launch_recover(p, d.dtype, ctx->li, s, &nl)); ctx->launches += nl;
+  }
+  auto back = [&](void* hp, const void* dp, size_t bytes) {
+    if (hp && dp && bytes) CK(cudaMemcpyAsync(hp, dp, bytes, cudaMemcpyDeviceToHost, s));
+  };
+  back(h->accept_len, d.accept_len, (size_t)B * 4); back(h->accept_flags, d.accept_flags, (size_t)B * K);
+  back(h->alpha, d.alpha, (size_t)B * K * 4); back(h->logp_llm, d.logp_llm, (size_t)B * K * 4);
+  back(h->logp_minus, d.logp_minus, (size_t)B * K * 4); back(h->logp_plus, d.logp_plus, (size_t)B * K * 4);
+  back(h->logp_star, d.logp_star, (size_t)B * K * 4); back(h->log_z, d.log_z, (size_t)B * K1 * 4);
+  back(h->rec_token, d.rec_token, (size_t)B * 4); back(h->rec_logprob, d.rec_logprob, (size_t)B * 4);
+  back(h->out_tokens, d.out_tokens, (size_t)B * K1 * 4); back(h->n_out, d.n_out, (size_t)B * 4);
+  back(h->req_status, d.req_status, (size_t)B * 4);
+#undef CK
+  if (cudaStreamSynchronize(s) != cudaSuccess) fail = true;
+  ctx->verified = false;
+  if (fail) { cudaGetLastError(); return SPECSTEER_ERR_CUDA; }
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_ctx_device_error(specsteer_ctx* ctx) {
+  if (!ctx) return SPECSTEER_ERR_INVALID_ARG;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  int flag = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (cudaMemcpy(&flag, ctx->dev_error, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (flag) ctx->poisoned = true;
+  return flag ? SPECSTEER_ERR_TIMEOUT : SPECSTEER_OK;
+}
+
+size_t specsteer_ctx_workspace_bytes(const specsteer_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }
+uint64_t specsteer_ctx_launch_count(const specsteer_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* specsteer_status_string(specsteer_status s) {
+  switch (s) {
+    case SPECSTEER_OK: return "ok";
+    case SPECSTEER_ERR_INVALID_ARG: return "invalid argument";
+    case SPECSTEER_ERR_UNSUPPORTED: return "shape exceeds the context's maxima";
+    case SPECSTEER_ERR_WORKSPACE: return "device allocation failed";
+    case SPECSTEER_ERR_CUDA: return "CUDA runtime error";
+    case SPECSTEER_ERR_ORDER: return "recover_sample without a matching verify_round";
+    case SPECSTEER_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+  }
+  return "unknown status";
+}
+
+uint32_t specsteer_version(void) { return (0u << 16) | (1u << 8) | 0u; }
+
+}  // extern "C"

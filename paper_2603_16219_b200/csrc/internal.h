@@ -1,0 +1,47 @@
+// Host/device structures shared by the translation units of the library (not part of the ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace specsteer {
+
+// One vocabulary chunk = one tile of the streaming pass = one partial record.
+constexpr int kTile = 2048;
+constexpr int kMaxSlabB = 4096;  // requests handled by one launch (the per-CTA row prefix lives in shared memory)
+
+struct RoundParams {
+  int B, K, V;
+  long long ld_row, ld_req;  // elements
+  int accept_mode, recover_mode;
+  unsigned flags;
+  int n_chunks;  // ceil(V / kTile)
+  const void *h_llm, *h_plus, *h_minus;
+  const int* draft_tokens;
+  const int* draft_len;
+  const float *lambda, *beta, *temperature, *u_accept, *u_recover;
+  int* accept_len;
+  uint8_t* accept_flags;
+  float *alpha, *logp_llm, *logp_minus, *logp_plus, *logp_star, *log_z;
+  int* rec_token;
+  float* rec_logprob;
+  int* out_tokens;
+  int* n_out;
+  int* req_status;
+  // workspace
+  float* part;        // [B*(K+1)][n_chunks][8]  partial records {mL,sL,mP,sP,mM,sM,mR,sR}
+  float* lse2;        // [B*(K+1)][4]            base-2 log-normalisers {L,P,M,R}
+  unsigned* counter;  // [B]                     tiles finished per request (self-resetting)
+  int* status_ws;     // [B]                     request status when the caller passes no req_status
+  int* dev_error;     // [1]                     set when a bounded wait gave up
+};
+
+struct LaunchInfo {
+  int sm_count;
+  int max_smem_optin;
+};
+
+cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
+                          int* n_launches);
+cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);
+
+}  // namespace specsteer

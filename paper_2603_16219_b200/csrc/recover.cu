@@ -1,0 +1,267 @@
+// Recovery kernels (Algorithm 1 Phase 3; Eq. 8): one CTA per request samples one token from the row of
+// the first rejection by inverse CDF in vocabulary order.  The STEER kernel finds the chunk from the
+// per-chunk partial sums the verification pass left in the workspace and re-reads only that chunk.
+// The RESIDUAL kernel makes two extra passes over the row in double precision.
+#include "common.cuh"
+#include "internal.h"
+#include "specsteer.h"
+
+namespace specsteer {
+
+constexpr int kRecThreads = 256;
+constexpr int kPerThread = kTile / kRecThreads;  // 8 consecutive vocabulary entries per thread
+constexpr int kRecWarps = kRecThreads / 32;
+
+struct PickShared {
+  double warp_tot[kRecWarps];
+  double base, target, W;
+  int jstar;
+  int tok_min, tok_max_pos;
+};
+
+// Exclusive prefix of one double per thread over the CTA, in thread order.
+__device__ __forceinline__ double block_excl_scan(double v, double* warp_tot, int tid) {
+  const int lane = tid & 31, warp = tid >> 5;
+  double inc = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    double u = __shfl_up_sync(kFullMask, inc, o);
+    if (lane >= o) inc += u;
+  }
+  if (lane == 31) warp_tot[warp] = inc;
+  __syncthreads();
+  double off = 0.0;
+  for (int w = 0; w < warp; ++w) off += warp_tot[w];
+  __syncthreads();
+  return off + inc - v;
+}
+
+// Walk chunk `jstar`: the smallest v with base + sum_{chunk start..v} w > target, else the last v with w > 0.
+// w[] are this thread's kPerThread weights for entries v0 .. v0+kPerThread-1 (0 beyond V).
+__device__ __forceinline__ int pick_in_chunk(const double (&w)[kPerThread], int v0, PickShared* sh, int tid) {
+  double local = 0.0;
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) local += w[i];
+  const double excl = block_excl_scan(local, sh->warp_tot, tid);
+  double run = sh->base + excl;
+  int cand = 0x7fffffff, lastpos = -1;
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    run += w[i];
+    if (w[i] > 0.0) lastpos = v0 + i;
+    if (run > sh->target && cand == 0x7fffffff) cand = v0 + i;
+  }
+  if (cand != 0x7fffffff) atomicMin(&sh->tok_min, cand);
+  if (lastpos >= 0) atomicMax(&sh->tok_max_pos, lastpos);
+  __syncthreads();
+  return sh->tok_min != 0x7fffffff ? sh->tok_min : sh->tok_max_pos;
+}
+
+struct ReqState {
+  int n, len, status;
+  bool sample;  // a token is to be drawn from row n
+};
+
+__device__ __forceinline__ ReqState request_state(const RoundParams& p, int b) {
+  ReqState s;
+  s.n = p.accept_len[b];
+  s.status = p.status_ws[b];
+  s.len = p.draft_len[b];
+  if (s.len < 0 || s.len > p.K) s.len = 0;
+  const bool bad = (s.status & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+  s.sample = !bad && (s.n < s.len || (p.flags & SPECSTEER_FLAG_BONUS));
+  return s;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundParams p) {
+  extern __shared__ double cw[];  // [n_chunks] chunk weights
+  __shared__ PickShared sh;
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int K = p.K, K1 = K + 1;
+  const ReqState st = request_state(p, b);
+
+  if (p.out_tokens)
+    for (int t = tid; t <= K; t += kRecThreads)
+      p.out_tokens[(long long)b * K1 + t] = (t < st.n) ? p.draft_tokens[(long long)b * K + t] : -1;
+  if (!st.sample) {
+    if (tid == 0) {
+      if (p.rec_token) p.rec_token[b] = -1;
+      if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+      if (p.n_out) p.n_out[b] = st.n;
+    }
+    return;
+  }
+  const long long row = (long long)b * K1 + st.n;
+  const double lseR = (double)p.lse2[row * 4 + Q_R];
+  const float* rec = p.part + row * p.n_chunks * 8;
+  for (int j = tid; j < p.n_chunks; j += kRecThreads) {
+    const float m = rec[j * 8 + 6], s = rec[j * 8 + 7];
+    cw[j] = (m == kNegInf) ? 0.0 : (double)s * exp2((double)m - lseR);
+  }
+  if (tid == 0) { sh.tok_min = 0x7fffffff; sh.tok_max_pos = -1; }
+  __syncthreads();
+  if (tid == 0) {
+    double W = 0.0;
+    for (int j = 0; j < p.n_chunks; ++j) W += cw[j];
+    const double target = (double)p.u_recover[b] * W;
+    double c = 0.0, base = 0.0, base_last = 0.0;
+    int jstar = -1, jlast = 0;
+    for (int j = 0; j < p.n_chunks; ++j) {
+      if (cw[j] > 0.0) { jlast = j; base_last = c; }
+      if (c + cw[j] > target) { jstar = j; base = c; break; }
+      c += cw[j];
+    }
+    if (jstar < 0) { jstar = jlast; base = base_last; }
+    sh.jstar = jstar; sh.base = base; sh.target = target; sh.W = W;
+  }
+  __syncthreads();
+
+  const T* hl = reinterpret_cast<const T*>(p.h_llm);
+  const T* hp = reinterpret_cast<const T*>(p.h_plus);
+  const T* hm = reinterpret_cast<const T*>(p.h_minus);
+  const double beta = (double)p.beta[b];
+  const double cd = (double)(kLog2e / p.temperature[b]);
+  const long long off = (long long)b * p.ld_req + (long long)st.n * p.ld_row;
+  const int v0 = sh.jstar * kTile + tid * kPerThread;
+  double w[kPerThread], y2[kPerThread];
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int v = v0 + i;
+    w[i] = 0.0; y2[i] = 0.0;
+    if (v < p.V) {
+      const double l = (double)load_logit<T>(hl, off + v), pp = (double)load_logit<T>(hp, off + v),
+                   m = (double)load_logit<T>(hm, off + v);
+      y2[i] = (l + beta * (pp - m)) * cd - lseR;  // log2 of Softmax(h_rec)(v)
+      w[i] = exp2(y2[i]);
+    }
+  }
+  const int tok = pick_in_chunk(w, v0, &sh, tid);
+  if (tok >= v0 && tok < v0 + kPerThread) {
+    if (p.rec_token) p.rec_token[b] = tok;
+    if (p.rec_logprob) p.rec_logprob[b] = (float)(y2[tok - v0] * 0.6931471805599453 - log(sh.W));
+    if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
+    if (p.n_out) p.n_out[b] = st.n + 1;
+  }
+  if (tok < 0 && tid == 0) {  // no positive weight anywhere in the chunk: nothing can be sampled
+    if (p.rec_token) p.rec_token[b] = -1;
+    if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+    if (p.n_out) p.n_out[b] = st.n;
+  }
+}
+
+// RESIDUAL: w(v) = max(0, Softmax(h_rec)(v) - P_SLM+(v)) on the rejection row, all in double.
+// Runs after the STEER kernel and overrides its result unless the residual has no mass.
+template <typename T>
+__global__ void __launch_bounds__(kRecThreads) recover_residual_kernel(const RoundParams p) {
+  extern __shared__ double cw[];  // [n_chunks]
+  __shared__ PickShared sh;
+  __shared__ double red[2][kRecWarps];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K1 = p.K + 1;
+  const ReqState st = request_state(p, b);
+  if (!st.sample || st.n >= st.len) return;  // the bonus row is always STEER
+
+  const T* hl = reinterpret_cast<const T*>(p.h_llm);
+  const T* hp = reinterpret_cast<const T*>(p.h_plus);
+  const T* hm = reinterpret_cast<const T*>(p.h_minus);
+  const double beta = (double)p.beta[b];
+  const double cd = (double)(kLog2e / p.temperature[b]);
+  const long long off = (long long)b * p.ld_req + (long long)st.n * p.ld_row;
+  const long long row = (long long)b * K1 + st.n;
+  const double refR = (double)p.lse2[row * 4 + Q_R], refP = (double)p.lse2[row * 4 + Q_P];
+
+  // pass 1: the two normalisers in double, using the single-precision ones as reference exponents
+  double sR = 0.0, sP = 0.0;
+  for (int v = tid; v < p.V; v += kRecThreads) {
+    const double l = (double)load_logit<T>(hl, off + v), pp = (double)load_logit<T>(hp, off + v),
+                 m = (double)load_logit<T>(hm, off + v);
+    sR += exp2((l + beta * (pp - m)) * cd - refR);
+    sP += exp2(pp * cd - refP);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    sR += __shfl_xor_sync(kFullMask, sR, o);
+    sP += __shfl_xor_sync(kFullMask, sP, o);
+  }
+  if (lane == 0) { red[0][warp] = sR; red[1][warp] = sP; }
+  if (tid == 0) { sh.tok_min = 0x7fffffff; sh.tok_max_pos = -1; }
+  __syncthreads();
+  sR = 0.0; sP = 0.0;
+  for (int w = 0; w < kRecWarps; ++w) { sR += red[0][w]; sP += red[1][w]; }
+  const double lseR = refR + log2(sR), lseP = refP + log2(sP);
+
+  // pass 2: residual mass per chunk, one warp per chunk
+  for (int j = warp; j < p.n_chunks; j += kRecWarps) {
+    double acc = 0.0;
+    const int vend = min(p.V, (j + 1) * kTile);
+    for (int v = j * kTile + lane; v < vend; v += 32) {
+      const double l = (double)load_logit<T>(hl, off + v), pp = (double)load_logit<T>(hp, off + v),
+                   m = (double)load_logit<T>(hm, off + v);
+      const double d = exp2((l + beta * (pp - m)) * cd - lseR) - exp2(pp * cd - lseP);
+      if (d > 0.0) acc += d;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(kFullMask, acc, o);
+    if (lane == 0) cw[j] = acc;
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double W = 0.0;
+    for (int j = 0; j < p.n_chunks; ++j) W += cw[j];
+    const double target = (double)p.u_recover[b] * W;
+    double c = 0.0, base = 0.0, base_last = 0.0;
+    int jstar = -1, jlast = 0;
+    for (int j = 0; j < p.n_chunks; ++j) {
+      if (cw[j] > 0.0) { jlast = j; base_last = c; }
+      if (c + cw[j] > target) { jstar = j; base = c; break; }
+      c += cw[j];
+    }
+    if (jstar < 0) { jstar = jlast; base = base_last; }
+    sh.jstar = jstar; sh.base = base; sh.target = target; sh.W = W;
+  }
+  __syncthreads();
+  if (!(sh.W > 0.0)) {  // no residual mass: keep the STEER sample already written
+    if (tid == 0) {
+      p.status_ws[b] = st.status | SPECSTEER_REQ_RESIDUAL_EMPTY;
+      if (p.req_status) p.req_status[b] = st.status | SPECSTEER_REQ_RESIDUAL_EMPTY;
+    }
+    return;
+  }
+  const int v0 = sh.jstar * kTile + tid * kPerThread;
+  double w[kPerThread];
+#pragma unroll
+  for (int i = 0; i < kPerThread; ++i) {
+    const int v = v0 + i;
+    w[i] = 0.0;
+    if (v < p.V) {
+      const double l = (double)load_logit<T>(hl, off + v), pp = (double)load_logit<T>(hp, off + v),
+                   m = (double)load_logit<T>(hm, off + v);
+      const double d = exp2((l + beta * (pp - m)) * cd - lseR) - exp2(pp * cd - lseP);
+      w[i] = d > 0.0 ? d : 0.0;
+    }
+  }
+  const int tok = pick_in_chunk(w, v0, &sh, tid);
+  if (tok >= v0 && tok < v0 + kPerThread) {
+    if (p.rec_token) p.rec_token[b] = tok;
+    if (p.rec_logprob) p.rec_logprob[b] = (float)log(w[tok - v0] / sh.W);
+    if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
+    if (p.n_out) p.n_out[b] = st.n + 1;
+  }
+}
+
+cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches) {
+  (void)li;
+  const size_t smem = (size_t)p.n_chunks * sizeof(double);
+  *n_launches = 1;
+  if (dtype == SPECSTEER_F32) recover_steer_kernel<float><<<p.B, kRecThreads, smem, s>>>(p);
+  else recover_steer_kernel<uint16_t><<<p.B, kRecThreads, smem, s>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess || p.recover_mode != SPECSTEER_RECOVER_RESIDUAL) return e;
+  *n_launches = 2;
+  if (dtype == SPECSTEER_F32) recover_residual_kernel<float><<<p.B, kRecThreads, smem, s>>>(p);
+  else recover_residual_kernel<uint16_t><<<p.B, kRecThreads, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+}  // namespace specsteer

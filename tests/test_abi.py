@@ -1,0 +1,88 @@
+"""Host-side checks that need no GPU: the library builds, loads, and exports what the header declares."""
+import ctypes as C
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2603_16219_b200 import binding, build
+    build.build()
+    return binding.load_library()
+
+
+def _declared_symbols():
+    names = set()
+    inc = os.path.join(ROOT, "include")
+    for f in os.listdir(inc):
+        if f.endswith(".h"):
+            txt = open(os.path.join(inc, f)).read()
+            txt = re.sub(r"/\*.*?\*/", "", txt, flags=re.S)
+            names |= set(re.findall(r"\b(specsteer_[a-z_0-9]+)\s*\(", txt))
+    return names
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2603_16219_b200 import binding
+    declared = _declared_symbols()
+    assert declared, "no declarations found"
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+
+
+def test_version_and_status_strings(lib):
+    assert lib.specsteer_version() >= 0x000100
+    seen = {lib.specsteer_status_string(i).decode() for i in range(7)}
+    assert len(seen) == 7 and "ok" in seen
+    assert lib.specsteer_status_string(99).decode() == "unknown status"
+
+
+def test_descriptor_layout_matches_header(lib):
+    """The ctypes mirror must have the header's field order and a size the C compiler agrees with."""
+    from paper_2603_16219_b200 import binding
+    hdr = open(os.path.join(ROOT, "include", "specsteer.h")).read()
+    body = hdr[hdr.index("typedef struct {"):hdr.index("} specsteer_round_desc;")]
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    fields = []
+    for decl in body.split(";"):
+        decl = decl.replace("typedef struct {", "").strip()
+        if not decl:
+            continue
+        for part in decl.split(","):
+            fields.append(re.findall(r"([A-Za-z_0-9]+)\s*$", part.strip())[0])
+    mirror = [n for n, _ in binding.RoundDesc._fields_]
+    assert [f if f != "lambda" else "lam" for f in fields] == mirror
+    assert C.sizeof(binding.RoundDesc) == 3 * 4 + 4 + 2 * 8 + 4 * 4 + 23 * 8
+
+
+def test_host_checkable_errors_launch_nothing(lib):
+    """NULL context / descriptor are rejected before any CUDA call is made."""
+    from paper_2603_16219_b200 import binding
+    d = binding.RoundDesc()
+    assert lib.specsteer_verify_round(None, C.byref(d), None) == binding.ERR_INVALID_ARG
+    assert lib.specsteer_recover_sample(None, C.byref(d), None) == binding.ERR_INVALID_ARG
+    assert lib.specsteer_round_host(None, C.byref(d), None) == binding.ERR_INVALID_ARG
+    assert lib.specsteer_ctx_destroy(None) == binding.ERR_INVALID_ARG
+    assert lib.specsteer_ctx_create(None, 0, 1, 1, 1) == binding.ERR_INVALID_ARG
+    h = C.c_void_p()
+    assert lib.specsteer_ctx_create(C.byref(h), 0, 0, 1, 1) == binding.ERR_INVALID_ARG
+    assert lib.specsteer_ctx_workspace_bytes(None) == 0
+
+
+def test_product_has_no_cpu_fallback_and_never_imports_the_oracle():
+    import torch
+    from paper_2603_16219_b200 import binding
+    if not torch.cuda.is_available():
+        with pytest.raises(RuntimeError):
+            binding.Context(1, 1, 8)
+    pkg = os.path.join(ROOT, "paper_2603_16219_b200")
+    for dirpath, _, files in os.walk(pkg):
+        for f in files:
+            if f.endswith((".py", ".cu", ".cuh", ".h")):
+                txt = open(os.path.join(dirpath, f)).read()
+                assert "oracle" not in txt.replace("the CPU oracle", ""), f

@@ -1,0 +1,276 @@
+"""GPU-vs-oracle parity, through the C ABI, on seeded synthetic rounds.
+
+Configurations 0-2 are compared request by request in full; configurations 3 and 4 run at full size in
+the launch configuration the benchmark times and are compared on sampled requests plus invariants that
+hold at any size.  Edge cases cover ragged and empty inputs, tails, unaligned rows and degenerate logits.
+"""
+import numpy as np
+import pytest
+import torch
+
+import _parity as P
+
+pytestmark = pytest.mark.gpu
+
+MODES = [("ratio_steer_bonus", 0, 0, 1), ("exact_residual", 1, 1, 0)]
+
+
+@pytest.fixture(scope="module")
+def env(oracle_mod):
+    from paper_2603_16219_b200 import binding, build, synth
+    assert torch.cuda.is_available(), "these tests need the CUDA device"
+    build.build()
+    ctx = binding.Context(max_B=8192, max_K=8, max_V=262144, device=0)
+    yield {"ctx": ctx, "binding": binding, "synth": synth, "oracle": oracle_mod}
+    ctx.close()
+
+
+def _small(synth, B, K, V, dtype="f32", seed=0, **kw):
+    spec = synth.RoundSpec("small", B, K, V, dtype, **kw)
+    return spec, synth.make_round(spec, device="cuda", seed=seed)
+
+
+# ------------------------------------------------------------------ the five configurations
+@pytest.mark.parametrize("cfg", [0, 1, 2])
+@pytest.mark.parametrize("mode", MODES, ids=[m[0] for m in MODES])
+def test_config_full_parity(env, cfg, mode):
+    synth = env["synth"]
+    spec = synth.CONFIGS[cfg]
+    inputs = synth.make_round(spec, device="cuda", seed=0)
+    _, am, rm, fl = mode
+    gpu = P.run_gpu(env["ctx"], inputs, am, rm, fl)
+    stats = P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, fl, P.TOL[inputs["h_llm"].dtype])
+    print(spec.name, mode[0], stats, "acceptance", gpu["accept_len"].sum() / inputs["draft_len"].sum().item())
+    assert stats["excused_accept"] + stats["excused_token"] <= max(1, spec.B // 16)
+
+
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_config_full_size_sampled_parity(env, cfg):
+    synth = env["synth"]
+    spec = synth.CONFIGS[cfg]
+    inputs = synth.make_round(spec, device="cuda", seed=0)
+    for _, am, rm, fl in MODES:
+        gpu = P.run_gpu(env["ctx"], inputs, am, rm, fl)
+        P.invariants(gpu, inputs, fl)
+        rng = np.random.default_rng(cfg)
+        sel = np.sort(rng.choice(spec.B, size=12, replace=False))
+        sel[0], sel[-1] = 0, spec.B - 1          # the first and the last request always
+        npin = P.to_np_inputs(inputs, torch.as_tensor(sel, device="cuda"))
+        stats = P.compare(env["oracle"], gpu, npin, am, rm, fl, P.TOL[inputs["h_llm"].dtype], sel=sel)
+        print(spec.name, stats)
+    # run-to-run determinism on the full-size launch (fixed reduction order everywhere)
+    again = P.run_gpu(env["ctx"], inputs, *MODES[1][1:])
+    for k in gpu:
+        assert np.array_equal(gpu[k], again[k], equal_nan=True), k
+
+
+# ------------------------------------------------------------------ shapes, tails, strides
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V", [1, 3, 8, 100, 2047, 2048, 2049, 4100, 6151])
+def test_vocabulary_tails(env, V, dtype):
+    spec, inputs = _small(env["synth"], 5, 3, V, dtype, seed=V, ragged=True, beta_choices=(0.5, 1.0, 2.0),
+                          temp_choices=(0.7, 1.0))
+    for _, am, rm, fl in MODES:
+        gpu = P.run_gpu(env["ctx"], inputs, am, rm, fl)
+        P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, fl, P.TOL[inputs["h_llm"].dtype])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("V,ld", [(1000, 1000 + 8), (1001, 1001), (2500, 2503), (4099, 4104)])
+def test_row_strides_and_unaligned_rows(env, V, ld, dtype):
+    """Row stride > V, and strides that break 16-byte alignment (served by the generic kernel)."""
+    spec, inputs = _small(env["synth"], 4, 2, V, dtype, seed=ld)
+    for k in ("h_llm", "h_slm_plus", "h_slm_minus"):
+        padded = torch.full((4, 3, ld), float("nan"), dtype=inputs[k].dtype, device="cuda")
+        padded[:, :, :V] = inputs[k]
+        inputs[k] = padded
+    gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1, V=V)
+    npin = P.to_np_inputs(inputs)
+    P.compare(env["oracle"], gpu, npin, 0, 0, 1, P.TOL[inputs["h_llm"].dtype], V=V)
+    # a base pointer that is not 16-byte aligned
+    if ld > V:
+        shifted = dict(inputs)
+        for k in ("h_llm", "h_slm_plus", "h_slm_minus"):
+            flat = inputs[k].reshape(-1)
+            n = 4 * 3 * ld
+            buf = torch.empty(n + 1, dtype=flat.dtype, device="cuda")
+            buf[1:] = flat
+            shifted[k] = buf[1:].view(4, 3, ld)
+        gpu2 = P.run_gpu(env["ctx"], shifted, 0, 0, 1, V=V)
+        for key in ("accept_len", "rec_token", "accept_flags"):
+            assert np.array_equal(gpu[key], gpu2[key])
+        np.testing.assert_allclose(gpu["logp_star"], gpu2["logp_star"], atol=1e-5, equal_nan=True)
+
+
+def test_draft_length_extremes_and_no_bonus(env):
+    """len 0 (with and without the bonus row: a request that reads nothing), len K, ragged in between."""
+    spec, inputs = _small(env["synth"], 9, 4, 3000, "f32", seed=3)
+    inputs["draft_len"] = torch.tensor([0, 4, 1, 0, 2, 3, 0, 4, 4], dtype=torch.int32, device="cuda")
+    for am, rm, fl in ((0, 0, 0), (0, 0, 1), (1, 1, 0)):
+        gpu = P.run_gpu(env["ctx"], inputs, am, rm, fl)
+        P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, fl, 1e-4)
+        if fl == 0:
+            assert (gpu["n_out"][[0, 3, 6]] == 0).all() and (gpu["rec_token"][[0, 3, 6]] == -1).all()
+
+
+def test_all_accepted_and_rejected_at_row_zero(env):
+    spec, inputs = _small(env["synth"], 6, 5, 5000, "bf16", seed=4)
+    inputs["h_slm_minus"] = inputs["h_llm"].clone()                 # ratio >= 1 everywhere (lambda 0.5)
+    gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
+    assert (gpu["accept_len"] == 5).all() and (gpu["alpha"] == 1).all() and (gpu["n_out"] == 6).all()
+    P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), 0, 0, 1, 2e-3)
+    inputs["lam"] = torch.full((6,), 1e30, device="cuda")           # ratio ~ 0: rejected at row 0
+    inputs["u_accept"] = torch.full((6, 5), 0.5, device="cuda")
+    gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 0)
+    assert (gpu["accept_len"] == 0).all() and (gpu["n_out"] == 1).all()
+    P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), 0, 0, 0, 2e-3)
+
+
+def test_degenerate_logits_and_status_words(env):
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 8, 2, 2600, "f32", seed=5)
+    L, Pp, M = inputs["h_llm"], inputs["h_slm_plus"], inputs["h_slm_minus"]
+    L[0, :, 100:2300] = float("-inf"); Pp[0, :, 100:2300] = float("-inf"); M[0, :, 100:2300] = float("-inf")  # masked vocabulary -> NaN in r
+    L[1, :, ::2] = float("-inf")                                    # half of the generalist's vocabulary masked
+    L[2, 1, 7] = float("nan")                                       # NaN in a reached row
+    L[3, 0, :] *= 40.0; Pp[3, 0, :] *= 40.0; M[3, 0, :] *= 40.0     # huge dynamic range
+    inputs["draft_tokens"][4, 0] = 2600                             # token out of range
+    inputs["draft_len"][5] = 7                                      # length out of range
+    inputs["temperature"][6] = 0.0                                  # bad temperature
+    L[7, 2, 5] = float("inf")                                       # +inf in the bonus row
+    inputs["u_accept"][:] = 0.0
+    inputs["u_accept"][2, 0] = 0.0
+    for am, rm, fl in ((0, 0, 1), (1, 1, 1)):
+        gpu = P.run_gpu(env["ctx"], inputs, am, rm, fl)
+        stats = P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, fl, 1e-4)
+        assert gpu["req_status"][0] == b.REQ_NONFINITE
+        assert gpu["req_status"][4] & b.REQ_BAD_TOKEN and gpu["accept_len"][4] == 0
+        assert gpu["req_status"][5] == b.REQ_BAD_LEN
+        assert gpu["req_status"][6] == b.REQ_BAD_PARAM and gpu["n_out"][6] == 0
+        assert gpu["req_status"][2] & b.REQ_NONFINITE or gpu["accept_len"][2] == 0
+
+
+def test_many_requests_cross_the_slab_limit(env):
+    spec, inputs = _small(env["synth"], 5000, 2, 64, "bf16", seed=6, ragged=True)
+    gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
+    rng = np.random.default_rng(0)
+    sel = np.sort(np.concatenate([[0, 4095, 4096, 4999], rng.choice(5000, 60, replace=False)]))
+    sel = np.unique(sel)
+    npin = P.to_np_inputs(inputs, torch.as_tensor(sel, device="cuda"))
+    P.compare(env["oracle"], gpu, npin, 0, 0, 1, 2e-3, sel=sel)
+
+
+def test_zero_requests_and_zero_drafts(env):
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 3, 0, 500, "f32", seed=7)
+    gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)                     # K = 0: only the bonus row
+    P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), 0, 0, 1, 1e-4)
+    empty = {k: v[:0] for k, v in inputs.items()}
+    out = b.verify_recover_round(env["ctx"], empty, flags=1)
+    assert out["accept_len"].numel() == 0
+
+
+# ------------------------------------------------------------------ the law, on the GPU
+def test_output_law_monte_carlo_on_gpu(env):
+    """4096 identical V=8 requests x 64 rounds with fresh drafts and uniforms against the closed-form law."""
+    import scipy.special as sps
+    V, K, Bn, rounds, lam, beta = 8, 2, 4096, 64, 0.7, 1.2
+    g = torch.Generator(device="cpu"); g.manual_seed(21)
+    rows = [(1.5 * torch.randn(K + 1, V, generator=g)) for _ in range(3)]
+    L, Pp, M = rows[0], rows[0] + rows[1], rows[0] + 0.7 * rows[2]
+    l, p, m = (x.double().numpy() for x in (L, Pp, M))
+    pl, pp, pm = sps.softmax(l, -1), sps.softmax(p, -1), sps.softmax(m, -1)
+    pstar = sps.softmax(l + beta * (p - m), -1)
+    alpha = np.minimum(1.0, pl / (lam * pm))
+    a = (pp * alpha).sum(-1)
+    reach = np.concatenate([[1.0], np.cumprod(a[:K])])
+    want_n = np.array([reach[t] * (1 - a[t]) for t in range(K)] + [reach[K]])
+    inputs = {
+        "h_llm": L.expand(Bn, K + 1, V).contiguous().cuda(), "h_slm_plus": Pp.expand(Bn, K + 1, V).contiguous().cuda(),
+        "h_slm_minus": M.expand(Bn, K + 1, V).contiguous().cuda(),
+        "draft_len": torch.full((Bn,), K, dtype=torch.int32, device="cuda"),
+        "lam": torch.full((Bn,), lam, device="cuda"), "beta": torch.full((Bn,), beta, device="cuda"),
+        "temperature": torch.ones(Bn, device="cuda"),
+    }
+    cnt_n = np.zeros(K + 1); cnt_tok = np.zeros((K + 1, V))
+    gg = torch.Generator(device="cuda"); gg.manual_seed(22)
+    ppt = torch.from_numpy(pp).cuda()
+    for _ in range(rounds):
+        inputs["draft_tokens"] = torch.stack(
+            [torch.multinomial(ppt[t], Bn, replacement=True, generator=gg) for t in range(K)], 1).to(torch.int32)
+        inputs["u_accept"] = torch.rand(Bn, K, device="cuda", generator=gg)
+        inputs["u_recover"] = torch.rand(Bn, device="cuda", generator=gg)
+        gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
+        cnt_n += np.bincount(gpu["accept_len"], minlength=K + 1)
+        for t in range(K + 1):
+            cnt_tok[t] += np.bincount(gpu["rec_token"][gpu["accept_len"] == t], minlength=V)
+    N = Bn * rounds
+    np.testing.assert_allclose(cnt_n / N, want_n, atol=5.0 / np.sqrt(N))
+    for t in range(K + 1):
+        np.testing.assert_allclose(cnt_tok[t] / N, want_n[t] * pstar[t], atol=5.0 / np.sqrt(N))
+
+
+# ------------------------------------------------------------------ boundary behaviour
+def test_guard_regions_and_determinism(env):
+    """Outputs live inside sentinel-filled buffers: nothing outside the declared extents may change,
+    and a second run must reproduce every byte."""
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 7, 3, 4100, "bf16", seed=8, ragged=True)
+    B, K = 7, 3
+    PAD = 64
+    bufs, outs = {}, {}
+    for name, (dt, shp) in b._OUT_SPECS.items():
+        n = B * int(np.prod(shp(K))) if shp(K) else B
+        raw = torch.full((n + 2 * PAD,), 0x5A, dtype=torch.uint8, device="cuda").repeat_interleave(
+            torch.empty((), dtype=dt).element_size())
+        bufs[name] = raw
+        es = torch.empty((), dtype=dt).element_size()
+        outs[name] = raw[PAD * es:(PAD + n) * es].view(dt).view((B,) + shp(K))
+    runs = []
+    for _ in range(2):
+        b.verify_recover_round(env["ctx"], inputs, accept_mode=1, recover_mode=1, flags=1, outputs=outs)
+        torch.cuda.synchronize()
+        runs.append({k: v.clone() for k, v in bufs.items()})
+    for name, raw in bufs.items():
+        es = torch.empty((), dtype=b._OUT_SPECS[name][0]).element_size()
+        assert (raw[:PAD * es] == 0x5A).all() and (raw[-PAD * es:] == 0x5A).all(), name
+        assert torch.equal(runs[0][name], runs[1][name]), name
+
+
+def test_error_codes_on_device(env):
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 2, 2, 300, "f32", seed=9)
+    outs = b.alloc_outputs(2, 2, "cuda")
+    desc = b.make_desc(inputs, outs, flags=1)
+    small_ctx = b.Context(max_B=1, max_K=2, max_V=300)
+    with pytest.raises(b.SpecSteerError) as e:
+        small_ctx.verify_round(desc)
+    assert e.value.code == b.ERR_UNSUPPORTED
+    fresh = b.Context(max_B=4, max_K=2, max_V=300)
+    with pytest.raises(b.SpecSteerError) as e:
+        fresh.recover_sample(desc)
+    assert e.value.code == b.ERR_ORDER
+    desc.ld_row = 299
+    with pytest.raises(b.SpecSteerError) as e:
+        fresh.verify_round(desc)
+    assert e.value.code == b.ERR_INVALID_ARG
+    desc.ld_row = 300
+    desc.accept_len = None
+    with pytest.raises(b.SpecSteerError) as e:
+        fresh.verify_round(desc)
+    assert e.value.code == b.ERR_INVALID_ARG
+    assert fresh.launch_count == 0 and fresh.workspace_bytes > 0
+    small_ctx.close(); fresh.close()
+
+
+def test_host_round_matches_device_round(env):
+    """The host-buffer entry point (copies inside the call) gives the same bytes as the device path."""
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 37, 3, 9000, "bf16", seed=10, ragged=True)
+    dev = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
+    host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
+    host_out = b.alloc_outputs(37, 3, "cpu", pin=True)
+    desc = b.make_desc(host_in, host_out, flags=1)
+    env["ctx"].round_host(desc)
+    for k, v in host_out.items():
+        assert np.array_equal(dev[k], v.numpy(), equal_nan=True), k
