@@ -174,6 +174,9 @@ def run_cuda(args, rank, world, local_rank):
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
     spec = synth.CONFIGS[args.config]
+    if args.requests:   # a reduced batch of the same recipe, for profiler captures that must stay small
+        import dataclasses
+        spec = dataclasses.replace(spec, B=args.requests, name="%s_first%d" % (spec.name, args.requests))
     flags = binding.FLAG_BONUS
     inputs = synth.make_round(spec, device=dev, seed=rank)     # every rank owns its own requests
     rows = synth.used_rows(spec, inputs["draft_len"], bonus=True)
@@ -245,6 +248,16 @@ def run_cuda(args, rank, world, local_rank):
     ms_per_step = total_ms / args.steps
     value = world * positions / (ms_per_step * 1e-3)
 
+    if args.kernels_only:
+        sampler.stop()
+        if rank == 0:
+            print(json.dumps({"workload": spec.name, "ms_per_step": ms_per_step, "verify_kernel_ms": kernel_ms,
+                              "verify_gbs": logit_bytes / (kernel_ms * 1e-3) / 1e9, "positions_per_s": value,
+                              "clocks": sampler.summary()}), flush=True)
+        if dist is not None:
+            dist.barrier()
+            dist.destroy_process_group()
+        return
     # ---- end to end: pinned host buffers in, pinned host results out, copies inside the timed region
     host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
     host_out = binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True)
@@ -290,13 +303,16 @@ def run_cuda(args, rank, world, local_rank):
         import oracle
         oracle.build()
         cores = oracle.max_threads()
-        sel = _sample_requests(spec, 2 * cores if spec.B > 2 * cores else spec.B)
+        probe = _sample_requests(spec, min(spec.B, cores))
+        dt, pos, _ = _oracle_time(oracle, synth, inputs, probe, oracle.FLAG_BONUS, cores)
+        n = int(min(spec.B, max(len(probe), 20.0 / max(dt / len(probe), 1e-9))))     # about 20 s of wall time at most
+        sel = _sample_requests(spec, n)
         dt, pos, ora = _oracle_time(oracle, synth, inputs, sel, oracle.FLAG_BONUS, cores)
         got = outs["accept_len"].cpu().numpy()[sel]
         agree = int((got == ora["accept_len"]).sum())
         cpu = {"value": pos / dt, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": "%d of %d requests (evenly spaced over the batch), %.1f s of CPU wall time; "
-                         "accept_len equal to the GPU's on %d of them" % (len(sel), spec.B, dt, agree)}
+               "sample": "%d of %d requests (evenly spaced over the batch), %.2f s wall on %d threads; "
+                         "accept_len equal to the GPU's on %d of them" % (len(sel), spec.B, dt, cores, agree)}
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -328,6 +344,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--config", type=int, default=3, help="index into the five benchmark configurations")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--requests", type=int, default=0, help="override B (reduced batch for profiler captures)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="time only the device-resident steps and print a short line (profiling aid)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

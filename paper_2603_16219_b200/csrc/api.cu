@@ -18,7 +18,6 @@ struct specsteer_ctx {
   size_t ws_bytes;
   float* part;
   float* lse2;
-  unsigned* counter;
   int* status_ws;
   int* dev_error;
   // last verified round, for the order check
@@ -54,6 +53,9 @@ struct DeviceGuard {
   }
 };
 
+int tile_of(int dtype) { return dtype == SPECSTEER_F32 ? kTileF32 : kTileBF16; }
+int n_chunks_of(int V, int tile) { return (V + tile - 1) / tile; }
+
 specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
   if (!ctx || !d) return SPECSTEER_ERR_INVALID_ARG;
   if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
@@ -71,10 +73,12 @@ specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc
     if (d->K > 0 && (!d->draft_tokens || !d->u_accept)) return SPECSTEER_ERR_INVALID_ARG;
   }
   if (d->B > ctx->max_B || d->K > ctx->max_K || d->V > ctx->max_V) return SPECSTEER_ERR_UNSUPPORTED;
+  // tiles of one launch are indexed with 31 bits
+  const size_t slab_b = d->B < kMaxSlabB ? d->B : kMaxSlabB;
+  if (slab_b * (size_t)(d->K + 1) * (size_t)n_chunks_of(d->V, kTileMin) >= ((size_t)1 << 31)) return SPECSTEER_ERR_UNSUPPORTED;
   return SPECSTEER_OK;
 }
 
-int n_chunks_of(int V) { return (V + kTile - 1) / kTile; }
 
 // Parameters for the slab of requests [b0, b0 + nb).
 RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d, int b0, int nb) {
@@ -85,7 +89,8 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
   p.B = nb; p.K = K; p.V = d->V;
   p.ld_row = d->ld_row; p.ld_req = d->ld_req;
   p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
-  p.n_chunks = n_chunks_of(d->V);
+  p.tile = tile_of(d->dtype);
+  p.n_chunks = n_chunks_of(d->V, p.tile);
   auto lg = [&](const void* base) { return (const void*)((const char*)base + (size_t)b0 * d->ld_req * es); };
   p.h_llm = lg(d->h_llm); p.h_plus = lg(d->h_slm_plus); p.h_minus = lg(d->h_slm_minus);
 #define OFF(ptr, stride) ((ptr) ? (ptr) + (size_t)b0 * (stride) : nullptr)
@@ -100,7 +105,6 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
   p.out_tokens = OFF(d->out_tokens, K1); p.n_out = OFF(d->n_out, 1); p.req_status = OFF(d->req_status, 1);
   p.part = ctx->part + (size_t)b0 * K1 * p.n_chunks * 8;
   p.lse2 = ctx->lse2 + (size_t)b0 * K1 * 4;
-  p.counter = ctx->counter + b0;
   p.status_ws = ctx->status_ws + b0;
 #undef OFF
   p.dev_error = ctx->dev_error;
@@ -153,18 +157,18 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   if (!c) return SPECSTEER_ERR_WORKSPACE;
   memset(c, 0, sizeof *c);
   c->device = device; c->max_B = max_B; c->max_K = max_K; c->max_V = max_V;
+  c->li.device = device;
   if (cudaDeviceGetAttribute(&c->li.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->li.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
     delete c;
     return SPECSTEER_ERR_CUDA;
   }
   const size_t rows = (size_t)max_B * (max_K + 1);
-  const size_t nch = (size_t)n_chunks_of(max_V);
+  const size_t nch = (size_t)n_chunks_of(max_V, kTileMin);
   const size_t b_part = align_up(rows * nch * 8 * sizeof(float), 256);
   const size_t b_lse = align_up(rows * 4 * sizeof(float), 256);
-  const size_t b_cnt = align_up((size_t)max_B * sizeof(unsigned), 256);
   const size_t b_st = align_up((size_t)max_B * sizeof(int), 256);
-  c->ws_bytes = b_part + b_lse + b_cnt + b_st + 256;
+  c->ws_bytes = b_part + b_lse + b_st + 256;
   if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
     cudaGetLastError();
     delete c;
@@ -173,7 +177,6 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   char* w = (char*)c->ws;
   c->part = (float*)w; w += b_part;
   c->lse2 = (float*)w; w += b_lse;
-  c->counter = (unsigned*)w; w += b_cnt;
   c->status_ws = (int*)w; w += b_st;
   c->dev_error = (int*)w;
   if (cudaMemset(c->ws, 0, c->ws_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {

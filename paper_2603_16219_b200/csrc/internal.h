@@ -5,8 +5,10 @@
 
 namespace specsteer {
 
-// One vocabulary chunk = one tile of the streaming pass = one partial record.
-constexpr int kTile = 2048;
+// One vocabulary chunk = one tile of the streaming pass = one partial record.  12 KB per stream either way.
+constexpr int kTileF32 = 1024;
+constexpr int kTileBF16 = 2048;
+constexpr int kTileMin = 1024;
 constexpr int kMaxSlabB = 4096;  // requests handled by one launch (the per-CTA row prefix lives in shared memory)
 
 struct RoundParams {
@@ -14,7 +16,8 @@ struct RoundParams {
   long long ld_row, ld_req;  // elements
   int accept_mode, recover_mode;
   unsigned flags;
-  int n_chunks;  // ceil(V / kTile)
+  int tile;      // vocabulary entries per chunk (kTileF32 or kTileBF16)
+  int n_chunks;  // ceil(V / tile)
   const void *h_llm, *h_plus, *h_minus;
   const int* draft_tokens;
   const int* draft_len;
@@ -30,12 +33,12 @@ struct RoundParams {
   // workspace
   float* part;        // [B*(K+1)][n_chunks][8]  partial records {mL,sL,mP,sP,mM,sM,mR,sR}
   float* lse2;        // [B*(K+1)][4]            base-2 log-normalisers {L,P,M,R}
-  unsigned* counter;  // [B]                     tiles finished per request (self-resetting)
   int* status_ws;     // [B]                     request status when the caller passes no req_status
   int* dev_error;     // [1]                     set when a bounded wait gave up
 };
 
 struct LaunchInfo {
+  int device;
   int sm_count;
   int max_smem_optin;
 };

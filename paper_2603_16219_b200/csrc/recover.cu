@@ -9,7 +9,6 @@
 namespace specsteer {
 
 constexpr int kRecThreads = 256;
-constexpr int kPerThread = kTile / kRecThreads;  // 8 consecutive vocabulary entries per thread
 constexpr int kRecWarps = kRecThreads / 32;
 
 struct PickShared {
@@ -37,8 +36,10 @@ __device__ __forceinline__ double block_excl_scan(double v, double* warp_tot, in
 }
 
 // Walk chunk `jstar`: the smallest v with base + sum_{chunk start..v} w > target, else the last v with w > 0.
-// w[] are this thread's kPerThread weights for entries v0 .. v0+kPerThread-1 (0 beyond V).
-__device__ __forceinline__ int pick_in_chunk(const double (&w)[kPerThread], int v0, PickShared* sh, int tid) {
+// w[] are this thread's PER weights for entries v0 .. v0+PER-1 (0 beyond V).
+template <int PER>
+__device__ __forceinline__ int pick_in_chunk(const double (&w)[PER], int v0, PickShared* sh, int tid) {
+  constexpr int kPerThread = PER;
   double local = 0.0;
 #pragma unroll
   for (int i = 0; i < kPerThread; ++i) local += w[i];
@@ -73,8 +74,10 @@ __device__ __forceinline__ ReqState request_state(const RoundParams& p, int b) {
   return s;
 }
 
-template <typename T>
+template <typename T, int TILE>
 __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundParams p) {
+  constexpr int kPerThread = TILE / kRecThreads;  // consecutive vocabulary entries per thread
+  constexpr int kTile = TILE;
   extern __shared__ double cw[];  // [n_chunks] chunk weights
   __shared__ PickShared sh;
   const int b = blockIdx.x, tid = threadIdx.x;
@@ -152,8 +155,10 @@ __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundP
 
 // RESIDUAL: w(v) = max(0, Softmax(h_rec)(v) - P_SLM+(v)) on the rejection row, all in double.
 // Runs after the STEER kernel and overrides its result unless the residual has no mass.
-template <typename T>
+template <typename T, int TILE>
 __global__ void __launch_bounds__(kRecThreads) recover_residual_kernel(const RoundParams p) {
+  constexpr int kPerThread = TILE / kRecThreads;
+  constexpr int kTile = TILE;
   extern __shared__ double cw[];  // [n_chunks]
   __shared__ PickShared sh;
   __shared__ double red[2][kRecWarps];
@@ -254,13 +259,13 @@ cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li
   (void)li;
   const size_t smem = (size_t)p.n_chunks * sizeof(double);
   *n_launches = 1;
-  if (dtype == SPECSTEER_F32) recover_steer_kernel<float><<<p.B, kRecThreads, smem, s>>>(p);
-  else recover_steer_kernel<uint16_t><<<p.B, kRecThreads, smem, s>>>(p);
+  if (dtype == SPECSTEER_F32) recover_steer_kernel<float, kTileF32><<<p.B, kRecThreads, smem, s>>>(p);
+  else recover_steer_kernel<uint16_t, kTileBF16><<<p.B, kRecThreads, smem, s>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || p.recover_mode != SPECSTEER_RECOVER_RESIDUAL) return e;
   *n_launches = 2;
-  if (dtype == SPECSTEER_F32) recover_residual_kernel<float><<<p.B, kRecThreads, smem, s>>>(p);
-  else recover_residual_kernel<uint16_t><<<p.B, kRecThreads, smem, s>>>(p);
+  if (dtype == SPECSTEER_F32) recover_residual_kernel<float, kTileF32><<<p.B, kRecThreads, smem, s>>>(p);
+  else recover_residual_kernel<uint16_t, kTileBF16><<<p.B, kRecThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 
