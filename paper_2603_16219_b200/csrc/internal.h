@@ -9,7 +9,7 @@ namespace specsteer {
 constexpr int kTileF32 = 1024;
 constexpr int kTileBF16 = 2048;
 constexpr int kTileMin = 1024;
-constexpr int kMaxSlabB = 4096;  // requests handled by one launch (the per-CTA row prefix lives in shared memory)
+constexpr int kMaxSlabB = 1024;  // requests handled by one launch (per-request tables live in shared memory)
 
 struct RoundParams {
   int B, K, V;

@@ -315,8 +315,11 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 }
 
 // ---- the persistent streaming kernel --------------------------------------------------------------
-template <typename T, int TILE, int STAGES, int NCW, bool BULK>
-__global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundParams p) {
+// Warps [0, NCW) consume tiles; warps [NCW, NCW+NPW) each run one elected producer thread that owns the
+// stages congruent to its index modulo NPW (one thread cannot issue tiles fast enough for a whole SM).
+template <typename T, int TILE, int STAGES, int NCW, int NPW, bool BULK>
+__global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
+  static_assert(STAGES % NPW == 0, "each producer owns a fixed subset of the stages");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int kStageBytes = 3 * TILE * (int)sizeof(T);
   T* tiles = reinterpret_cast<T*>(smem_raw);
@@ -324,14 +327,16 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
   uint64_t* empty = full + STAGES;
   TileMeta* meta = reinterpret_cast<TileMeta*>(empty + STAGES);
   int* abort_flag = reinterpret_cast<int*>(meta + STAGES);
-  int* row_start = abort_flag + 4;  // [B + 1]
+  int* row_start = abort_flag + 4;                           // [B + 1]
+  float* beta_s = reinterpret_cast<float*>(row_start + p.B + 1);  // [B]
+  float* c_s = beta_s + p.B;                                 // [B]  log2(e) / T_b
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int nthreads = (NCW + 1) * 32;
+  constexpr int nthreads = (NCW + NPW) * 32;
   const bool bonus = (p.flags & SPECSTEER_FLAG_BONUS) != 0;
   const int K = p.K;
 
-  // ---- prologue: barriers, and the prefix of used rows per request (draft_len lives on the device)
+  // ---- prologue: barriers, per-request constants, and the prefix of used rows per request
   if (tid == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
     *abort_flag = 0;
@@ -342,6 +347,8 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
     int len = p.draft_len[b];
     if (len < 0 || len > K) len = 0;
     row_start[b + 1] = len + (bonus ? 1 : 0);
+    beta_s[b] = p.beta[b];
+    c_s[b] = kLog2e / p.temperature[b];
   }
   __syncthreads();
   if (warp == 0) {  // inclusive scan, 32 entries at a time
@@ -362,23 +369,29 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
   const int total_tiles = row_start[p.B] * p.n_chunks;  // the host guarantees this fits in 31 bits
   const int cta = blockIdx.x, G = gridDim.x;
 
-  if (warp == NCW) {
-    // ================= producer warp =================
+  if (warp >= NCW) {
+    // ================= producer warps =================
+    const int pw = warp - NCW;
     const T* hl = reinterpret_cast<const T*>(p.h_llm);
     const T* hp = reinterpret_cast<const T*>(p.h_plus);
     const T* hm = reinterpret_cast<const T*>(p.h_minus);
     int issued = 0;
     // tile g = cta + j*G  ->  (compact row cr, chunk); advanced incrementally, no division in the loop
-    const int step_rows = G / p.n_chunks, step_chunks = G % p.n_chunks;
-    int cr = cta / p.n_chunks, chunk = cta % p.n_chunks;
+    const int g0 = cta + pw * G, gstep = NPW * G;
+    const int step_rows = gstep / p.n_chunks, step_chunks = gstep % p.n_chunks;
+    int cr = g0 / p.n_chunks, chunk = g0 % p.n_chunks;
     int b = 0;
     const int K1 = K + 1;
-    for (int j = 0, g = cta; g < total_tiles; ++j, g += G) {
+    for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
       const int stage = j % STAGES;
       const uint32_t phase = (uint32_t)((j / STAGES) & 1);
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(&empty[stage], phase ^ 1u);
-      ok = __shfl_sync(kFullMask, ok ? 1 : 0, 0) != 0;
+      if (BULK) {
+        if (lane == 0) ok = mbar_wait(&empty[stage], phase ^ 1u);
+        ok = __shfl_sync(kFullMask, ok ? 1 : 0, 0) != 0;
+      } else {
+        ok = __all_sync(kFullMask, mbar_wait(&empty[stage], phase ^ 1u));
+      }
       if (!ok || *reinterpret_cast<volatile int*>(abort_flag)) {
         if (lane == 0) { *reinterpret_cast<volatile int*>(abort_flag) = 1; atomicExch(p.dev_error, 1); }
         break;
@@ -390,7 +403,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
       T* dst = tiles + (size_t)stage * 3 * TILE;
       if (BULK) {
         if (lane == 0) {
-          meta[stage] = TileMeta{b * K1 + t, chunk, n_valid, p.beta[b], kLog2e / p.temperature[b]};
+          meta[stage] = TileMeta{b * K1 + t, chunk, n_valid, beta_s[b], c_s[b]};
           const int n_bulk = (int)(((size_t)n_valid * sizeof(T)) & ~(size_t)15) / (int)sizeof(T);
           for (int e = n_bulk; e < n_valid; ++e) {  // ragged end of the last chunk: < 16 bytes per stream
             dst[e] = hl[off + e]; dst[TILE + e] = hp[off + e]; dst[2 * TILE + e] = hm[off + e];
@@ -412,7 +425,7 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
         }
         __syncwarp();
         if (lane == 0) {
-          meta[stage] = TileMeta{b * K1 + t, chunk, n_valid, p.beta[b], kLog2e / p.temperature[b]};
+          meta[stage] = TileMeta{b * K1 + t, chunk, n_valid, beta_s[b], c_s[b]};
           mbar_arrive(&full[stage]);
         }
       }
@@ -423,8 +436,12 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
     // On an abort, copies already issued may still be landing: wait for them (bounded) before the CTA exits.
     __syncwarp();
     if (BULK && lane == 0 && *reinterpret_cast<volatile int*>(abort_flag)) {
-      const int first = issued > STAGES ? issued - STAGES : 0;
-      for (int j = first; j < issued; ++j) mbar_wait(&full[j % STAGES], (uint32_t)((j / STAGES) & 1));
+      constexpr int kOwn = STAGES / NPW;
+      const int first = issued > kOwn ? issued - kOwn : 0;
+      for (int i = first; i < issued; ++i) {
+        const int j = pw + i * NPW;
+        mbar_wait(&full[j % STAGES], (uint32_t)((j / STAGES) & 1));
+      }
     }
   } else {
     // ================= consumer warps =================
@@ -457,20 +474,21 @@ __global__ void __launch_bounds__((NCW + 1) * 32, 1) verify_kernel(const RoundPa
 }
 
 // ---- launch -------------------------------------------------------------------------------------------
-template <typename T, int TILE, int STAGES, int NCW, bool BULK>
+template <typename T, int TILE, int STAGES, int NCW, int NPW, bool BULK>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
-  const size_t smem = (size_t)STAGES * 3 * TILE * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
-                      STAGES * sizeof(TileMeta) + 16 + (size_t)(p.B + 1) * sizeof(int);
-  auto kern = verify_kernel<T, TILE, STAGES, NCW, BULK>;
+  const size_t fixed = (size_t)STAGES * 3 * TILE * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
+                       STAGES * sizeof(TileMeta) + 16;
+  const size_t smem = fixed + (size_t)(3 * p.B + 1) * sizeof(int);
+  auto kern = verify_kernel<T, TILE, STAGES, NCW, NPW, BULK>;
   static bool attr_set_dev[64] = {};  // per instantiation and device; sized for the largest slab
   bool& attr_set = attr_set_dev[li.device & 63];
   if (!attr_set) {
-    const size_t smem_max = smem + (size_t)(kMaxSlabB - p.B) * sizeof(int);
+    const size_t smem_max = fixed + (size_t)(3 * kMaxSlabB + 1) * sizeof(int);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  kern<<<li.sm_count, (NCW + 1) * 32, smem, s>>>(p);
+  kern<<<li.sm_count, (NCW + NPW) * 32, smem, s>>>(p);
   return cudaGetLastError();
 }
 
@@ -479,13 +497,13 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
   *n_launches = 2;
   cudaError_t e;
   if (dtype == SPECSTEER_F32) {
-    e = aligned ? launch_stream<float, kTileF32, 16, 8, true>(p, li, s)
-                : launch_stream<float, kTileF32, 16, 8, false>(p, li, s);
+    e = aligned ? launch_stream<float, kTileF32, 16, 8, 4, true>(p, li, s)
+                : launch_stream<float, kTileF32, 16, 8, 4, false>(p, li, s);
     if (e != cudaSuccess) return e;
     epilogue_kernel<float><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   } else {
-    e = aligned ? launch_stream<uint16_t, kTileBF16, 16, 8, true>(p, li, s)
-                : launch_stream<uint16_t, kTileBF16, 16, 8, false>(p, li, s);
+    e = aligned ? launch_stream<uint16_t, kTileBF16, 16, 8, 4, true>(p, li, s)
+                : launch_stream<uint16_t, kTileBF16, 16, 8, 4, false>(p, li, s);
     if (e != cudaSuccess) return e;
     epilogue_kernel<uint16_t><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   }

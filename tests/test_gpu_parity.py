@@ -154,7 +154,7 @@ def test_many_requests_cross_the_slab_limit(env):
     spec, inputs = _small(env["synth"], 5000, 2, 64, "bf16", seed=6, ragged=True)
     gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
     rng = np.random.default_rng(0)
-    sel = np.sort(np.concatenate([[0, 4095, 4096, 4999], rng.choice(5000, 60, replace=False)]))
+    sel = np.sort(np.concatenate([[0, 1023, 1024, 2047, 2048, 4095, 4096, 4999], rng.choice(5000, 60, replace=False)]))
     sel = np.unique(sel)
     npin = P.to_np_inputs(inputs, torch.as_tensor(sel, device="cuda"))
     P.compare(env["oracle"], gpu, npin, 0, 0, 1, 2e-3, sel=sel)
