@@ -5,4 +5,4 @@ The product is the C-ABI CUDA library under ``csrc/`` (declared in
 ``synth`` manufactures seeded inputs.  Nothing here computes on the CPU: every
 call fails loudly if the CUDA library has not been built.
 """
-__all__ = ["binding", "synth", "build"]
+__all__ = ["binding", "synth", "build", "sharding"]
