@@ -43,7 +43,8 @@ typedef enum {
   SPECSTEER_ERR_WORKSPACE = 3,   /* device allocation failed */
   SPECSTEER_ERR_CUDA = 4,        /* a CUDA runtime call failed (launch error, wrong device) */
   SPECSTEER_ERR_ORDER = 5,       /* recover_sample without a preceding verify_round of the same shape */
-  SPECSTEER_ERR_TIMEOUT = 6      /* a bounded device-side wait gave up (reported by specsteer_ctx_device_error) */
+  SPECSTEER_ERR_TIMEOUT = 6,     /* a bounded device-side wait gave up (reported by specsteer_ctx_device_error) */
+  SPECSTEER_ERR_STATIC_LIMIT = 7 /* specsteer_verify_round_static: the shape does not fit the fixed scratch */
 } specsteer_status;
 
 typedef enum { SPECSTEER_F32 = 0, SPECSTEER_BF16 = 1 } specsteer_dtype;
@@ -136,6 +137,30 @@ specsteer_status specsteer_recover_sample(specsteer_ctx *ctx, const specsteer_ro
  * processed in slabs so that the copy of one slab overlaps the kernels of the previous one.
  * Errors: as the two calls above, plus WORKSPACE. */
 specsteer_status specsteer_round_host(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
+
+/* Verification without a context and without any allocation.  (The paper has no counterpart: this is a
+ * packaging of specsteer_verify_round for hosts that cannot allocate device memory.)
+ *
+ * Who needs it: code that runs where a device allocation is forbidden or harmful - a plug-in inside a
+ * serving process whose memory manager owns the whole device and hands out no more after start-up, a
+ * latency-critical loop that cannot afford the device-wide synchronisation cudaMalloc may imply, or a
+ * process so close to its memory budget that a late allocation could fail.  specsteer_ctx_create allocates
+ * a workspace; this call instead keeps its workspace in a fixed 8 MiB array that is part of the library's
+ * device image, so every GPU that loads the library holds those 8 MiB until the process exits.
+ *
+ * It runs the same two kernels as specsteer_verify_round (same descriptor, same outputs, same error
+ * behaviour, device pointers, the current CUDA device) and calls no cudaMalloc, cudaFree or other allocating
+ * routine.  specsteer_recover_sample needs a context and cannot follow it.
+ *   - Limits: B <= 1024, B*(K+1) <= 16384, and B*(K+1)*ceil(V/C) <= 229376 with C = 1024 for float32 and
+ *     2048 for bf16 logits.  Larger shapes return SPECSTEER_ERR_STATIC_LIMIT and launch nothing.
+ *   - The first call on each device resolves the array's device address (cudaGetSymbolAddress) and reads
+ *     the device's attributes; make that first call outside any stream capture.
+ *   - All calls on a device share the one array.  Nothing in it has to be cleared between calls (every word
+ *     a call reads it has written first), but two calls whose kernels overlap on the GPU - different
+ *     streams, or different host threads - race on it: serialise them.
+ *   - A bounded device-side wait that gives up is not reported by this entry point.
+ * Errors: INVALID_ARG, STATIC_LIMIT, UNSUPPORTED (device index >= 64), CUDA. */
+specsteer_status specsteer_verify_round_static(const specsteer_round_desc *desc, void *cuda_stream);
 
 /* Synchronise the context's device and report whether any kernel of this context gave up a bounded wait:
  * SPECSTEER_OK or SPECSTEER_ERR_TIMEOUT (sticky until the context is destroyed). */

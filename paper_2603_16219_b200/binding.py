@@ -15,7 +15,7 @@ import torch
 from . import build as _build
 
 OK = 0
-ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_ORDER, ERR_TIMEOUT = 1, 2, 3, 4, 5, 6
+ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_ORDER, ERR_TIMEOUT, ERR_STATIC_LIMIT = 1, 2, 3, 4, 5, 6, 7
 F32, BF16 = 0, 1
 ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
 RECOVER_STEER, RECOVER_RESIDUAL = 0, 1
@@ -26,6 +26,7 @@ EXPORTS = (
     "specsteer_ctx_create", "specsteer_ctx_destroy", "specsteer_verify_round", "specsteer_recover_sample",
     "specsteer_round_host", "specsteer_ctx_device_error", "specsteer_ctx_workspace_bytes",
     "specsteer_ctx_launch_count", "specsteer_status_string", "specsteer_version",
+    "specsteer_verify_round_static",
 )
 
 
@@ -69,6 +70,8 @@ def load_library(path: Optional[str] = None):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_void_p]
         fn.restype = C.c_int
+    lib.specsteer_verify_round_static.argtypes = [C.POINTER(RoundDesc), C.c_void_p]
+    lib.specsteer_verify_round_static.restype = C.c_int
     lib.specsteer_ctx_device_error.argtypes = [C.c_void_p]
     lib.specsteer_ctx_device_error.restype = C.c_int
     lib.specsteer_ctx_workspace_bytes.argtypes = [C.c_void_p]
@@ -201,6 +204,19 @@ class Context:
     @property
     def launch_count(self) -> int:
         return int(self._lib.specsteer_ctx_launch_count(self._h))
+
+
+def verify_round_static(desc: RoundDesc, stream=None):
+    """Verification through the entry point that allocates nothing (fixed scratch inside the library).
+
+    For hosts that cannot allocate device memory; runs on the current CUDA device and needs no Context.
+    Raises SpecSteerError(ERR_STATIC_LIMIT) when the shape does not fit the fixed scratch.
+    """
+    if not torch.cuda.is_available():
+        raise RuntimeError("specsteer needs a CUDA device; there is no CPU fallback")
+    s = stream if stream is not None else torch.cuda.current_stream()
+    _check(load_library().specsteer_verify_round_static(C.byref(desc), C.c_void_p(s.cuda_stream)),
+           "specsteer_verify_round_static")
 
 
 def verify_recover_round(ctx: Context, inputs, *, accept_mode=ACCEPT_RATIO, recover_mode=RECOVER_STEER, flags=0,

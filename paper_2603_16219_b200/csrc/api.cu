@@ -354,6 +354,9 @@ const char* specsteer_status_string(specsteer_status s) {
     case SPECSTEER_ERR_CUDA: return "CUDA runtime error";
     case SPECSTEER_ERR_ORDER: return "recover_sample without a matching verify_round";
     case SPECSTEER_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case SPECSTEER_ERR_STATIC_LIMIT:
+      return "shape exceeds the fixed scratch of specsteer_verify_round_static "
+             "(B <= 1024, B*(K+1) <= 16384, B*(K+1)*ceil(V/chunk) <= 229376)";
   }
   return "unknown status";
 }
