@@ -109,7 +109,7 @@ typedef struct {
 
 /* Create a context on CUDA device `device` able to run rounds up to the given maxima.  Allocates the
  * workspace (row normalisers and per-chunk partial sums; about
- * max_B*(max_K+1)*(16 + 32*ceil(max_V/1024)) bytes) once; no later call of the device-pointer entry points allocates.
+ * max_B*(max_K+1)*(16 + 32*ceil(max_V/512)) bytes) once; no later call of the device-pointer entry points allocates.
  * Errors: INVALID_ARG (NULL out, non-positive maxima), CUDA, WORKSPACE. */
 specsteer_status specsteer_ctx_create(specsteer_ctx **out, int device, int32_t max_B, int32_t max_K, int32_t max_V);
 
@@ -151,8 +151,8 @@ specsteer_status specsteer_round_host(specsteer_ctx *ctx, const specsteer_round_
  * It runs the same two kernels as specsteer_verify_round (same descriptor, same outputs, same error
  * behaviour, device pointers, the current CUDA device) and calls no cudaMalloc, cudaFree or other allocating
  * routine.  specsteer_recover_sample needs a context and cannot follow it.
- *   - Limits: B <= 1024, B*(K+1) <= 16384, and B*(K+1)*ceil(V/C) <= 229376 with C = 1024 for float32 and
- *     2048 for bf16 logits.  Larger shapes return SPECSTEER_ERR_STATIC_LIMIT and launch nothing.
+ *   - Limits: B <= 1024, B*(K+1) <= 16384, and B*(K+1)*ceil(V/C) <= 229376 with C = 512 for float32 and
+ *     1024 for bf16 logits.  Larger shapes return SPECSTEER_ERR_STATIC_LIMIT and launch nothing.
  *   - The first call on each device resolves the array's device address (cudaGetSymbolAddress) and reads
  *     the device's attributes; make that first call outside any stream capture.
  *   - All calls on a device share the one array.  Nothing in it has to be cleared between calls (every word

@@ -53,7 +53,7 @@ struct DeviceGuard {
   }
 };
 
-int tile_of(int dtype) { return dtype == SPECSTEER_F32 ? kTileF32 : kTileBF16; }
+int tile_of(int dtype) { return dtype == SPECSTEER_F32 ? kChunkF32 : kChunkBF16; }
 int n_chunks_of(int V, int tile) { return (V + tile - 1) / tile; }
 
 specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
@@ -75,7 +75,7 @@ specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc
   if (d->B > ctx->max_B || d->K > ctx->max_K || d->V > ctx->max_V) return SPECSTEER_ERR_UNSUPPORTED;
   // tiles of one launch are indexed with 31 bits
   const size_t slab_b = d->B < kMaxSlabB ? d->B : kMaxSlabB;
-  if (slab_b * (size_t)(d->K + 1) * (size_t)n_chunks_of(d->V, kTileMin) >= ((size_t)1 << 31)) return SPECSTEER_ERR_UNSUPPORTED;
+  if (slab_b * (size_t)(d->K + 1) * (size_t)n_chunks_of(d->V, kChunkMin) >= ((size_t)1 << 31)) return SPECSTEER_ERR_UNSUPPORTED;
   return SPECSTEER_OK;
 }
 
@@ -164,7 +164,7 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
     return SPECSTEER_ERR_CUDA;
   }
   const size_t rows = (size_t)max_B * (max_K + 1);
-  const size_t nch = (size_t)n_chunks_of(max_V, kTileMin);
+  const size_t nch = (size_t)n_chunks_of(max_V, kChunkMin);
   const size_t b_part = align_up(rows * nch * 8 * sizeof(float), 256);
   const size_t b_lse = align_up(rows * 4 * sizeof(float), 256);
   const size_t b_st = align_up((size_t)max_B * sizeof(int), 256);

@@ -60,26 +60,32 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {
+// One poll of the barrier's phase.  The thread may be suspended by the hardware for up to `hint_ns`
+// nanoseconds (it is woken as soon as the phase completes), so a waiting warp issues few instructions.
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity, uint32_t hint_ns) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(hint_ns)
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up after kWaitPolls polls (each poll may itself block for a short,
-// hardware-defined time) and returns false; the caller then records an error and unwinds.
-constexpr uint32_t kWaitPolls = 1u << 22;
+// Bounded wait: gives up once kWaitCycles SM clocks (a few seconds) have passed and returns false;
+// the caller then records an error and unwinds.
+constexpr long long kWaitCycles = 1ll << 33;
+constexpr uint32_t kSuspendNs = 2000;
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kWaitPolls; ++i) {
-    if (mbar_test(bar, parity)) return true;
-    if (i > 64) __nanosleep(64);
+  if (mbar_test(bar, parity, kSuspendNs)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 256; ++i)
+      if (mbar_test(bar, parity, kSuspendNs)) return true;
+    if (clock64() - t0 > kWaitCycles) return false;
   }
-  return false;
 }
 // 1-D bulk copy global -> shared, completion counted in bytes on `bar`.  No multicast.
 // Both addresses must be 16-byte aligned and `bytes` a multiple of 16.

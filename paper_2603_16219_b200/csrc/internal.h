@@ -5,10 +5,11 @@
 
 namespace specsteer {
 
-// One vocabulary chunk = one tile of the streaming pass = one partial record.  12 KB per stream either way.
-constexpr int kTileF32 = 1024;
-constexpr int kTileBF16 = 2048;
-constexpr int kTileMin = 1024;
+// One vocabulary chunk = what one warp of the streaming pass reduces = one partial record (2 KB per stream).
+// The streaming pass copies tiles of two chunks (4 KB per stream, 12 KB per stage).
+constexpr int kChunkF32 = 512;
+constexpr int kChunkBF16 = 1024;
+constexpr int kChunkMin = 512;
 constexpr int kMaxSlabB = 1024;  // requests handled by one launch (per-request tables live in shared memory)
 
 struct RoundParams {
@@ -16,7 +17,7 @@ struct RoundParams {
   long long ld_row, ld_req;  // elements
   int accept_mode, recover_mode;
   unsigned flags;
-  int tile;      // vocabulary entries per chunk (kTileF32 or kTileBF16)
+  int tile;      // vocabulary entries per chunk (kChunkF32 or kChunkBF16)
   int n_chunks;  // ceil(V / tile)
   const void *h_llm, *h_plus, *h_minus;
   const int* draft_tokens;

@@ -259,13 +259,13 @@ cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li
   (void)li;
   const size_t smem = (size_t)p.n_chunks * sizeof(double);
   *n_launches = 1;
-  if (dtype == SPECSTEER_F32) recover_steer_kernel<float, kTileF32><<<p.B, kRecThreads, smem, s>>>(p);
-  else recover_steer_kernel<uint16_t, kTileBF16><<<p.B, kRecThreads, smem, s>>>(p);
+  if (dtype == SPECSTEER_F32) recover_steer_kernel<float, kChunkF32><<<p.B, kRecThreads, smem, s>>>(p);
+  else recover_steer_kernel<uint16_t, kChunkBF16><<<p.B, kRecThreads, smem, s>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess || p.recover_mode != SPECSTEER_RECOVER_RESIDUAL) return e;
   *n_launches = 2;
-  if (dtype == SPECSTEER_F32) recover_residual_kernel<float, kTileF32><<<p.B, kRecThreads, smem, s>>>(p);
-  else recover_residual_kernel<uint16_t, kTileBF16><<<p.B, kRecThreads, smem, s>>>(p);
+  if (dtype == SPECSTEER_F32) recover_residual_kernel<float, kChunkF32><<<p.B, kRecThreads, smem, s>>>(p);
+  else recover_residual_kernel<uint16_t, kChunkBF16><<<p.B, kRecThreads, smem, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -17,139 +17,210 @@ namespace specsteer {
 constexpr float kSlack = 16.f;  // a lane's reference exponent may lag its running maximum by this much
 
 struct TileMeta {
-  int row, chunk, n_valid;  // padded row index b*(K+1)+t, chunk within the row, valid entries
-  float beta, c;            // beta_b and log2(e)/T_b of the owning request
+  int row, tile, n_valid;  // padded row index b*(K+1)+t, tile within the row, valid entries in the tile
+  float beta, c, inv_c;    // beta_b, log2(e)/T_b and its reciprocal for the owning request
 };
 
-struct Acc {
-  float ref[4];   // integer-valued reference exponent (base 2), -inf while nothing was seen
-  float nref[4];  // -ref, or 0 while empty: the addend of the exponent FMA
-  float s[4];     // sum of 2^(x*c - ref)
-};
-
-__device__ __forceinline__ void acc_init(Acc& a) {
-#pragma unroll
-  for (int q = 0; q < 4; ++q) { a.ref[q] = kNegInf; a.nref[q] = 0.f; a.s[q] = 0.f; }
+// Packed pairs of float32 (sm_100 f32x2 arithmetic): one instruction, two lanes of a 64-bit register.
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float a, float b) {
+  f32x2 r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
+  return r;
 }
+__device__ __forceinline__ void unpack2(f32x2 v, float& a, float& b) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a), "=f"(b) : "l"(v));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {
+  f32x2 d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
+  f32x2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// Reduce four per-lane values over the warp at once (22 instructions instead of 40): after the first
+// two exchange steps each lane carries one of the four quantities.  On return lanes [8q, 8q+8) hold the
+// reduction of v[q] in the return value.
+template <bool IS_MAX>
+__device__ __forceinline__ float warp_reduce4(const float (&v)[4], int lane) {
+  const bool hi16 = (lane & 16) != 0, hi8 = (lane & 8) != 0;
+  const float keep_a = hi16 ? v[2] : v[0], keep_b = hi16 ? v[3] : v[1];
+  const float send_a = hi16 ? v[0] : v[2], send_b = hi16 ? v[1] : v[3];
+  const float xa = __shfl_xor_sync(kFullMask, send_a, 16), xb = __shfl_xor_sync(kFullMask, send_b, 16);
+  const float ra = IS_MAX ? fmaxf(keep_a, xa) : keep_a + xa;
+  const float rb = IS_MAX ? fmaxf(keep_b, xb) : keep_b + xb;
+  const float keep = hi8 ? rb : ra, send = hi8 ? ra : rb;
+  const float x = __shfl_xor_sync(kFullMask, send, 8);
+  float r = IS_MAX ? fmaxf(keep, x) : keep + x;
+#pragma unroll
+  for (int o = 4; o > 0; o >>= 1) {
+    const float y = __shfl_xor_sync(kFullMask, r, o);
+    r = IS_MAX ? fmaxf(r, y) : r + y;
+  }
+  return r;
+}
+
+// A warp's running state for the four normalisers of a chunk (L, P, M and r of Eq. 8).  The reference
+// exponents are the same in every lane; the sums are per lane.
+struct Acc {
+  float ref[4];    // integer-valued reference exponent (base 2), -inf while nothing finite was seen
+  float thr[4];    // (ref + kSlack) / c: a logit above it raises the reference
+  f32x2 nref2[4];  // (-ref, -ref), or (0, 0) while ref is -inf: the addend of the exponent FMA
+  f32x2 s2[4];     // two partial sums of 2^(x*c - ref)
+};
 
 // 2^d for an integer-valued d <= 0 (exact); 0 below the normal range.
 __device__ __forceinline__ float pow2_nonpos_int(float d) {
   return (d < -126.f) ? 0.f : __int_as_float(((int)d + 127) << 23);
 }
 
-__device__ __forceinline__ void acc_raise(Acc& a, int q, float cand) {
-  float nr = fmaxf(a.ref[q], ceilf(cand));
-  if (nr > a.ref[q]) {
-    float f = (a.ref[q] == kNegInf || nr == -kNegInf) ? 0.f : pow2_nonpos_int(a.ref[q] - nr);
-    a.s[q] *= f;
-    a.ref[q] = nr;
-    a.nref[q] = -nr;
-  }
+__device__ __forceinline__ void acc_set_ref(Acc& a, int q, float nr, float inv_c) {
+  a.ref[q] = nr;
+  const float n = (nr > kNegInf) ? -nr : 0.f;  // also 0 for a NaN reference
+  a.nref2[q] = pack2(n, n);
+  a.thr[q] = (nr + kSlack) * inv_c;
 }
 
-__device__ __forceinline__ float sum8(const float (&e)[8]) {
-  return ((e[0] + e[1]) + (e[2] + e[3])) + ((e[4] + e[5]) + (e[6] + e[7]));
-}
-
-// Eight vocabulary entries of the three streams: r = l + beta (p - m)  (Eq. 8), then the four sums.
-template <bool MASKED>
-__device__ __forceinline__ void accum8(Acc& a, float (&l)[8], float (&p)[8], float (&m)[8], float beta, float c,
-                                       unsigned vmask) {
-  float r[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) r[i] = fmaf(beta, p[i] - m[i], l[i]);
-  if (MASKED) {
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-      if (!((vmask >> i) & 1u)) { l[i] = kNegInf; p[i] = kNegInf; m[i] = kNegInf; r[i] = kNegInf; }
-  }
-  const float cl = max8(l) * c, cp = max8(p) * c, cm = max8(m) * c, cr = max8(r) * c;
-  const bool upd = (cl > a.ref[Q_L] + kSlack) | (cp > a.ref[Q_P] + kSlack) | (cm > a.ref[Q_M] + kSlack) |
-                   (cr > a.ref[Q_R] + kSlack);
-  if (__any_sync(kFullMask, upd)) {
-    acc_raise(a, Q_L, cl); acc_raise(a, Q_P, cp); acc_raise(a, Q_M, cm); acc_raise(a, Q_R, cr);
-  }
-  float e[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(l[i], c, a.nref[Q_L]));
-  a.s[Q_L] += sum8(e);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(p[i], c, a.nref[Q_P]));
-  a.s[Q_P] += sum8(e);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(m[i], c, a.nref[Q_M]));
-  a.s[Q_M] += sum8(e);
-#pragma unroll
-  for (int i = 0; i < 8; ++i) e[i] = ex2(fmaf(r[i], c, a.nref[Q_R]));
-  a.s[Q_R] += sum8(e);
-}
-
-// ---- one tile from shared memory, one warp ---------------------------------------------------
-template <typename T, int TILE, bool MASKED> struct TilePass;
-
-template <int TILE, bool MASKED> struct TilePass<float, TILE, MASKED> {
-  static __device__ __forceinline__ void run(Acc& a, const float* sl, const float* sp, const float* sm, int lane,
-                                             int n_valid, float beta, float c) {
-    const float4* vl = reinterpret_cast<const float4*>(sl);
-    const float4* vp = reinterpret_cast<const float4*>(sp);
-    const float4* vm = reinterpret_cast<const float4*>(sm);
-#pragma unroll 2
-    for (int it = 0; it < TILE / 256; ++it) {
-      const int i0 = it * 64 + lane, i1 = i0 + 32;  // two conflict-free 16-byte vectors per stream
-      if (MASKED && it * 256 >= n_valid) break;       // warp-uniform: nothing left for any lane
-      float4 a0 = vl[i0], a1 = vl[i1], b0 = vp[i0], b1 = vp[i1], c0 = vm[i0], c1 = vm[i1];
-      float l[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
-      float p[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
-      float m[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
-      unsigned vmask = 0xffu;
-      if (MASKED) {
-        vmask = 0;
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          if (i0 * 4 + i < n_valid) vmask |= 1u << i;
-          if (i1 * 4 + i < n_valid) vmask |= 1u << (4 + i);
-        }
-      }
-      accum8<MASKED>(a, l, p, m, beta, c, vmask);
-    }
-  }
-};
-
-template <int TILE, bool MASKED> struct TilePass<uint16_t, TILE, MASKED> {
-  static __device__ __forceinline__ void run(Acc& a, const uint16_t* sl, const uint16_t* sp, const uint16_t* sm,
-                                             int lane, int n_valid, float beta, float c) {
-    const uint4* vl = reinterpret_cast<const uint4*>(sl);
-    const uint4* vp = reinterpret_cast<const uint4*>(sp);
-    const uint4* vm = reinterpret_cast<const uint4*>(sm);
-#pragma unroll 2
-    for (int it = 0; it < TILE / 256; ++it) {
-      const int i0 = it * 32 + lane;
-      if (MASKED && it * 256 >= n_valid) break;
-      uint4 a0 = vl[i0], b0 = vp[i0], c0 = vm[i0];
-      float l[8] = {bf16lo(a0.x), bf16hi(a0.x), bf16lo(a0.y), bf16hi(a0.y), bf16lo(a0.z), bf16hi(a0.z), bf16lo(a0.w), bf16hi(a0.w)};
-      float p[8] = {bf16lo(b0.x), bf16hi(b0.x), bf16lo(b0.y), bf16hi(b0.y), bf16lo(b0.z), bf16hi(b0.z), bf16lo(b0.w), bf16hi(b0.w)};
-      float m[8] = {bf16lo(c0.x), bf16hi(c0.x), bf16lo(c0.y), bf16hi(c0.y), bf16lo(c0.z), bf16hi(c0.z), bf16lo(c0.w), bf16hi(c0.w)};
-      unsigned vmask = 0xffu;
-      if (MASKED) {
-        vmask = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          if (i0 * 8 + i < n_valid) vmask |= 1u << i;
-      }
-      accum8<MASKED>(a, l, p, m, beta, c, vmask);
-    }
-  }
-};
-
-// Combine the lanes' pairs into one (reference, sum) per normaliser; every lane gets the result.
-__device__ __forceinline__ void warp_combine(Acc& a) {
+// First batch of a chunk: the references come from the warp-wide maxima of this batch.
+__device__ __forceinline__ void acc_start(Acc& a, const float (&bm)[4], float c, float inv_c, int lane) {
+  const float mine = warp_reduce4<true>(bm, lane);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    const float M = warp_max(a.ref[q]);
-    float s = a.s[q];
-    if (a.ref[q] != M) s = (a.ref[q] == kNegInf || M == -kNegInf) ? 0.f : s * pow2_nonpos_int(a.ref[q] - M);
-    a.s[q] = warp_sum(s);
-    a.ref[q] = M;
+    acc_set_ref(a, q, ceilf(__shfl_sync(kFullMask, mine, 8 * q) * c), inv_c);
+    a.s2[q] = 0ull;
+  }
+}
+
+// A later batch holds a logit above a threshold: raise the references (rarely taken).
+__device__ __forceinline__ void acc_raise(Acc& a, const float (&bm)[4], float c, float inv_c, int lane) {
+  const float mine = warp_reduce4<true>(bm, lane);
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const float nr = fmaxf(a.ref[q], ceilf(__shfl_sync(kFullMask, mine, 8 * q) * c));
+    if (nr > a.ref[q]) {
+      const float f = (a.ref[q] == kNegInf || nr == -kNegInf) ? 0.f : pow2_nonpos_int(a.ref[q] - nr);
+      a.s2[q] = mul2(a.s2[q], pack2(f, f));
+      acc_set_ref(a, q, nr, inv_c);
+    }
+  }
+}
+
+__device__ __forceinline__ float max8(const f32x2 (&v)[4]) {
+  float x[8];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) unpack2(v[i], x[2 * i], x[2 * i + 1]);
+  return fmaxf(max3(max3(x[0], x[1], x[2]), max3(x[3], x[4], x[5]), x[6]), x[7]);
+}
+
+// sum += 2^(x*c - ref) over eight entries of one stream
+__device__ __forceinline__ void exp_sum8(f32x2& s2, const f32x2 (&x)[4], f32x2 c2, f32x2 nref2) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a0, a1;
+    unpack2(fma2(x[i], c2, nref2), a0, a1);
+    s2 = add2(s2, pack2(ex2(a0), ex2(a1)));
+  }
+}
+
+// Eight vocabulary entries per lane of the three streams: r = l + beta (p - m)  (Eq. 8), then the four sums.
+template <bool MASKED, bool FIRST>
+__device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32x2 (&m)[4], f32x2 beta2, f32x2 c2,
+                                       float c, float inv_c, unsigned vmask, int lane) {
+  f32x2 r[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
+  if (MASKED) {
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const bool k0 = (vmask >> (2 * i)) & 1u, k1 = (vmask >> (2 * i + 1)) & 1u;
+      if (!(k0 && k1)) {
+        float x0, x1;
+        unpack2(l[i], x0, x1); l[i] = pack2(k0 ? x0 : kNegInf, k1 ? x1 : kNegInf);
+        unpack2(p[i], x0, x1); p[i] = pack2(k0 ? x0 : kNegInf, k1 ? x1 : kNegInf);
+        unpack2(m[i], x0, x1); m[i] = pack2(k0 ? x0 : kNegInf, k1 ? x1 : kNegInf);
+        unpack2(r[i], x0, x1); r[i] = pack2(k0 ? x0 : kNegInf, k1 ? x1 : kNegInf);
+      }
+    }
+  }
+  const float bm[4] = {max8(l), max8(p), max8(m), max8(r)};  // order of Q_L, Q_P, Q_M, Q_R
+  if (FIRST) {
+    acc_start(a, bm, c, inv_c, lane);
+  } else {
+    const bool upd = (bm[0] > a.thr[0]) | (bm[1] > a.thr[1]) | (bm[2] > a.thr[2]) | (bm[3] > a.thr[3]);
+    if (__any_sync(kFullMask, upd)) acc_raise(a, bm, c, inv_c, lane);
+  }
+  exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+  exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+  exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+  exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+}
+
+// ---- one chunk (half a tile) from shared memory, one warp ---------------------------------------
+template <typename T> struct Batch;
+
+template <> struct Batch<float> {
+  // batch `it` of a chunk: two conflict-free 16-byte vectors per stream and lane (entries 4*i0.., 4*i1..)
+  static __device__ __forceinline__ void load(const float* s, int it, int lane, f32x2 (&x)[4]) {
+    const ulonglong2* v = reinterpret_cast<const ulonglong2*>(s);
+    const ulonglong2 a0 = v[it * 64 + lane], a1 = v[it * 64 + 32 + lane];
+    x[0] = a0.x; x[1] = a0.y; x[2] = a1.x; x[3] = a1.y;
+  }
+  static __device__ __forceinline__ unsigned mask(int it, int lane, int n_valid) {
+    unsigned vm = 0;
+    const int e0 = (it * 64 + lane) * 4, e1 = e0 + 128;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      if (e0 + i < n_valid) vm |= 1u << i;
+      if (e1 + i < n_valid) vm |= 1u << (4 + i);
+    }
+    return vm;
+  }
+};
+
+template <> struct Batch<uint16_t> {
+  static __device__ __forceinline__ void load(const uint16_t* s, int it, int lane, f32x2 (&x)[4]) {
+    const uint4 a = reinterpret_cast<const uint4*>(s)[it * 32 + lane];
+    x[0] = pack2(bf16lo(a.x), bf16hi(a.x)); x[1] = pack2(bf16lo(a.y), bf16hi(a.y));
+    x[2] = pack2(bf16lo(a.z), bf16hi(a.z)); x[3] = pack2(bf16lo(a.w), bf16hi(a.w));
+  }
+  static __device__ __forceinline__ unsigned mask(int it, int lane, int n_valid) {
+    unsigned vm = 0;
+    const int e0 = (it * 32 + lane) * 8;
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+      if (e0 + i < n_valid) vm |= 1u << i;
+    return vm;
+  }
+};
+
+template <typename T, int CHUNK, bool MASKED>
+__device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, const T* sm, int lane, int n_valid,
+                                           float beta, float c, float inv_c) {
+  const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
+#pragma unroll
+  for (int it = 0; it < CHUNK / 256; ++it) {
+    if (MASKED && it > 0 && it * 256 >= n_valid) break;  // warp-uniform: nothing left for any lane
+    f32x2 l[4], p[4], m[4];
+    Batch<T>::load(sl, it, lane, l);
+    Batch<T>::load(sp, it, lane, p);
+    Batch<T>::load(sm, it, lane, m);
+    const unsigned vmask = MASKED ? Batch<T>::mask(it, lane, n_valid) : 0xffu;
+    if (it == 0) accum8<MASKED, true>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
+    else accum8<MASKED, false>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
   }
 }
 
@@ -315,10 +386,17 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 }
 
 // ---- the persistent streaming kernel --------------------------------------------------------------
-// Warps [0, NCW) consume tiles; warps [NCW, NCW+NPW) each run one elected producer thread that owns the
-// stages congruent to its index modulo NPW (one thread cannot issue tiles fast enough for a whole SM).
-template <typename T, int TILE, int STAGES, int NCW, int NPW, bool BULK>
+// A tile is 2*CHUNK vocabulary entries of one used row, all three streams (three bulk copies, one stage).
+// Warps [0, NCW) consume: warps 2k and 2k+1 share the tiles congruent to k modulo NCW/2 and each reduces
+// one chunk (half) of the tile into its own partial record.  Warps [NCW, NCW+NPW) each run one elected
+// producer thread that owns the stages congruent to its index modulo NPW (one thread cannot issue tiles
+// fast enough for a whole SM).  Every stage is always consumed by the same pair of warps, so a waiting
+// warp is never a whole barrier phase ahead of the data.
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
+  constexpr int TILE = 2 * CHUNK;
+  constexpr int NPAIR = NCW / 2;
+  static_assert(NCW % 2 == 0 && STAGES % NPAIR == 0, "each stage belongs to one fixed pair of consumer warps");
   static_assert(STAGES % NPW == 0, "each producer owns a fixed subset of the stages");
   extern __shared__ __align__(128) unsigned char smem_raw[];
   constexpr int kStageBytes = 3 * TILE * (int)sizeof(T);
@@ -327,18 +405,20 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   uint64_t* empty = full + STAGES;
   TileMeta* meta = reinterpret_cast<TileMeta*>(empty + STAGES);
   int* abort_flag = reinterpret_cast<int*>(meta + STAGES);
-  int* row_start = abort_flag + 4;                           // [B + 1]
+  int* row_start = abort_flag + 4;                                // [B + 1]
   float* beta_s = reinterpret_cast<float*>(row_start + p.B + 1);  // [B]
-  float* c_s = beta_s + p.B;                                 // [B]  log2(e) / T_b
+  float* c_s = beta_s + p.B;                                      // [B]  log2(e) / T_b
+  float* ic_s = c_s + p.B;                                        // [B]  T_b / log2(e)
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int nthreads = (NCW + NPW) * 32;
   const bool bonus = (p.flags & SPECSTEER_FLAG_BONUS) != 0;
   const int K = p.K;
+  const int tiles_per_row = (p.V + TILE - 1) / TILE;
 
   // ---- prologue: barriers, per-request constants, and the prefix of used rows per request
   if (tid == 0) {
-    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 2); }
     *abort_flag = 0;
     row_start[0] = 0;
     fence_barrier_init();
@@ -349,6 +429,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
     row_start[b + 1] = len + (bonus ? 1 : 0);
     beta_s[b] = p.beta[b];
     c_s[b] = kLog2e / p.temperature[b];
+    ic_s[b] = p.temperature[b] * kLn2;
   }
   __syncthreads();
   if (warp == 0) {  // inclusive scan, 32 entries at a time
@@ -366,7 +447,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
     }
   }
   __syncthreads();
-  const int total_tiles = row_start[p.B] * p.n_chunks;  // the host guarantees this fits in 31 bits
+  const int total_tiles = row_start[p.B] * tiles_per_row;  // the host guarantees this fits in 31 bits
   const int cta = blockIdx.x, G = gridDim.x;
 
   if (warp >= NCW) {
@@ -375,37 +456,31 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
     const T* hl = reinterpret_cast<const T*>(p.h_llm);
     const T* hp = reinterpret_cast<const T*>(p.h_plus);
     const T* hm = reinterpret_cast<const T*>(p.h_minus);
-    int issued = 0;
-    // tile g = cta + j*G  ->  (compact row cr, chunk); advanced incrementally, no division in the loop
+    // tile g = cta + j*G  ->  (compact row cr, tile in row); advanced incrementally, no division in the loop
     const int g0 = cta + pw * G, gstep = NPW * G;
-    const int step_rows = gstep / p.n_chunks, step_chunks = gstep % p.n_chunks;
-    int cr = g0 / p.n_chunks, chunk = g0 % p.n_chunks;
+    const int step_rows = gstep / tiles_per_row, step_tiles = gstep % tiles_per_row;
+    int cr = g0 / tiles_per_row, tr = g0 % tiles_per_row;
     int b = 0;
     const int K1 = K + 1;
-    for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
-      const int stage = j % STAGES;
-      const uint32_t phase = (uint32_t)((j / STAGES) & 1);
-      bool ok = true;
-      if (BULK) {
-        if (lane == 0) ok = mbar_wait(&empty[stage], phase ^ 1u);
-        ok = __shfl_sync(kFullMask, ok ? 1 : 0, 0) != 0;
-      } else {
-        ok = __all_sync(kFullMask, mbar_wait(&empty[stage], phase ^ 1u));
-      }
-      if (!ok || *reinterpret_cast<volatile int*>(abort_flag)) {
-        if (lane == 0) { *reinterpret_cast<volatile int*>(abort_flag) = 1; atomicExch(p.dev_error, 1); }
-        break;
-      }
-      while (row_start[b + 1] <= cr) ++b;  // cr < row_start[B], so b stays below B
-      const int t = cr - row_start[b];
-      const int n_valid = min(TILE, p.V - chunk * TILE);
-      const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)chunk * TILE;
-      T* dst = tiles + (size_t)stage * 3 * TILE;
-      if (BULK) {
-        if (lane == 0) {
-          meta[stage] = TileMeta{b * K1 + t, chunk, n_valid, beta_s[b], c_s[b]};
+    if (BULK) {
+      if (lane == 0) {  // one elected thread issues the bulk copies
+        int issued = 0;
+        for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
+          const int stage = j % STAGES;
+          const uint32_t phase = (uint32_t)((j / STAGES) & 1);
+          if (*reinterpret_cast<volatile int*>(abort_flag) || !mbar_wait(&empty[stage], phase ^ 1u)) {
+            *reinterpret_cast<volatile int*>(abort_flag) = 1;
+            atomicExch(p.dev_error, 1);
+            break;
+          }
+          while (row_start[b + 1] <= cr) ++b;  // cr < row_start[B], so b stays below B
+          const int t = cr - row_start[b];
+          const int n_valid = min(TILE, p.V - tr * TILE);
+          const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)tr * TILE;
+          T* dst = tiles + (size_t)stage * 3 * TILE;
+          meta[stage] = TileMeta{b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b]};
           const int n_bulk = (int)(((size_t)n_valid * sizeof(T)) & ~(size_t)15) / (int)sizeof(T);
-          for (int e = n_bulk; e < n_valid; ++e) {  // ragged end of the last chunk: < 16 bytes per stream
+          for (int e = n_bulk; e < n_valid; ++e) {  // ragged end of the last tile: < 16 bytes per stream
             dst[e] = hl[off + e]; dst[TILE + e] = hp[off + e]; dst[2 * TILE + e] = hm[off + e];
           }
           const uint32_t bytes = (uint32_t)(n_bulk * sizeof(T));
@@ -417,35 +492,51 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
           } else {
             mbar_arrive(&full[stage]);
           }
+          ++issued;
+          cr += step_rows; tr += step_tiles;
+          if (tr >= tiles_per_row) { tr -= tiles_per_row; ++cr; }
         }
-      } else {
-        // rows that are not 16-byte aligned: the warp copies element by element
+        // On an abort, copies already issued may still be landing: wait for them (bounded) before the CTA exits.
+        if (*reinterpret_cast<volatile int*>(abort_flag)) {
+          constexpr int kOwn = STAGES / NPW;
+          const int first = issued > kOwn ? issued - kOwn : 0;
+          for (int i = first; i < issued; ++i) {
+            const int j = pw + i * NPW;
+            mbar_wait(&full[j % STAGES], (uint32_t)((j / STAGES) & 1));
+          }
+        }
+      }
+    } else {
+      // rows that are not 16-byte aligned: the warp copies element by element
+      for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
+        const int stage = j % STAGES;
+        const uint32_t phase = (uint32_t)((j / STAGES) & 1);
+        const bool ok = __all_sync(kFullMask, mbar_wait(&empty[stage], phase ^ 1u));
+        if (!ok || *reinterpret_cast<volatile int*>(abort_flag)) {
+          if (lane == 0) { *reinterpret_cast<volatile int*>(abort_flag) = 1; atomicExch(p.dev_error, 1); }
+          break;
+        }
+        while (row_start[b + 1] <= cr) ++b;
+        const int t = cr - row_start[b];
+        const int n_valid = min(TILE, p.V - tr * TILE);
+        const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)tr * TILE;
+        T* dst = tiles + (size_t)stage * 3 * TILE;
         for (int e = lane; e < n_valid; e += 32) {
           dst[e] = hl[off + e]; dst[TILE + e] = hp[off + e]; dst[2 * TILE + e] = hm[off + e];
         }
         __syncwarp();
         if (lane == 0) {
-          meta[stage] = TileMeta{b * K1 + t, chunk, n_valid, beta_s[b], c_s[b]};
+          meta[stage] = TileMeta{b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b]};
           mbar_arrive(&full[stage]);
         }
-      }
-      ++issued;
-      cr += step_rows; chunk += step_chunks;
-      if (chunk >= p.n_chunks) { chunk -= p.n_chunks; ++cr; }
-    }
-    // On an abort, copies already issued may still be landing: wait for them (bounded) before the CTA exits.
-    __syncwarp();
-    if (BULK && lane == 0 && *reinterpret_cast<volatile int*>(abort_flag)) {
-      constexpr int kOwn = STAGES / NPW;
-      const int first = issued > kOwn ? issued - kOwn : 0;
-      for (int i = first; i < issued; ++i) {
-        const int j = pw + i * NPW;
-        mbar_wait(&full[j % STAGES], (uint32_t)((j / STAGES) & 1));
+        cr += step_rows; tr += step_tiles;
+        if (tr >= tiles_per_row) { tr -= tiles_per_row; ++cr; }
       }
     }
   } else {
     // ================= consumer warps =================
-    for (int j = warp, g = cta + warp * G; g < total_tiles; j += NCW, g += NCW * G) {
+    const int pair = warp >> 1, half = warp & 1;
+    for (int j = pair, g = cta + pair * G; g < total_tiles; j += NPAIR, g += NPAIR * G) {
       const int stage = j % STAGES;
       const uint32_t phase = (uint32_t)((j / STAGES) & 1);
       // every lane observes the phase itself: that is what makes the copied bytes visible to it
@@ -456,34 +547,44 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
         break;
       }
       const TileMeta mt = meta[stage];
-      const T* sl = tiles + (size_t)stage * 3 * TILE;
+      const int nv = mt.n_valid - half * CHUNK;  // valid entries in this warp's chunk
+      const T* sl = tiles + (size_t)stage * 3 * TILE + half * CHUNK;
       Acc a;
-      acc_init(a);
-      if (mt.n_valid == TILE) TilePass<T, TILE, false>::run(a, sl, sl + TILE, sl + 2 * TILE, lane, TILE, mt.beta, mt.c);
-      else TilePass<T, TILE, true>::run(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.n_valid, mt.beta, mt.c);
+      if (nv >= CHUNK) chunk_pass<T, CHUNK, false>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
+      else if (nv > 0) chunk_pass<T, CHUNK, true>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);  // the stage may be refilled while we reduce
-      warp_combine(a);
-      if (lane == 0) {
-        float* rec = p.part + ((long long)mt.row * p.n_chunks + mt.chunk) * 8;
-        *reinterpret_cast<float4*>(rec) = make_float4(a.ref[Q_L], a.s[Q_L], a.ref[Q_P], a.s[Q_P]);
-        *reinterpret_cast<float4*>(rec + 4) = make_float4(a.ref[Q_M], a.s[Q_M], a.ref[Q_R], a.s[Q_R]);
+      if (nv > 0) {
+        float s4[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          float s0, s1;
+          unpack2(a.s2[q], s0, s1);
+          s4[q] = s0 + s1;
+        }
+        const float tot = warp_reduce4<false>(s4, lane);  // lanes [8q, 8q+8) hold the sum of normaliser q
+        if ((lane & 7) == 0) {
+          const int q = lane >> 3;
+          const float rq = q == 0 ? a.ref[0] : (q == 1 ? a.ref[1] : (q == 2 ? a.ref[2] : a.ref[3]));
+          float* rec = p.part + ((long long)mt.row * p.n_chunks + (mt.tile * 2 + half)) * 8;
+          *reinterpret_cast<float2*>(rec + 2 * q) = make_float2(rq, tot);
+        }
       }
     }
   }
 }
 
 // ---- launch -------------------------------------------------------------------------------------------
-template <typename T, int TILE, int STAGES, int NCW, int NPW, bool BULK>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
-  const size_t fixed = (size_t)STAGES * 3 * TILE * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
+  const size_t fixed = (size_t)STAGES * 3 * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
                        STAGES * sizeof(TileMeta) + 16;
-  const size_t smem = fixed + (size_t)(3 * p.B + 1) * sizeof(int);
-  auto kern = verify_kernel<T, TILE, STAGES, NCW, NPW, BULK>;
+  const size_t smem = fixed + (size_t)(4 * p.B + 1) * sizeof(int);
+  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK>;
   static bool attr_set_dev[64] = {};  // per instantiation and device; sized for the largest slab
   bool& attr_set = attr_set_dev[li.device & 63];
   if (!attr_set) {
-    const size_t smem_max = fixed + (size_t)(3 * kMaxSlabB + 1) * sizeof(int);
+    const size_t smem_max = fixed + (size_t)(4 * kMaxSlabB + 1) * sizeof(int);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
     attr_set = true;
@@ -497,13 +598,13 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
   *n_launches = 2;
   cudaError_t e;
   if (dtype == SPECSTEER_F32) {
-    e = aligned ? launch_stream<float, kTileF32, 16, 8, 4, true>(p, li, s)
-                : launch_stream<float, kTileF32, 16, 8, 4, false>(p, li, s);
+    e = aligned ? launch_stream<float, kChunkF32, 16, 16, 4, true>(p, li, s)
+                : launch_stream<float, kChunkF32, 16, 16, 4, false>(p, li, s);
     if (e != cudaSuccess) return e;
     epilogue_kernel<float><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   } else {
-    e = aligned ? launch_stream<uint16_t, kTileBF16, 16, 8, 4, true>(p, li, s)
-                : launch_stream<uint16_t, kTileBF16, 16, 8, 4, false>(p, li, s);
+    e = aligned ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true>(p, li, s)
+                : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false>(p, li, s);
     if (e != cudaSuccess) return e;
     epilogue_kernel<uint16_t><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   }
