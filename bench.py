@@ -26,8 +26,10 @@ METRIC = "verified_draft_positions_per_sec"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0
 NOMINAL_HBM_GBS = 8000.0
-# DRAM bytes per launch of the streaming kernel from ncu (profiles/), keyed by configuration; None = not captured
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes (read + write) per used row of the streaming kernel, from the ncu captures summarised under
+# profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows), keyed by
+# configuration.  Absent = not captured for the kernel as it stands.
+NCU_TRAFFIC_BYTES_PER_ROW = {3: 1852523, 4: 1559272}
 
 
 def _peaks():
@@ -226,16 +228,20 @@ def run_cuda(args, rank, world, local_rank):
     sampler.window(w0, w1)
     gpu_launches = ctx.launch_count - launches0
     total_ms = e0.elapsed_time(e1)
-    # ---- timed region 2: the streaming kernel alone, one event pair per launch (same warm state)
+    # ---- timed region 2: the streaming kernel alone; the library records one event pair per launch around it
     ksteps = min(args.steps, 200)
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(ksteps)]
+    for a, b in evs:            # a first record creates the CUDA handles the hook needs
+        a.record(stream)
+        b.record(stream)
+    torch.cuda.synchronize(dev)
     w0 = time.perf_counter()
     for i in range(ksteps):
         d = sets[i % n_sets][1]
-        evs[i][0].record(stream)
+        ctx.time_streaming(*evs[i])
         ctx.verify_round(d, stream)
-        evs[i][1].record(stream)
         ctx.recover_sample(d, stream)
+    ctx.time_streaming(None, None)
     barrier()
     sampler.window(w0, time.perf_counter())
     kernel_ms = sum(a.elapsed_time(b) for a, b in evs) / ksteps
@@ -293,7 +299,8 @@ def run_cuda(args, rank, world, local_rank):
     achieved = logit_bytes / (kernel_ms * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": "verify_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-        "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": NCU_TRAFFIC_BYTES.get(args.config),
+        "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.config] * rows if args.config in NCU_TRAFFIC_BYTES_PER_ROW
+                    and not args.requests else None),
         "algorithmic_bytes_per_launch": logit_bytes, "kernel_ms": kernel_ms,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "whole_step_gbs": logit_bytes / (ms_per_step * 1e-3) / 1e9,

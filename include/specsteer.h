@@ -166,6 +166,14 @@ specsteer_status specsteer_verify_round_static(const specsteer_round_desc *desc,
  * SPECSTEER_OK or SPECSTEER_ERR_TIMEOUT (sticky until the context is destroyed). */
 specsteer_status specsteer_ctx_device_error(specsteer_ctx *ctx);
 
+/* Profiling hook: from now on specsteer_verify_round records the two caller-owned CUDA events (cudaEvent_t
+ * passed as void*, created with timing enabled) on its stream just before and just after the streaming
+ * kernel, the launch that reads all the logits, so that a benchmark can time that kernel alone; the per-request
+ * epilogue kernel follows the second event.  With more than 1024 requests the round runs in several slabs and
+ * the events bracket everything from the first slab's streaming kernel to the last one's.  Pass two NULLs to
+ * switch the hook off.  Errors: INVALID_ARG (NULL ctx, or only one event given). */
+specsteer_status specsteer_ctx_time_streaming(specsteer_ctx *ctx, void *ev_begin, void *ev_end);
+
 /* Bytes of device workspace owned by the context. */
 size_t specsteer_ctx_workspace_bytes(const specsteer_ctx *ctx);
 

@@ -26,7 +26,7 @@ EXPORTS = (
     "specsteer_ctx_create", "specsteer_ctx_destroy", "specsteer_verify_round", "specsteer_recover_sample",
     "specsteer_round_host", "specsteer_ctx_device_error", "specsteer_ctx_workspace_bytes",
     "specsteer_ctx_launch_count", "specsteer_status_string", "specsteer_version",
-    "specsteer_verify_round_static",
+    "specsteer_verify_round_static", "specsteer_ctx_time_streaming",
 )
 
 
@@ -76,6 +76,8 @@ def load_library(path: Optional[str] = None):
     lib.specsteer_ctx_device_error.restype = C.c_int
     lib.specsteer_ctx_workspace_bytes.argtypes = [C.c_void_p]
     lib.specsteer_ctx_workspace_bytes.restype = C.c_size_t
+    lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.specsteer_ctx_time_streaming.restype = C.c_int
     lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
     lib.specsteer_ctx_launch_count.restype = C.c_uint64
     lib.specsteer_status_string.argtypes = [C.c_int]
@@ -193,6 +195,14 @@ class Context:
 
     def round_host(self, desc: RoundDesc, stream=None):
         _check(self._lib.specsteer_round_host(self._h, C.byref(desc), self._stream(stream)), "specsteer_round_host")
+
+    def time_streaming(self, ev_begin=None, ev_end=None):
+        """Record two timing-enabled torch.cuda.Event objects around the streaming kernel of every later
+        verify_round (None, None switches it off).  The events must have been recorded once already so that
+        their CUDA handles exist."""
+        a = C.c_void_p(ev_begin.cuda_event) if ev_begin is not None else None
+        b = C.c_void_p(ev_end.cuda_event) if ev_end is not None else None
+        _check(self._lib.specsteer_ctx_time_streaming(self._h, a, b), "specsteer_ctx_time_streaming")
 
     def device_error(self) -> int:
         return int(self._lib.specsteer_ctx_device_error(self._h))

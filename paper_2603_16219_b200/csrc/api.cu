@@ -32,6 +32,8 @@ struct specsteer_ctx {
   cudaStream_t copy_stream;
   cudaEvent_t ev_copied[2], ev_done[2];
   bool host_ready;
+  // optional timing hooks around the streaming kernel (caller-owned events)
+  cudaEvent_t ev_stream_begin, ev_stream_end;
 };
 
 static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
@@ -124,7 +126,10 @@ specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cu
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
     RoundParams p = slab_params(ctx, d, b0, nb);
     int nl = 0;
-    if (launch_verify(p, d->dtype, aligned, ctx->li, s, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    const bool first = b0 == 0, last = b0 + nb >= d->B;
+    if (launch_verify(p, d->dtype, aligned, ctx->li, s, &nl, first ? ctx->ev_stream_begin : nullptr,
+                      last ? ctx->ev_stream_end : nullptr) != cudaSuccess)
+      return SPECSTEER_ERR_CUDA;
     ctx->launches += nl;
   }
   return SPECSTEER_OK;
@@ -340,6 +345,13 @@ specsteer_status specsteer_ctx_device_error(specsteer_ctx* ctx) {
   if (cudaMemcpy(&flag, ctx->dev_error, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (flag) ctx->poisoned = true;
   return flag ? SPECSTEER_ERR_TIMEOUT : SPECSTEER_OK;
+}
+
+specsteer_status specsteer_ctx_time_streaming(specsteer_ctx* ctx, void* ev_begin, void* ev_end) {
+  if (!ctx || ((ev_begin == nullptr) != (ev_end == nullptr))) return SPECSTEER_ERR_INVALID_ARG;
+  ctx->ev_stream_begin = (cudaEvent_t)ev_begin;
+  ctx->ev_stream_end = (cudaEvent_t)ev_end;
+  return SPECSTEER_OK;
 }
 
 size_t specsteer_ctx_workspace_bytes(const specsteer_ctx* ctx) { return ctx ? ctx->ws_bytes : 0; }

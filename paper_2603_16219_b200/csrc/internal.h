@@ -44,8 +44,9 @@ struct LaunchInfo {
   int max_smem_optin;
 };
 
+// ev_begin / ev_end, when not null, are recorded on `s` just before and just after the streaming kernel.
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
-                          int* n_launches);
+                          int* n_launches, cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);
 
 }  // namespace specsteer

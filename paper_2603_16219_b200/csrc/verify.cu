@@ -594,20 +594,21 @@ static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cud
 }
 
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
-                          int* n_launches) {
+                          int* n_launches, cudaEvent_t ev_begin, cudaEvent_t ev_end) {
   *n_launches = 2;
   cudaError_t e;
+  if (ev_begin && (e = cudaEventRecord(ev_begin, s)) != cudaSuccess) return e;
   if (dtype == SPECSTEER_F32) {
     e = aligned ? launch_stream<float, kChunkF32, 16, 16, 4, true>(p, li, s)
                 : launch_stream<float, kChunkF32, 16, 16, 4, false>(p, li, s);
-    if (e != cudaSuccess) return e;
-    epilogue_kernel<float><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   } else {
     e = aligned ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true>(p, li, s)
                 : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false>(p, li, s);
-    if (e != cudaSuccess) return e;
-    epilogue_kernel<uint16_t><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   }
+  if (e != cudaSuccess) return e;
+  if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;
+  if (dtype == SPECSTEER_F32) epilogue_kernel<float><<<p.B, kEpiWarps * 32, 0, s>>>(p);
+  else epilogue_kernel<uint16_t><<<p.B, kEpiWarps * 32, 0, s>>>(p);
   return cudaGetLastError();
 }
 
