@@ -14,6 +14,10 @@
 
 namespace specsteer {
 
+#ifndef SPECSTEER_POLY_PAIRS_BF16
+#define SPECSTEER_POLY_PAIRS_BF16 4
+#endif
+constexpr int kPolyPairsBF16 = SPECSTEER_POLY_PAIRS_BF16;
 constexpr float kSlack = 16.f;  // a lane's reference exponent may lag its running maximum by this much
 
 struct TileMeta {
@@ -95,12 +99,13 @@ __device__ __forceinline__ void acc_set_ref(Acc& a, int q, float nr, float inv_c
   a.thr[q] = (nr + kSlack) * inv_c;
 }
 
-// First batch of a chunk: the references come from the warp-wide maxima of this batch.
-__device__ __forceinline__ void acc_start(Acc& a, const float (&bm)[4], float c, float inv_c, int lane) {
+// First batch of a chunk: the references come from the warp-wide maxima of this batch, plus `bias`.
+__device__ __forceinline__ void acc_start(Acc& a, const float (&bm)[4], float c, float inv_c, int lane,
+                                          float bias = 0.f) {
   const float mine = warp_reduce4<true>(bm, lane);
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    acc_set_ref(a, q, ceilf(__shfl_sync(kFullMask, mine, 8 * q) * c), inv_c);
+    acc_set_ref(a, q, ceilf(__shfl_sync(kFullMask, mine, 8 * q) * c) + bias, inv_c);
     a.s2[q] = 0ull;
   }
 }
@@ -126,13 +131,44 @@ __device__ __forceinline__ float max8(const f32x2 (&v)[4]) {
   return fmaxf(max3(max3(x[0], x[1], x[2]), max3(x[3], x[4], x[5]), x[6]), x[7]);
 }
 
-// sum += 2^(x*c - ref) over eight entries of one stream
+// 2^a for a pair of arguments a < 127.5 on the FMA pipe (no special-function unit): a is clamped to
+// >= -126, split into round(a) + f with f in [-0.5, 0.5] by the 1.5*2^23 trick, 2^f is a degree-5
+// polynomial (relative error 2.1e-7 in float32 Horner form), and round(a) is added to the exponent field.
+__device__ __forceinline__ f32x2 exp2_poly2(f32x2 a) {
+  const float kMagic = 12582912.f;  // 1.5 * 2^23
+  float a0, a1;
+  unpack2(a, a0, a1);
+  const f32x2 ac = pack2(fmaxf(a0, -126.f), fmaxf(a1, -126.f));
+  const f32x2 magic2 = pack2(kMagic, kMagic);
+  const f32x2 t = add2(ac, magic2);
+  const f32x2 f = sub2(ac, sub2(t, magic2));
+  f32x2 q = pack2(0.001327645150013268f, 0.001327645150013268f);
+  q = fma2(q, f, pack2(0.009675540030002594f, 0.009675540030002594f));
+  q = fma2(q, f, pack2(0.05550713464617729f, 0.05550713464617729f));
+  q = fma2(q, f, pack2(0.24022120237350464f, 0.24022120237350464f));
+  q = fma2(q, f, pack2(0.6931469440460205f, 0.6931469440460205f));
+  q = fma2(q, f, pack2(1.0000001192092896f, 1.0000001192092896f));
+  float q0, q1, t0, t1;
+  unpack2(q, q0, q1);
+  unpack2(t, t0, t1);
+  return pack2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23)),
+               __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23)));
+}
+
+// sum += 2^(x*c - ref) over eight entries of one stream; the first POLY_N of the four pairs take the
+// FMA-pipe polynomial, the others ex2.approx
+template <int POLY_N>
 __device__ __forceinline__ void exp_sum8(f32x2& s2, const f32x2 (&x)[4], f32x2 c2, f32x2 nref2) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    float a0, a1;
-    unpack2(fma2(x[i], c2, nref2), a0, a1);
-    s2 = add2(s2, pack2(ex2(a0), ex2(a1)));
+    const f32x2 arg = fma2(x[i], c2, nref2);
+    if (i < POLY_N) {
+      s2 = add2(s2, exp2_poly2(arg));
+    } else {
+      float a0, a1;
+      unpack2(arg, a0, a1);
+      s2 = add2(s2, pack2(ex2(a0), ex2(a1)));
+    }
   }
 }
 
@@ -163,10 +199,10 @@ __device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32
     const bool upd = (bm[0] > a.thr[0]) | (bm[1] > a.thr[1]) | (bm[2] > a.thr[2]) | (bm[3] > a.thr[3]);
     if (__any_sync(kFullMask, upd)) acc_raise(a, bm, c, inv_c, lane);
   }
-  exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-  exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-  exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-  exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+  exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+  exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+  exp_sum8<0>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+  exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
 }
 
 // ---- one chunk (half a tile) from shared memory, one warp ---------------------------------------
@@ -222,6 +258,64 @@ __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, con
     if (it == 0) accum8<MASKED, true>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
     else accum8<MASKED, false>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
   }
+}
+
+// The fast variant for a full chunk.  Only the first batch computes maxima: the references are set kBias
+// binades above them, so that later entries may exceed the first batch's maximum by 2^(kBias + 120)
+// before a sum overflows, while entries down to 2^-(126 - kBias) of it still count.  Nothing is tested
+// inside the chunk; at its end a sum that is not below 2^120 (or is NaN), or a polynomial argument
+// that left the polynomial's range, makes the warp return false and the caller redoes the chunk with
+// chunk_pass, which tests every batch.
+constexpr float kBias = 60.f;
+
+template <typename T, int CHUNK, int POLY_N>
+__device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, const T* sm, int lane, float beta,
+                                           float c, float inv_c) {
+  const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
+  float run_m = kNegInf;  // running maximum of the stream that takes the polynomial
+  {
+    f32x2 l[4], p[4], m[4], r[4];
+    Batch<T>::load(sl, 0, lane, l);
+    Batch<T>::load(sp, 0, lane, p);
+    Batch<T>::load(sm, 0, lane, m);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
+    const float bm[4] = {max8(l), max8(p), max8(m), max8(r)};
+    acc_start(a, bm, c, inv_c, lane, kBias);
+    run_m = bm[Q_M];
+    exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+    exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+    exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+  }
+#pragma unroll 1
+  for (int it = 1; it < CHUNK / 256; ++it) {
+    f32x2 l[4], p[4], m[4], r[4];
+    Batch<T>::load(sl, it, lane, l);
+    Batch<T>::load(sp, it, lane, p);
+    Batch<T>::load(sm, it, lane, m);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
+    if (POLY_N > 0) run_m = fmaxf(run_m, max8(m));
+    exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+    exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+    exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+  }
+  const float kBig = 1.329227995784916e36f;  // 2^120
+  bool bad = false;
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    float s0, s1;
+    unpack2(a.s2[q], s0, s1);
+    bad |= !(s0 + s1 < kBig);
+  }
+  if (POLY_N > 0) {
+    float n0, n1;
+    unpack2(a.nref2[Q_M], n0, n1);
+    bad |= !(fmaf(run_m, c, n0) < 120.f);
+  }
+  return !__any_sync(kFullMask, bad);
 }
 
 // ---- per-request epilogue: Eq. 6/7 and the accepted length ------------------------------------------
@@ -395,6 +489,9 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
   constexpr int TILE = 2 * CHUNK;
+  // 16-bit logits carry half the bytes per power of two, so there the special-function unit binds before
+  // HBM does: the h_SLM- stream takes the FMA-pipe polynomial for POLY_N of its four pairs per batch
+  constexpr int POLY_N = sizeof(T) == 2 ? kPolyPairsBF16 : 0;
   constexpr int NPAIR = NCW / 2;
   static_assert(NCW % 2 == 0 && STAGES % NPAIR == 0, "each stage belongs to one fixed pair of consumer warps");
   static_assert(STAGES % NPW == 0, "each producer owns a fixed subset of the stages");
@@ -550,8 +647,10 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       const int nv = mt.n_valid - half * CHUNK;  // valid entries in this warp's chunk
       const T* sl = tiles + (size_t)stage * 3 * TILE + half * CHUNK;
       Acc a;
-      if (nv >= CHUNK) chunk_pass<T, CHUNK, false>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
-      else if (nv > 0) chunk_pass<T, CHUNK, true>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
+      if (nv >= CHUNK) {
+        if (!chunk_fast<T, CHUNK, POLY_N>(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.beta, mt.c, mt.inv_c))
+          chunk_pass<T, CHUNK, false>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
+      } else if (nv > 0) chunk_pass<T, CHUNK, true>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);  // the stage may be refilled while we reduce
       if (nv > 0) {
@@ -566,8 +665,19 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
         if ((lane & 7) == 0) {
           const int q = lane >> 3;
           const float rq = q == 0 ? a.ref[0] : (q == 1 ? a.ref[1] : (q == 2 ? a.ref[2] : a.ref[3]));
+          // normalise to a sum in [1, 2): readers compare the exponents of different chunks and expect
+          // the sums to be of order one (the fast path leaves them anywhere in the float32 range)
+          float m_out = rq, s_out = tot;
+          const unsigned bits = __float_as_uint(tot);
+          const int ex = (int)((bits >> 23) & 0xffu);
+          if (ex != 0 && ex != 255 && (bits >> 31) == 0) {
+            m_out = rq + (float)(ex - 127);
+            s_out = __uint_as_float((bits & 0x007fffffu) | 0x3f800000u);
+          } else if (tot == 0.f) {
+            m_out = kNegInf;
+          }
           float* rec = p.part + ((long long)mt.row * p.n_chunks + (mt.tile * 2 + half)) * 8;
-          *reinterpret_cast<float2*>(rec + 2 * q) = make_float2(rq, tot);
+          *reinterpret_cast<float2*>(rec + 2 * q) = make_float2(m_out, s_out);
         }
       }
     }
