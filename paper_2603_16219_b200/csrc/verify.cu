@@ -15,7 +15,7 @@
 namespace specsteer {
 
 #ifndef SPECSTEER_POLY_PAIRS_BF16
-#define SPECSTEER_POLY_PAIRS_BF16 4
+#define SPECSTEER_POLY_PAIRS_BF16 0
 #endif
 constexpr int kPolyPairsBF16 = SPECSTEER_POLY_PAIRS_BF16;
 constexpr float kSlack = 16.f;  // a lane's reference exponent may lag its running maximum by this much
