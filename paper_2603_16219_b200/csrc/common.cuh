@@ -97,6 +97,13 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
 }
 __device__ __forceinline__ void fence_barrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start
+// while the previous kernel of the stream is still running once every CTA of that kernel has called
+// pdl_launch_dependents() (or exited); it must call pdl_wait() before it touches anything the previous
+// kernel wrote.  Without the attribute both are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // loads that must observe other SMs' writes (workspace written earlier in the same kernel)
 __device__ __forceinline__ float4 ld_cg_f4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
 

@@ -14,7 +14,7 @@ constexpr int kRecWarps = kRecThreads / 32;
 struct PickShared {
   double warp_tot[kRecWarps];
   double base, target, W;
-  int jstar;
+  int jstar, jlast;
   int tok_min, tok_max_pos;
 };
 
@@ -58,6 +58,43 @@ __device__ __forceinline__ int pick_in_chunk(const double (&w)[PER], int v0, Pic
   return sh->tok_min != 0x7fffffff ? sh->tok_min : sh->tok_max_pos;
 }
 
+
+// Chunk search over the chunk weights cw[0..n): W = sum, target = u*W, the first chunk j whose inclusive
+// cumulative weight exceeds the target (else the last chunk with positive weight) and the cumulative
+// weight before it.  Each thread owns a contiguous run of chunks; a block-wide scan joins the runs.
+// Every thread must call it; on return sh->{jstar, base, target, W} are set and visible to all.
+__device__ __forceinline__ void find_chunk(const double* cw, int n, double u, PickShared* sh, int tid) {
+  const int per = (n + kRecThreads - 1) / kRecThreads;
+  const int j0 = min(tid * per, n), j1 = min(j0 + per, n);
+  double local = 0.0;
+  for (int j = j0; j < j1; ++j) local += cw[j];
+  if (tid == 0) { sh->jstar = 0x7fffffff; sh->jlast = -1; }
+  const double excl = block_excl_scan(local, sh->warp_tot, tid);  // two barriers inside
+  if (tid == kRecThreads - 1) { sh->W = excl + local; sh->target = u * (excl + local); }
+  __syncthreads();
+  const double target = sh->target;
+  double c = excl;
+  int mine = 0x7fffffff, lastpos = -1;
+  for (int j = j0; j < j1; ++j) {
+    if (cw[j] > 0.0) lastpos = j;
+    if (mine == 0x7fffffff && c + cw[j] > target) mine = j;
+    c += cw[j];
+  }
+  if (mine != 0x7fffffff) atomicMin(&sh->jstar, mine);
+  if (lastpos >= 0) atomicMax(&sh->jlast, lastpos);
+  __syncthreads();
+  const int jstar = sh->jstar != 0x7fffffff ? sh->jstar : max(sh->jlast, 0);
+  // the owner of jstar publishes the cumulative weight before it
+  if (jstar >= j0 && jstar < j1) {
+    double base = excl;
+    for (int j = j0; j < jstar; ++j) base += cw[j];
+    sh->base = base;
+  }
+  __syncthreads();
+  if (tid == 0) sh->jstar = jstar;
+  __syncthreads();
+}
+
 struct ReqState {
   int n, len, status;
   bool sample;  // a token is to be drawn from row n
@@ -82,6 +119,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundP
   __shared__ PickShared sh;
   const int b = blockIdx.x, tid = threadIdx.x;
   const int K = p.K, K1 = K + 1;
+  pdl_wait();  // launched behind the epilogue kernel: nothing is read before that one has finished
   const ReqState st = request_state(p, b);
 
   if (p.out_tokens)
@@ -104,21 +142,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundP
   }
   if (tid == 0) { sh.tok_min = 0x7fffffff; sh.tok_max_pos = -1; }
   __syncthreads();
-  if (tid == 0) {
-    double W = 0.0;
-    for (int j = 0; j < p.n_chunks; ++j) W += cw[j];
-    const double target = (double)p.u_recover[b] * W;
-    double c = 0.0, base = 0.0, base_last = 0.0;
-    int jstar = -1, jlast = 0;
-    for (int j = 0; j < p.n_chunks; ++j) {
-      if (cw[j] > 0.0) { jlast = j; base_last = c; }
-      if (c + cw[j] > target) { jstar = j; base = c; break; }
-      c += cw[j];
-    }
-    if (jstar < 0) { jstar = jlast; base = base_last; }
-    sh.jstar = jstar; sh.base = base; sh.target = target; sh.W = W;
-  }
-  __syncthreads();
+  find_chunk(cw, p.n_chunks, (double)p.u_recover[b], &sh, tid);
 
   const T* hl = reinterpret_cast<const T*>(p.h_llm);
   const T* hp = reinterpret_cast<const T*>(p.h_plus);
@@ -211,21 +235,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_residual_kernel(const Rou
     if (lane == 0) cw[j] = acc;
   }
   __syncthreads();
-  if (tid == 0) {
-    double W = 0.0;
-    for (int j = 0; j < p.n_chunks; ++j) W += cw[j];
-    const double target = (double)p.u_recover[b] * W;
-    double c = 0.0, base = 0.0, base_last = 0.0;
-    int jstar = -1, jlast = 0;
-    for (int j = 0; j < p.n_chunks; ++j) {
-      if (cw[j] > 0.0) { jlast = j; base_last = c; }
-      if (c + cw[j] > target) { jstar = j; base = c; break; }
-      c += cw[j];
-    }
-    if (jstar < 0) { jstar = jlast; base = base_last; }
-    sh.jstar = jstar; sh.base = base; sh.target = target; sh.W = W;
-  }
-  __syncthreads();
+  find_chunk(cw, p.n_chunks, (double)p.u_recover[b], &sh, tid);
   if (!(sh.W > 0.0)) {  // no residual mass: keep the STEER sample already written
     if (tid == 0) {
       p.status_ws[b] = st.status | SPECSTEER_REQ_RESIDUAL_EMPTY;
@@ -259,9 +269,18 @@ cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li
   (void)li;
   const size_t smem = (size_t)p.n_chunks * sizeof(double);
   *n_launches = 1;
-  if (dtype == SPECSTEER_F32) recover_steer_kernel<float, kChunkF32><<<p.B, kRecThreads, smem, s>>>(p);
-  else recover_steer_kernel<uint16_t, kChunkBF16><<<p.B, kRecThreads, smem, s>>>(p);
-  cudaError_t e = cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.B);
+  cfg.blockDim = dim3(kRecThreads);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaError_t e = dtype == SPECSTEER_F32 ? cudaLaunchKernelEx(&cfg, recover_steer_kernel<float, kChunkF32>, p)
+                                         : cudaLaunchKernelEx(&cfg, recover_steer_kernel<uint16_t, kChunkBF16>, p);
   if (e != cudaSuccess || p.recover_mode != SPECSTEER_RECOVER_RESIDUAL) return e;
   *n_launches = 2;
   if (dtype == SPECSTEER_F32) recover_residual_kernel<float, kChunkF32><<<p.B, kRecThreads, smem, s>>>(p);

@@ -333,25 +333,87 @@ struct RowResult {
   int8_t tok_ok;
 };
 
-// One warp: combine the partial records of `row` in chunk order (exact power-of-two rescale, sums in
-// double) and, for a drafted row, the log-probabilities, alpha and the accept decision.
+// log2(x) in double for x > 0 (about 1e-12 absolute): exponent plus the atanh series of the mantissa
+// folded into [sqrt(1/2), sqrt(2)).  Short on purpose: the library routine costs several times the
+// instructions and every warp of the epilogue is latency-bound.  x = 0 gives -inf, x = +inf gives +inf,
+// negative or NaN gives NaN; subnormal inputs do not occur here (sums of float32 values >= 1, or 0).
+__device__ __forceinline__ double log2_pos(double x) {
+  if (!(x > 0.0)) return (x == 0.0) ? -__longlong_as_double(0x7ff0000000000000ll) : __longlong_as_double(0x7ff8000000000000ll);
+  const int hi = __double2hiint(x), lo = __double2loint(x);
+  if (hi >= 0x7ff00000) return x;  // +inf
+  int e = (hi >> 20) - 1023;
+  double m = __hiloint2double((hi & 0x000fffff) | 0x3ff00000, lo);  // [1, 2)
+  if (m > 1.4142135623730951) { m *= 0.5; e += 1; }
+  const double z = (m - 1.0) / (m + 1.0), w = z * z;
+  double q = 1.0 / 13.0;
+  q = fma(q, w, 1.0 / 11.0);
+  q = fma(q, w, 1.0 / 9.0);
+  q = fma(q, w, 1.0 / 7.0);
+  q = fma(q, w, 1.0 / 5.0);
+  q = fma(q, w, 1.0 / 3.0);
+  q = fma(q, w, 1.0);
+  return fma(z * q, 2.8853900817779268 /* 2/ln 2 */, (double)e);
+}
+
+// exp(x) in double for x <= 0 (about 1e-14 relative); 0 below the normal range.
+__device__ __forceinline__ double exp_nonpos(double x) {
+  const double y = x * 1.4426950408889634;
+  if (!(y > -1000.0)) return (y != y) ? y : 0.0;
+  const double k = rint(y), f = (y - k) * 0.6931471805599453;  // |f| <= 0.347
+  double q = 1.0 / 39916800.0;
+  q = fma(q, f, 1.0 / 3628800.0);
+  q = fma(q, f, 1.0 / 362880.0);
+  q = fma(q, f, 1.0 / 40320.0);
+  q = fma(q, f, 1.0 / 5040.0);
+  q = fma(q, f, 1.0 / 720.0);
+  q = fma(q, f, 1.0 / 120.0);
+  q = fma(q, f, 1.0 / 24.0);
+  q = fma(q, f, 1.0 / 6.0);
+  q = fma(q, f, 0.5);
+  q = fma(q, f, 1.0);
+  q = fma(q, f, 1.0);
+  return __hiloint2double(__double2hiint(q) + ((int)k << 20), __double2loint(q));
+}
+
+// One warp: combine the partial records of `row` (exact power-of-two rescale, sums in double) and, for a
+// drafted row, the log-probabilities, alpha and the accept decision.
 template <typename T>
 __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float beta, float lam, float c, int lane,
                              RowResult* out) {
   const int K = p.K, K1 = K + 1;
   const long long row = (long long)b * K1 + t;
   const float* rec = p.part + row * p.n_chunks * 8;
-  float M[4] = {kNegInf, kNegInf, kNegInf, kNegInf};
-  for (int ch = lane; ch < p.n_chunks; ch += 32) {
-    float4 x = ld_cg_f4(rec + ch * 8), y = ld_cg_f4(rec + ch * 8 + 4);
-    M[0] = fmaxf(M[0], x.x); M[1] = fmaxf(M[1], x.z); M[2] = fmaxf(M[2], y.x); M[3] = fmaxf(M[3], y.z);
+  // the drafted token's three logits: issued first so that their latency overlaps the record passes
+  int y = -1;
+  float gl = 0.f, gp = 0.f, gm = 0.f;
+  if (t < len) {
+    y = p.draft_tokens[(long long)b * K + t];
+    if (y >= 0 && y < p.V) {
+      const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
+      gl = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
+      gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
+      gm = load_logit<T>(reinterpret_cast<const T*>(p.h_minus), off);
+    }
   }
-#pragma unroll
-  for (int q = 0; q < 4; ++q) M[q] = warp_max(M[q]);
-  double S[4] = {0.0, 0.0, 0.0, 0.0};
+  pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
+  // pass 1: the largest exponent per normaliser; pass 2 (the same lines, now in L1): sums relative to it
+  float Ml[4] = {kNegInf, kNegInf, kNegInf, kNegInf};
+#pragma unroll 4
   for (int ch = lane; ch < p.n_chunks; ch += 32) {
-    float4 x = ld_cg_f4(rec + ch * 8), y = ld_cg_f4(rec + ch * 8 + 4);
-    const float mm[4] = {x.x, x.z, y.x, y.z}, ss[4] = {x.y, x.w, y.y, y.w};
+    const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
+    const float4 z = __ldg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
+    Ml[0] = fmaxf(Ml[0], x.x); Ml[1] = fmaxf(Ml[1], x.z); Ml[2] = fmaxf(Ml[2], z.x); Ml[3] = fmaxf(Ml[3], z.z);
+  }
+  const float mine = warp_reduce4<true>(Ml, lane);
+  float M[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) M[q] = __shfl_sync(kFullMask, mine, 8 * q);
+  double S[4] = {0.0, 0.0, 0.0, 0.0};
+#pragma unroll 4
+  for (int ch = lane; ch < p.n_chunks; ch += 32) {
+    const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
+    const float4 z = __ldg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
+    const float mm[4] = {x.x, x.z, z.x, z.z}, ss[4] = {x.y, x.w, z.y, z.w};
 #pragma unroll
     for (int q = 0; q < 4; ++q) {
       float w = ss[q];
@@ -359,17 +421,23 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
       S[q] += (double)w;
     }
   }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) S[q] += __shfl_xor_sync(kFullMask, S[q], o);
+  }
+  // lanes 0..3 take the logarithm of one sum each, lane 4 that of lambda
+  const double arg = lane == 0 ? S[0] : (lane == 1 ? S[1] : (lane == 2 ? S[2] : (lane == 3 ? S[3] : (double)lam)));
+  const double lg = log2_pos(arg);
   RowResult r;
   bool fin = true;
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    double s = S[q];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(kFullMask, s, o);
-    r.lse[q] = (double)M[q] + log2(s);
+    r.lse[q] = (double)M[q] + __shfl_sync(kFullMask, lg, q);
     fin = fin && isfinite(r.lse[q]);
   }
   const double ln2 = 0.6931471805599453;
+  const double log_lam = __shfl_sync(kFullMask, lg, 4) * ln2;
   r.logz = (r.lse[Q_R] - r.lse[Q_L] - (double)beta * (r.lse[Q_P] - r.lse[Q_M])) * ln2;
   r.fin = fin; r.testable = 0; r.accept = 0; r.tok_ok = 0; r.alpha = 0.f;
   r.lp[0] = r.lp[1] = r.lp[2] = r.lp[3] = __int_as_float(0x7fc00000);
@@ -378,24 +446,18 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
         make_float4((float)r.lse[0], (float)r.lse[1], (float)r.lse[2], (float)r.lse[3]);
   if (fin && t < len) {
     const long long i = (long long)b * K + t;
-    const int y = p.draft_tokens[i];
     if (y >= 0 && y < p.V) {
-      const T* hl = reinterpret_cast<const T*>(p.h_llm);
-      const T* hp = reinterpret_cast<const T*>(p.h_plus);
-      const T* hm = reinterpret_cast<const T*>(p.h_minus);
-      const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
       const double cd = (double)c;
-      const double l = (double)load_logit<T>(hl, off), pp = (double)load_logit<T>(hp, off),
-                   m = (double)load_logit<T>(hm, off);
+      const double l = (double)gl, pp = (double)gp, m = (double)gm;
       const double rr = l + (double)beta * (pp - m);  // Eq. 8
       const double lpL = (l * cd - r.lse[Q_L]) * ln2, lpP = (pp * cd - r.lse[Q_P]) * ln2,
                    lpM = (m * cd - r.lse[Q_M]) * ln2, lpS = (rr * cd - r.lse[Q_R]) * ln2;
       r.lp[Q_L] = (float)lpL; r.lp[Q_P] = (float)lpP; r.lp[Q_M] = (float)lpM; r.lp[Q_R] = (float)lpS;
       r.tok_ok = 1;
-      const double logrho = (p.accept_mode == SPECSTEER_ACCEPT_RATIO) ? (lpL - lpM - log((double)lam))  // Eq. 7
+      const double logrho = (p.accept_mode == SPECSTEER_ACCEPT_RATIO) ? (lpL - lpM - log_lam)  // Eq. 7
                                                                       : (lpS - lpP);                    // Eq. 6
       if (!isnan(logrho)) {
-        const double ald = exp(fmin(0.0, logrho));
+        const double ald = exp_nonpos(fmin(0.0, logrho));
         r.alpha = (float)ald;
         r.testable = 1;
         r.accept = ((double)p.u_accept[i] <= ald) ? 1 : 0;  // "Uniform(0,1) <= alpha_t", decided in double
@@ -408,6 +470,7 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
 template <typename T>
 __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundParams p) {
   __shared__ RowResult res[kEpiMaxRows];
+  pdl_launch_dependents();  // the recovery kernel may be set up behind this one
   const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int K = p.K, K1 = K + 1;
   int status = 0;
@@ -507,6 +570,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   float* c_s = beta_s + p.B;                                      // [B]  log2(e) / T_b
   float* ic_s = c_s + p.B;                                        // [B]  T_b / log2(e)
 
+  pdl_launch_dependents();  // the epilogue's CTAs may take over SMs as this grid's CTAs retire
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   constexpr int nthreads = (NCW + NPW) * 32;
   const bool bonus = (p.flags & SPECSTEER_FLAG_BONUS) != 0;
@@ -717,9 +781,19 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
   }
   if (e != cudaSuccess) return e;
   if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;
-  if (dtype == SPECSTEER_F32) epilogue_kernel<float><<<p.B, kEpiWarps * 32, 0, s>>>(p);
-  else epilogue_kernel<uint16_t><<<p.B, kEpiWarps * 32, 0, s>>>(p);
-  return cudaGetLastError();
+  // programmatic dependent launch: the epilogue reads its inputs while the streaming kernel drains
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.B);
+  cfg.blockDim = dim3(kEpiWarps * 32);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  if (dtype == SPECSTEER_F32) return cudaLaunchKernelEx(&cfg, epilogue_kernel<float>, p);
+  return cudaLaunchKernelEx(&cfg, epilogue_kernel<uint16_t>, p);
 }
 
 }  // namespace specsteer
