@@ -29,7 +29,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per used row of the streaming kernel, from the ncu captures summarised under
 # profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows), keyed by
 # configuration.  Absent = not captured for the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_ROW = {3: 1852523, 4: 1559272}
+NCU_TRAFFIC_BYTES_PER_ROW = {3: 1856749, 4: 1559000}
 
 
 def _peaks():
@@ -186,6 +186,9 @@ def run_cuda(args, rank, world, local_rank):
     logit_bytes = spec.logit_bytes(rows)
     ctx = binding.Context(spec.B, spec.K, spec.V, device=local_rank)
     outs = binding.alloc_outputs(spec.B, spec.K, dev)
+    if args.lean:   # only what Algorithm 1 needs: without these two the normaliser of h_SLM+ is not formed
+        outs.pop("logp_plus")
+        outs.pop("log_z")
     desc = binding.make_desc(inputs, outs, flags=flags)
     stream = torch.cuda.current_stream(dev)
 
@@ -257,7 +260,7 @@ def run_cuda(args, rank, world, local_rank):
     if args.kernels_only:
         sampler.stop()
         if rank == 0:
-            print(json.dumps({"workload": spec.name, "ms_per_step": ms_per_step, "verify_kernel_ms": kernel_ms,
+            print(json.dumps({"workload": spec.name, "outputs": "lean" if args.lean else "all", "ms_per_step": ms_per_step, "verify_kernel_ms": kernel_ms,
                               "verify_gbs": logit_bytes / (kernel_ms * 1e-3) / 1e9, "positions_per_s": value,
                               "clocks": sampler.summary()}), flush=True)
         if dist is not None:
@@ -267,6 +270,9 @@ def run_cuda(args, rank, world, local_rank):
     # ---- end to end: pinned host buffers in, pinned host results out, copies inside the timed region
     host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
     host_out = binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True)
+    if args.lean:
+        host_out.pop("logp_plus")
+        host_out.pop("log_z")
     hdesc = binding.make_desc(host_in, host_out, flags=flags)
     h2d = sum(v.numel() * v.element_size() for v in host_in.values())
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
@@ -327,6 +333,7 @@ def run_cuda(args, rank, world, local_rank):
         "config": {"workload": spec.name, "B": spec.B, "K": spec.K, "V": spec.V, "logit_dtype": spec.dtype,
                    "requests_per_gpu": spec.B, "rows_read_per_gpu": rows, "positions_per_step_per_gpu": positions,
                    "accept_mode": "ratio", "recover_mode": "steer", "bonus_row": True, "lambda": spec.lam,
+                   "outputs": "Algorithm 1 only (no logp_plus, log_z)" if args.lean else "all",
                    "acceptance_rate": float(outs["accept_len"].sum().item()) / max(1, positions),
                    "l2": ("inputs %.2f GB per step exceed L2" % (logit_bytes / 1e9)) if n_sets == 1 else
                          ("rotating %d input sets (%.2f GB) to exceed L2" % (n_sets, n_sets * logit_bytes / 1e9)),
@@ -352,6 +359,8 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="index into the five benchmark configurations")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--requests", type=int, default=0, help="override B (reduced batch for profiler captures)")
+    ap.add_argument("--lean", action="store_true",
+                    help="request only the outputs Algorithm 1 needs (no logp_plus, log_z): three normalisers per row")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the device-resident steps and print a short line (profiling aid)")
     args = ap.parse_args()

@@ -91,7 +91,11 @@ typedef struct {
   const float *u_accept;                        /* [B][K]   uniforms in [0,1) for "Uniform(0,1) <= alpha_t" */
   const float *u_recover;                       /* [B]      uniform in [0,1) for the recovery sample */
 
-  /* ---- outputs (caller-allocated; any may be NULL except accept_len) ---- */
+  /* ---- outputs (caller-allocated; any may be NULL except accept_len) ----
+   * Algorithm 1 itself needs three normalisers per row (h_LLM and h_SLM- for Eq. 7, h_rec for Eq. 8).  The
+   * fourth, of h_SLM+, is formed only when something asks for it: a non-NULL logp_plus or log_z, EXACT_Z
+   * acceptance or RESIDUAL recovery.  Leaving logp_plus and log_z NULL in RATIO + STEER mode therefore saves a
+   * quarter of the exponentials (it matters for 16-bit logits, where they bind before the memory does). */
   int32_t *accept_len;   /* [B]      drafts accepted before the first rejection */
   uint8_t *accept_flags; /* [B][K]   1 where u <= alpha (every drafted position, also after the first rejection) */
   float *alpha;          /* [B][K]   acceptance probability; 0 beyond draft_len */

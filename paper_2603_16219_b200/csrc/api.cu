@@ -91,6 +91,8 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
   p.B = nb; p.K = K; p.V = d->V;
   p.ld_row = d->ld_row; p.ld_req = d->ld_req;
   p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
+  p.need_p = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
+              d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? 1 : 0;
   p.tile = tile_of(d->dtype);
   p.n_chunks = n_chunks_of(d->V, p.tile);
   auto lg = [&](const void* base) { return (const void*)((const char*)base + (size_t)b0 * d->ld_req * es); };

@@ -17,6 +17,7 @@ struct RoundParams {
   long long ld_row, ld_req;  // elements
   int accept_mode, recover_mode;
   unsigned flags;
+  int need_p;    // the normaliser of h_SLM+ is wanted (logp_plus, log_z, EXACT_Z or RESIDUAL); Algorithm 1 itself is not
   int tile;      // vocabulary entries per chunk (kChunkF32 or kChunkBF16)
   int n_chunks;  // ceil(V / tile)
   const void *h_llm, *h_plus, *h_minus;

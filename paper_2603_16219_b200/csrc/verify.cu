@@ -18,6 +18,10 @@ namespace specsteer {
 #define SPECSTEER_POLY_PAIRS_BF16 0
 #endif
 constexpr int kPolyPairsBF16 = SPECSTEER_POLY_PAIRS_BF16;
+#ifndef SPECSTEER_POLY_PAIRS_BF16_LEAN
+#define SPECSTEER_POLY_PAIRS_BF16_LEAN 0
+#endif
+constexpr int kPolyPairsBF16Lean = SPECSTEER_POLY_PAIRS_BF16_LEAN;
 constexpr float kSlack = 16.f;  // a lane's reference exponent may lag its running maximum by this much
 
 struct TileMeta {
@@ -268,7 +272,7 @@ __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, con
 // chunk_pass, which tests every batch.
 constexpr float kBias = 60.f;
 
-template <typename T, int CHUNK, int POLY_N>
+template <typename T, int CHUNK, int POLY_N, bool NEED_P>
 __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, const T* sm, int lane, float beta,
                                            float c, float inv_c) {
   const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
@@ -280,11 +284,11 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     Batch<T>::load(sm, 0, lane, m);
 #pragma unroll
     for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
-    const float bm[4] = {max8(l), max8(p), max8(m), max8(r)};
+    const float bm[4] = {max8(l), NEED_P ? max8(p) : kNegInf, max8(m), max8(r)};
     acc_start(a, bm, c, inv_c, lane, kBias);
     run_m = bm[Q_M];
     exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (NEED_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
     exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
     exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
@@ -298,7 +302,7 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
     if (POLY_N > 0) run_m = fmaxf(run_m, max8(m));
     exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (NEED_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
     exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
     exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
@@ -434,7 +438,7 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     r.lse[q] = (double)M[q] + __shfl_sync(kFullMask, lg, q);
-    fin = fin && isfinite(r.lse[q]);
+    if (q != Q_P || p.need_p) fin = fin && isfinite(r.lse[q]);
   }
   const double ln2 = 0.6931471805599453;
   const double log_lam = __shfl_sync(kFullMask, lg, 4) * ln2;
@@ -549,12 +553,12 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 // producer thread that owns the stages congruent to its index modulo NPW (one thread cannot issue tiles
 // fast enough for a whole SM).  Every stage is always consumed by the same pair of warps, so a waiting
 // warp is never a whole barrier phase ahead of the data.
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, bool NEED_P>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
   constexpr int TILE = 2 * CHUNK;
   // 16-bit logits carry half the bytes per power of two, so there the special-function unit binds before
   // HBM does: the h_SLM- stream takes the FMA-pipe polynomial for POLY_N of its four pairs per batch
-  constexpr int POLY_N = sizeof(T) == 2 ? kPolyPairsBF16 : 0;
+  constexpr int POLY_N = sizeof(T) == 2 ? (NEED_P ? kPolyPairsBF16 : kPolyPairsBF16Lean) : 0;
   constexpr int NPAIR = NCW / 2;
   static_assert(NCW % 2 == 0 && STAGES % NPAIR == 0, "each stage belongs to one fixed pair of consumer warps");
   static_assert(STAGES % NPW == 0, "each producer owns a fixed subset of the stages");
@@ -712,7 +716,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       const T* sl = tiles + (size_t)stage * 3 * TILE + half * CHUNK;
       Acc a;
       if (nv >= CHUNK) {
-        if (!chunk_fast<T, CHUNK, POLY_N>(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.beta, mt.c, mt.inv_c))
+        if (!chunk_fast<T, CHUNK, POLY_N, NEED_P>(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.beta, mt.c, mt.inv_c))
           chunk_pass<T, CHUNK, false>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
       } else if (nv > 0) chunk_pass<T, CHUNK, true>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
@@ -749,12 +753,12 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
 }
 
 // ---- launch -------------------------------------------------------------------------------------------
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, bool NEED_P>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
   const size_t fixed = (size_t)STAGES * 3 * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
                        STAGES * sizeof(TileMeta) + 16;
   const size_t smem = fixed + (size_t)(4 * p.B + 1) * sizeof(int);
-  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK>;
+  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, NEED_P>;
   static bool attr_set_dev[64] = {};  // per instantiation and device; sized for the largest slab
   bool& attr_set = attr_set_dev[li.device & 63];
   if (!attr_set) {
@@ -772,12 +776,15 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
   *n_launches = 2;
   cudaError_t e;
   if (ev_begin && (e = cudaEventRecord(ev_begin, s)) != cudaSuccess) return e;
+  const bool np = p.need_p != 0;
   if (dtype == SPECSTEER_F32) {
-    e = aligned ? launch_stream<float, kChunkF32, 16, 16, 4, true>(p, li, s)
-                : launch_stream<float, kChunkF32, 16, 16, 4, false>(p, li, s);
+    e = aligned ? (np ? launch_stream<float, kChunkF32, 16, 16, 4, true, true>(p, li, s)
+                      : launch_stream<float, kChunkF32, 16, 16, 4, true, false>(p, li, s))
+                : launch_stream<float, kChunkF32, 16, 16, 4, false, true>(p, li, s);
   } else {
-    e = aligned ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true>(p, li, s)
-                : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false>(p, li, s);
+    e = aligned ? (np ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, true>(p, li, s)
+                      : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, false>(p, li, s))
+                : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, true>(p, li, s);
   }
   if (e != cudaSuccess) return e;
   if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;

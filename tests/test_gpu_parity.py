@@ -102,6 +102,26 @@ def test_row_strides_and_unaligned_rows(env, V, ld, dtype):
         np.testing.assert_allclose(gpu["logp_star"], gpu2["logp_star"], atol=1e-5, equal_nan=True)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_outputs_not_requested_skip_the_plus_normaliser(env, dtype):
+    """Algorithm 1 needs the normalisers of h_LLM, h_SLM- (Eq. 7) and h_rec (Eq. 8) only.  Without logp_plus and
+    log_z the library does not form the one of h_SLM+; every other output must be unchanged, bit for bit."""
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 7, 4, 9001, dtype, seed=21, ragged=True, beta_choices=(0.5, 1.0, 2.0))
+    full = b.alloc_outputs(spec.B, spec.K, "cuda")
+    lean = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in ("logp_plus", "log_z")}
+    for outs in (full, lean):
+        d = b.make_desc(inputs, outs, flags=b.FLAG_BONUS)
+        env["ctx"].verify_round(d)
+        env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0
+    for k, v in lean.items():
+        assert np.array_equal(v.cpu().numpy(), full[k].cpu().numpy(), equal_nan=True), k
+    gpu = {k: v.cpu().numpy() for k, v in full.items()}
+    P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), 0, 0, 1, P.TOL[inputs["h_llm"].dtype])
+
+
 def test_draft_length_extremes_and_no_bonus(env):
     """len 0 (with and without the bonus row: a request that reads nothing), len K, ragged in between."""
     spec, inputs = _small(env["synth"], 9, 4, 3000, "f32", seed=3)
