@@ -170,6 +170,26 @@ def test_degenerate_logits_and_status_words(env):
         assert gpu["req_status"][2] & b.REQ_NONFINITE or gpu["accept_len"][2] == 0
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_outliers_after_the_first_batch_of_a_chunk(env, dtype):
+    """Full chunks are reduced relative to the maxima of their first 256 entries; an entry hundreds of binades
+    above those must overflow that attempt and send the chunk through the variant that tests every batch.
+    Spikes sit past the first batch of a chunk, in each stream, at low temperature too.  Their size keeps the
+    spread of a row below ~1000 binades: log2(e)/T is a float32 in the kernels, so a log-probability carries an
+    error of about 2^-25 times the distance (in binades) of the token from the row maximum."""
+    spec, inputs = _small(env["synth"], 6, 3, 5000, dtype, seed=17, temp_choices=(0.25, 1.0), beta_choices=(1.0, 2.5))
+    L, Pp, M = inputs["h_llm"], inputs["h_slm_plus"], inputs["h_slm_minus"]
+    L[0, 0, 300] = 160.0                    # one stream only
+    Pp[1, 1, 1900] = 150.0
+    M[2, 0, 2900] = 170.0
+    L[3, :, 777] += 140.0; Pp[3, :, 777] += 140.0; M[3, :, 777] += 140.0   # a shared spike: r stays moderate
+    L[4, 2, 4999] = 165.0                   # in the ragged last chunk
+    Pp[5, 0, 600] = 150.0; M[5, 0, 601] = 155.0; L[5, 0, 1100] = 145.0
+    for am, rm in ((0, 0), (1, 1)):
+        gpu = P.run_gpu(env["ctx"], inputs, am, rm, 1)
+        P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, 1, P.TOL[L.dtype])
+
+
 def test_many_requests_cross_the_slab_limit(env):
     spec, inputs = _small(env["synth"], 5000, 2, 64, "bf16", seed=6, ragged=True)
     gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
