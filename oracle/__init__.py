@@ -19,6 +19,7 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "specsteer_oracle.c")
+_SRC_TOPK = os.path.join(_HERE, "specsteer_oracle_topk.c")
 _HDR = os.path.join(_HERE, "specsteer_oracle.h")
 _LIB = os.path.join(_HERE, "libspecsteer_oracle.so")
 
@@ -32,11 +33,11 @@ REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1
 def build(force: bool = False) -> str:
     """Compile the oracle into a shared object next to its source (gcc -O2 -fopenmp)."""
     stale = (not os.path.exists(_LIB)) or any(
-        os.path.getmtime(p) > os.path.getmtime(_LIB) for p in (_SRC, _HDR))
+        os.path.getmtime(p) > os.path.getmtime(_LIB) for p in (_SRC, _SRC_TOPK, _HDR))
     if force or stale:
         tmp = _LIB + ".tmp%d" % os.getpid()
         subprocess.check_call(["gcc", "-O2", "-fopenmp", "-std=c99", "-Wall", "-shared", "-fPIC",
-                               "-o", tmp, _SRC, "-lm"])
+                               "-o", tmp, _SRC, _SRC_TOPK, "-lm"])
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -77,6 +78,13 @@ def lib():
                                               C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         _lib.specsteer_oracle_row.restype = C.c_int
         _lib.specsteer_oracle_max_threads.restype = C.c_int
+        _lib.specsteer_oracle_cloud_topk_row.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_void_p, C.c_float, C.c_int,
+                                                         C.c_void_p, C.c_void_p]
+        _lib.specsteer_oracle_cloud_topk_row.restype = C.c_int
+        _lib.specsteer_oracle_edge_resample_row.argtypes = [C.c_int, C.c_int, C.c_void_p, C.c_float, C.c_float, C.c_int,
+                                                            C.c_void_p, C.c_void_p, C.c_double,
+                                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib.specsteer_oracle_edge_resample_row.restype = C.c_int
     return _lib
 
 
@@ -154,4 +162,55 @@ def verify_recover_round(h_llm, h_slm_plus, h_slm_minus, draft_tokens, draft_len
     rc = lib().specsteer_oracle_round(C.byref(a))
     if rc != 0:
         raise RuntimeError("oracle round failed: %d" % rc)
+    return out
+
+
+def cloud_topk_row(h_llm, h_minus, beta, k):
+    """Cloud half of the top-k split recovery on one row: (ids[k] int32, values[k] float32)."""
+    hl, dt = _logits(h_llm)
+    hm, dt2 = _logits(h_minus)
+    assert dt == dt2 and hl.ndim == 1 and hl.shape == hm.shape
+    idx = np.empty(k, np.int32)
+    val = np.empty(k, np.float32)
+    rc = lib().specsteer_oracle_cloud_topk_row(hl.shape[0], dt, _p(hl), _p(hm), float(beta), int(k), _p(idx), _p(val))
+    if rc != 0:
+        raise RuntimeError("oracle cloud_topk_row failed: %d" % rc)
+    return idx, val
+
+
+def edge_resample_row(h_plus, beta, temperature, idx, val, u):
+    """Edge half on one row: dict(token, logprob, probs[k], cdf_margin)."""
+    hp, dt = _logits(h_plus)
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    val = np.ascontiguousarray(val, dtype=np.float32)
+    k = idx.shape[0]
+    tok = np.empty(1, np.int32); lp = np.empty(1); probs = np.empty(k); mg = np.empty(1)
+    rc = lib().specsteer_oracle_edge_resample_row(hp.shape[0], dt, _p(hp), float(beta), float(temperature), k,
+                                                  _p(idx), _p(val), float(u), _p(tok), _p(lp), _p(probs), _p(mg))
+    if rc != 0:
+        raise RuntimeError("oracle edge_resample_row failed: %d" % rc)
+    return {"token": int(tok[0]), "logprob": float(lp[0]), "probs": probs, "cdf_margin": float(mg[0])}
+
+
+def topk_recover_round(h_llm, h_slm_plus, h_slm_minus, draft_len, beta, temperature, u_recover, accept_len, req_status,
+                       k, flags=0):
+    """Top-k split recovery for a verified batch: for every request that samples (accept_len < draft_len, or
+    always with FLAG_BONUS; never after a BAD_PARAM / NONFINITE status) the cloud's list of row accept_len and the
+    edge's token.  Returns dict(topk_idx[B,k], topk_val[B,k], rec_token[B], rec_logprob[B], cdf_margin[B])."""
+    B = h_llm.shape[0]
+    K = h_llm.shape[1] - 1
+    out = {"topk_idx": np.full((B, k), -1, np.int32), "topk_val": np.full((B, k), -np.inf, np.float32),
+           "rec_token": np.full(B, -1, np.int32), "rec_logprob": np.full(B, np.nan), "cdf_margin": np.full(B, np.inf)}
+    for b in range(B):
+        ln = int(draft_len[b])
+        if ln < 0 or ln > K:
+            ln = 0
+        n = int(accept_len[b])
+        bad = int(req_status[b]) & (REQ_BAD_PARAM | REQ_NONFINITE)
+        if bad or not (n < ln or (flags & FLAG_BONUS)):
+            continue
+        idx, val = cloud_topk_row(h_llm[b, n], h_slm_minus[b, n], beta[b], k)
+        r = edge_resample_row(h_slm_plus[b, n], beta[b], temperature[b], idx, val, float(u_recover[b]))
+        out["topk_idx"][b], out["topk_val"][b] = idx, val
+        out["rec_token"][b], out["rec_logprob"][b], out["cdf_margin"][b] = r["token"], r["logprob"], r["cdf_margin"]
     return out

@@ -61,6 +61,17 @@ int specsteer_oracle_row(int V, int dtype, const void *h_llm, const void *h_plus
 
 int specsteer_oracle_max_threads(void);
 
+/* ---- top-k split recovery (deployment appendix; specsteer_oracle_topk.c) ---- */
+/* Cloud half, one row: the k largest entries of h_LLM - beta*h_SLM- (float32, one fused multiply-add), value
+ * descending then token id ascending; slots beyond the number of non-NaN entries get id -1, value -inf. */
+int specsteer_oracle_cloud_topk_row(int V, int dtype, const void *h_llm, const void *h_minus, float beta, int k,
+                                    int32_t *idx_out, float *val_out);
+/* Edge half, one row: adds beta*h_SLM+ on the kept entries, softmax at temperature T in float64, inverse CDF in
+ * list order with uniform u.  token -1 when nothing can be sampled.  probs[k] and cdf_margin are optional. */
+int specsteer_oracle_edge_resample_row(int V, int dtype, const void *h_plus, float beta, float T, int k,
+                                       const int32_t *idx, const float *val, double u,
+                                       int32_t *token, double *logprob, double *probs, double *cdf_margin);
+
 #ifdef __cplusplus
 }
 #endif
