@@ -134,6 +134,29 @@ specsteer_status specsteer_verify_round(specsteer_ctx *ctx, const specsteer_roun
  * out_tokens, n_out.  Errors: INVALID_ARG, ORDER, CUDA. */
 specsteer_status specsteer_recover_sample(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
 
+/* Top-k split recovery (the paper's deployment appendix, "Minimal Downlink (Steering Recovery)", case "If
+ * rejected"), an alternative to specsteer_recover_sample for a deployment where h_SLM+ lives on another machine.
+ * Both calls must follow specsteer_verify_round with the same descriptor on the same stream (ERR_ORDER otherwise)
+ * and act on row accept_len of every request that samples (accept_len < draft_len, or always with FLAG_BONUS).
+ *
+ * Cloud half: h_cloud(v) = h_LLM(v) - beta*h_SLM-(v), formed in float32 by one fused multiply-add, truncated to the
+ * k entries with the highest values.  topk_idx[B][k] / topk_val[B][k] (device) receive them ordered by value,
+ * highest first, equal values by lower token id; NaN entries are never kept; unused slots and requests that do
+ * not sample get id -1 and value -inf.  Reads h_llm, h_slm_minus, beta, draft_len, accept_len; h_slm_plus is not
+ * touched.  1 <= k <= SPECSTEER_TOPK_MAX.  Errors: INVALID_ARG, UNSUPPORTED, ORDER, CUDA. */
+#define SPECSTEER_TOPK_MAX 32
+specsteer_status specsteer_cloud_topk(specsteer_ctx *ctx, const specsteer_round_desc *desc, int32_t k,
+                                      int32_t *topk_idx, float *topk_val, void *cuda_stream);
+
+/* Edge half: on the kept entries h_rec = topk_val + beta*h_SLM+[topk_idx] (Eq. 8), divided by the temperature;
+ * their softmax is taken in float64 and one token is drawn by inverse CDF in list order with u_recover (the
+ * smallest j whose cumulative weight exceeds u * total, else the last j with positive weight).  Writes rec_token,
+ * rec_logprob (log of its probability among the k), out_tokens and n_out exactly like specsteer_recover_sample.
+ * Reads h_slm_plus, beta, temperature, u_recover, draft_tokens, draft_len, accept_len and the two lists; h_llm and
+ * h_slm_minus are not touched.  Errors: as above. */
+specsteer_status specsteer_edge_resample(specsteer_ctx *ctx, const specsteer_round_desc *desc, int32_t k,
+                                         const int32_t *topk_idx, const float *topk_val, void *cuda_stream);
+
 /* Whole round from HOST memory: every pointer in `desc` is a HOST pointer (pinned memory makes the copies
  * asynchronous).  Copies inputs to device staging buffers owned by the context (allocated on the first
  * call, sized for the context's maxima: 3*max_B*(max_K+1)*max_V elements of 4 bytes), runs verification and

@@ -27,7 +27,9 @@ EXPORTS = (
     "specsteer_round_host", "specsteer_ctx_device_error", "specsteer_ctx_workspace_bytes",
     "specsteer_ctx_launch_count", "specsteer_status_string", "specsteer_version",
     "specsteer_verify_round_static", "specsteer_ctx_time_streaming",
+    "specsteer_cloud_topk", "specsteer_edge_resample",
 )
+TOPK_MAX = 32
 
 
 class RoundDesc(C.Structure):
@@ -76,6 +78,10 @@ def load_library(path: Optional[str] = None):
     lib.specsteer_ctx_device_error.restype = C.c_int
     lib.specsteer_ctx_workspace_bytes.argtypes = [C.c_void_p]
     lib.specsteer_ctx_workspace_bytes.restype = C.c_size_t
+    lib.specsteer_cloud_topk.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.specsteer_cloud_topk.restype = C.c_int
+    lib.specsteer_edge_resample.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
+    lib.specsteer_edge_resample.restype = C.c_int
     lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.specsteer_ctx_time_streaming.restype = C.c_int
     lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
@@ -162,6 +168,14 @@ def make_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor],
     return d
 
 
+def _check_topk(desc, topk_idx, topk_val) -> int:
+    if topk_idx.dtype != torch.int32 or topk_val.dtype != torch.float32 or topk_idx.shape != topk_val.shape or \
+            topk_idx.dim() != 2 or topk_idx.shape[0] != desc.B or not topk_idx.is_contiguous() or \
+            not topk_val.is_contiguous():
+        raise ValueError("top-k lists must be contiguous [B, k] int32 ids and float32 values")
+    return int(topk_idx.shape[1])
+
+
 class Context:
     """Owns one ``specsteer_ctx`` (device workspace sized for the given maxima)."""
 
@@ -192,6 +206,20 @@ class Context:
     def recover_sample(self, desc: RoundDesc, stream=None):
         _check(self._lib.specsteer_recover_sample(self._h, C.byref(desc), self._stream(stream)),
                "specsteer_recover_sample")
+
+    def cloud_topk(self, desc: RoundDesc, topk_idx: torch.Tensor, topk_val: torch.Tensor, stream=None):
+        """Cloud half of the top-k split recovery: fills topk_idx [B, k] int32 and topk_val [B, k] float32."""
+        k = _check_topk(desc, topk_idx, topk_val)
+        _check(self._lib.specsteer_cloud_topk(self._h, C.byref(desc), k, C.c_void_p(topk_idx.data_ptr()),
+                                              C.c_void_p(topk_val.data_ptr()), self._stream(stream)),
+               "specsteer_cloud_topk")
+
+    def edge_resample(self, desc: RoundDesc, topk_idx: torch.Tensor, topk_val: torch.Tensor, stream=None):
+        """Edge half: samples one token per request among the k kept entries."""
+        k = _check_topk(desc, topk_idx, topk_val)
+        _check(self._lib.specsteer_edge_resample(self._h, C.byref(desc), k, C.c_void_p(topk_idx.data_ptr()),
+                                                 C.c_void_p(topk_val.data_ptr()), self._stream(stream)),
+               "specsteer_edge_resample")
 
     def round_host(self, desc: RoundDesc, stream=None):
         _check(self._lib.specsteer_round_host(self._h, C.byref(desc), self._stream(stream)), "specsteer_round_host")

@@ -236,6 +236,44 @@ specsteer_status specsteer_recover_sample(specsteer_ctx* ctx, const specsteer_ro
   return do_recover(ctx, d, (cudaStream_t)cuda_stream);
 }
 
+specsteer_status specsteer_cloud_topk(specsteer_ctx* ctx, const specsteer_round_desc* d, int32_t k, int32_t* topk_idx,
+                                      float* topk_val, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if (k < 1 || k > SPECSTEER_TOPK_MAX || !topk_idx || !topk_val) return SPECSTEER_ERR_INVALID_ARG;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (!ctx->verified || ctx->v_B != d->B || ctx->v_K != d->K || ctx->v_V != d->V || ctx->v_dtype != d->dtype ||
+      ctx->v_h_llm != d->h_llm)
+    return SPECSTEER_ERR_ORDER;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  RoundParams p = slab_params(ctx, d, 0, d->B);
+  if (launch_cloud_topk(p, d->dtype, k, topk_idx, topk_val, (cudaStream_t)cuda_stream) != cudaSuccess)
+    return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_edge_resample(specsteer_ctx* ctx, const specsteer_round_desc* d, int32_t k,
+                                         const int32_t* topk_idx, const float* topk_val, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if (k < 1 || k > SPECSTEER_TOPK_MAX || !topk_idx || !topk_val) return SPECSTEER_ERR_INVALID_ARG;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (!ctx->verified || ctx->v_B != d->B || ctx->v_K != d->K || ctx->v_V != d->V || ctx->v_dtype != d->dtype ||
+      ctx->v_h_llm != d->h_llm)
+    return SPECSTEER_ERR_ORDER;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  RoundParams p = slab_params(ctx, d, 0, d->B);
+  if (launch_edge_resample(p, d->dtype, k, topk_idx, topk_val, (cudaStream_t)cuda_stream) != cudaSuccess)
+    return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
+  return SPECSTEER_OK;
+}
+
 specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_desc* h, void* cuda_stream) {
   specsteer_status st = check_desc(ctx, h);
   if (st != SPECSTEER_OK) return st;
