@@ -258,11 +258,39 @@ def run_cuda(args, rank, world, local_rank):
     value = world * positions / (ms_per_step * 1e-3)
 
     if args.kernels_only:
+        extra = {}
+        if args.topk:
+            # the top-k split recovery in place of recover_sample: the cloud kernel reads two rows per sampling request
+            k = args.topk
+            tidx = torch.empty((spec.B, k), dtype=torch.int32, device=dev)
+            tval = torch.empty((spec.B, k), dtype=torch.float32, device=dev)
+            n = min(args.steps, 100)
+            ea = [torch.cuda.Event(enable_timing=True) for _ in range(3 * n)]
+            for i in range(n + 3):
+                d = sets[i % n_sets][1]
+                ctx.verify_round(d, stream)
+                j = 3 * (i - 3)
+                if i >= 3:
+                    ea[j].record(stream)
+                ctx.cloud_topk(d, tidx, tval, stream)
+                if i >= 3:
+                    ea[j + 1].record(stream)
+                ctx.edge_resample(d, tidx, tval, stream)
+                if i >= 3:
+                    ea[j + 2].record(stream)
+            barrier()
+            cloud_ms = sum(ea[3 * i].elapsed_time(ea[3 * i + 1]) for i in range(n)) / n
+            edge_ms = sum(ea[3 * i + 1].elapsed_time(ea[3 * i + 2]) for i in range(n)) / n
+            topk_bytes = 2 * spec.B * spec.V * spec.elem_bytes      # with the bonus row every request samples
+            extra = {"topk_k": k, "cloud_topk_ms": cloud_ms, "cloud_topk_gbs": topk_bytes / (cloud_ms * 1e-3) / 1e9,
+                     "cloud_topk_bytes": topk_bytes, "edge_resample_ms": edge_ms}
         sampler.stop()
         if rank == 0:
-            print(json.dumps({"workload": spec.name, "outputs": "lean" if args.lean else "all", "ms_per_step": ms_per_step, "verify_kernel_ms": kernel_ms,
-                              "verify_gbs": logit_bytes / (kernel_ms * 1e-3) / 1e9, "positions_per_s": value,
-                              "clocks": sampler.summary()}), flush=True)
+            line = {"workload": spec.name, "outputs": "lean" if args.lean else "all", "ms_per_step": ms_per_step,
+                    "verify_kernel_ms": kernel_ms, "verify_gbs": logit_bytes / (kernel_ms * 1e-3) / 1e9,
+                    "positions_per_s": value, "clocks": sampler.summary()}
+            line.update(extra)
+            print(json.dumps(line), flush=True)
         if dist is not None:
             dist.barrier()
             dist.destroy_process_group()
@@ -361,6 +389,8 @@ def main():
     ap.add_argument("--requests", type=int, default=0, help="override B (reduced batch for profiler captures)")
     ap.add_argument("--lean", action="store_true",
                     help="request only the outputs Algorithm 1 needs (no logp_plus, log_z): three normalisers per row")
+    ap.add_argument("--topk", type=int, default=0,
+                    help="with --kernels-only: also time the top-k split recovery (cloud + edge kernels) with this k")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the device-resident steps and print a short line (profiling aid)")
     args = ap.parse_args()

@@ -113,7 +113,7 @@ typedef struct {
 
 /* Create a context on CUDA device `device` able to run rounds up to the given maxima.  Allocates the
  * workspace (row normalisers and per-chunk partial sums; about
- * max_B*(max_K+1)*(16 + 32*ceil(max_V/512)) bytes) once; no later call of the device-pointer entry points allocates.
+ * max_B*(max_K+1)*(16 + 32*ceil(max_V/512)) bytes, plus 4 KB per request for specsteer_cloud_topk) once; no later call of the device-pointer entry points allocates.
  * Errors: INVALID_ARG (NULL out, non-positive maxima), CUDA, WORKSPACE. */
 specsteer_status specsteer_ctx_create(specsteer_ctx **out, int device, int32_t max_B, int32_t max_K, int32_t max_V);
 

@@ -20,6 +20,8 @@ struct specsteer_ctx {
   float* lse2;
   int* status_ws;
   int* dev_error;
+  void* topk_lists;   // [max_B][kTopkMaxSplit][32] keys of the split top-k selection
+  int* topk_count;    // [max_B], zero between launches
   // last verified round, for the order check
   bool verified;
   int v_B, v_K, v_V, v_dtype;
@@ -175,7 +177,9 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   const size_t b_part = align_up(rows * nch * 8 * sizeof(float), 256);
   const size_t b_lse = align_up(rows * 4 * sizeof(float), 256);
   const size_t b_st = align_up((size_t)max_B * sizeof(int), 256);
-  c->ws_bytes = b_part + b_lse + b_st + 256;
+  const size_t b_tl = align_up((size_t)max_B * kTopkMaxSplit * 32 * sizeof(unsigned long long), 256);
+  const size_t b_tc = align_up((size_t)max_B * sizeof(int), 256);
+  c->ws_bytes = b_part + b_lse + b_st + 256 + b_tl + b_tc;
   if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
     cudaGetLastError();
     delete c;
@@ -185,7 +189,9 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   c->part = (float*)w; w += b_part;
   c->lse2 = (float*)w; w += b_lse;
   c->status_ws = (int*)w; w += b_st;
-  c->dev_error = (int*)w;
+  c->dev_error = (int*)w; w += 256;
+  c->topk_lists = (void*)w; w += b_tl;
+  c->topk_count = (int*)w;
   if (cudaMemset(c->ws, 0, c->ws_bytes) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) {
     cudaFree(c->ws);
     delete c;
@@ -249,7 +255,8 @@ specsteer_status specsteer_cloud_topk(specsteer_ctx* ctx, const specsteer_round_
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
   RoundParams p = slab_params(ctx, d, 0, d->B);
-  if (launch_cloud_topk(p, d->dtype, k, topk_idx, topk_val, (cudaStream_t)cuda_stream) != cudaSuccess)
+  if (launch_cloud_topk(p, d->dtype, k, topk_idx, topk_val, ctx->topk_lists, ctx->topk_count, ctx->li.sm_count,
+                        (cudaStream_t)cuda_stream) != cudaSuccess)
     return SPECSTEER_ERR_CUDA;
   ctx->launches += 1;
   return SPECSTEER_OK;

@@ -48,7 +48,10 @@ struct LaunchInfo {
 // ev_begin / ev_end, when not null, are recorded on `s` just before and just after the streaming kernel.
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
                           int* n_launches, cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
-cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_idx, float* topk_val, cudaStream_t s);
+constexpr int kTopkMaxSplit = 16;  // CTAs that may share one row in specsteer_cloud_topk
+// lists_ws: [B][kTopkMaxSplit][32] 64-bit keys; count_ws: [B] counters, zero between launches
+cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_idx, float* topk_val,
+                              void* lists_ws, int* count_ws, int sm_count, cudaStream_t s);
 cudaError_t launch_edge_resample(const RoundParams& p, int dtype, int k, const int* topk_idx, const float* topk_val,
                                  cudaStream_t s);
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);

@@ -39,15 +39,48 @@ __device__ __forceinline__ void warp_insert(u64& mykey, u64 nk, int lane) {
   }
 }
 
+__device__ __forceinline__ u64 umax64(u64 a, u64 b) { return a > b ? a : b; }
+__device__ __forceinline__ u64 umin64(u64 a, u64 b) { return a < b ? a : b; }
+
+// Sort a bitonic sequence held one key per lane into descending order (five compare-exchange stages).
+__device__ __forceinline__ u64 bitonic_merge_desc(u64 x, int lane) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const u64 y = __shfl_xor_sync(kFullMask, x, o);
+    x = (lane & o) ? umin64(x, y) : umax64(x, y);
+  }
+  return x;
+}
+// Sort 32 arbitrary keys, one per lane, into descending order.
+__device__ __forceinline__ u64 bitonic_sort_desc(u64 x, int lane) {
+#pragma unroll
+  for (int sz = 2; sz <= 32; sz <<= 1) {
+    const bool up = (lane & sz) != 0 && sz < 32;   // direction of this lane's block: alternate, final pass descending
+#pragma unroll
+    for (int o = sz >> 1; o > 0; o >>= 1) {
+      const u64 y = __shfl_xor_sync(kFullMask, x, o);
+      const bool take_min = ((lane & o) != 0) != up;
+      x = take_min ? umin64(x, y) : umax64(x, y);
+    }
+  }
+  return x;
+}
+// The 32 largest of two descending lists: `other_rev` is the second list read back to front.
+__device__ __forceinline__ u64 merge_top32(u64 mine, u64 other_rev, int lane) {
+  return bitonic_merge_desc(umax64(mine, other_rev), lane);
+}
+
 struct TopState {
   u64 key;      // this lane's list entry
   float tau;    // value of the 32nd entry, -inf while the list is not full
 };
 
-__device__ __forceinline__ void refresh_tau(TopState& st) {
+// The threshold only ever rises: it may already sit above the list's own 32nd value (CTA-wide bound).
+__device__ __forceinline__ void refresh_tau_floor(TopState& st) {
   const u64 last = __shfl_sync(kFullMask, st.key, 31);
-  st.tau = last ? order_val((uint32_t)(last >> 32)) : kNegInf;
+  if (last) st.tau = fmaxf(st.tau, order_val((uint32_t)(last >> 32)));
 }
+__device__ __forceinline__ void refresh_tau(TopState& st) { refresh_tau_floor(st); }
 
 // One candidate value per lane (NaN = none): those not below the warp's threshold are inserted one by one.
 __device__ __forceinline__ void offer(TopState& st, float h, int idx, int lane) {
@@ -68,19 +101,19 @@ __device__ __forceinline__ float h_cloud(float l, float m, float nbeta) { return
 template <typename T> struct Vec;
 template <> struct Vec<float> {
   static constexpr int N = 4;
-  static __device__ __forceinline__ void load(const float* p, float (&x)[4]) {
-    const float4 v = __ldcs(reinterpret_cast<const float4*>(p));
-    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  static __device__ __forceinline__ void unpack(const uint4& v, float (&x)[4]) {
+    x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
   }
 };
 template <> struct Vec<uint16_t> {
   static constexpr int N = 8;
-  static __device__ __forceinline__ void load(const uint16_t* p, float (&x)[8]) {
-    const uint4 v = __ldcs(reinterpret_cast<const uint4*>(p));
+  static __device__ __forceinline__ void unpack(const uint4& v, float (&x)[8]) {
     x[0] = bf16lo(v.x); x[1] = bf16hi(v.x); x[2] = bf16lo(v.y); x[3] = bf16hi(v.y);
     x[4] = bf16lo(v.z); x[5] = bf16hi(v.z); x[6] = bf16lo(v.w); x[7] = bf16hi(v.w);
   }
 };
+// the four 16-byte vectors a lane holds for one step: two of h_LLM, two of h_SLM-
+struct StepRegs { uint4 l0, m0, l1, m1; };
 
 struct TopReq {
   int n;        // row to recover from
@@ -97,16 +130,36 @@ __device__ __forceinline__ TopReq top_request(const RoundParams& p, int b) {
   return r;
 }
 
+// The 32 largest keys of all sixteen warps' lists, left sorted in lists[0][*].  Every thread of the CTA calls it.
+__device__ __forceinline__ void cta_merge(u64 (*lists)[32], u64 mykey, int warp, int lane) {
+  lists[warp][lane] = mykey;
+  __syncthreads();
+  u64 cur = mykey;
+#pragma unroll
+  for (int stride = 1; stride < kTopWarps; stride <<= 1) {
+    if ((warp & (2 * stride - 1)) == 0) {
+      cur = merge_top32(cur, lists[warp + stride][31 - lane], lane);
+      lists[warp][lane] = cur;
+    }
+    __syncthreads();
+  }
+}
+
+// Grid (B, S): CTA (b, s) selects over the s-th slice of the row.  With S > 1 the CTAs of a request leave their
+// lists in `lists_ws` [B][S][32] and the one that finishes last (a counter per request in `count_ws`, which it
+// puts back to zero) merges them; nobody waits for anybody.
 template <typename T>
-__global__ void __launch_bounds__(kTopThreads) cloud_topk_kernel(const RoundParams p, int k, int* topk_idx,
-                                                                  float* topk_val) {
+__global__ void __launch_bounds__(kTopThreads, 2) cloud_topk_kernel(const RoundParams p, int k, int* topk_idx,
+                                                                  float* topk_val, u64* lists_ws, int* count_ws) {
   constexpr int NE = Vec<T>::N;
   __shared__ u64 lists[kTopWarps][32];
-  const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  __shared__ int is_last;
+  const int b = blockIdx.x, split = blockIdx.y, S = gridDim.y;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   pdl_wait();
   const TopReq rq = top_request(p, b);
   if (!rq.sample) {
-    if (tid < k) { topk_idx[(long long)b * k + tid] = -1; topk_val[(long long)b * k + tid] = kNegInf; }
+    if (split == 0 && tid < k) { topk_idx[(long long)b * k + tid] = -1; topk_val[(long long)b * k + tid] = kNegInf; }
     return;
   }
   const long long off = (long long)b * p.ld_req + (long long)rq.n * p.ld_row;
@@ -120,45 +173,111 @@ __global__ void __launch_bounds__(kTopThreads) cloud_topk_kernel(const RoundPara
 
   const bool aligned = ((reinterpret_cast<uintptr_t>(hl) | reinterpret_cast<uintptr_t>(hm)) & 15u) == 0;
   const int nvec = aligned ? p.V / NE : 0;
-  // main part: warp w takes vectors [w*32, w*32+32) + j*512; two vectors per stream in flight per lane
-  for (int base = warp * 32; base < nvec; base += 2 * kTopThreads) {
-    const int v0 = base + lane, v1 = v0 + kTopThreads;
+  const int per = (nvec + S - 1) / S;
+  const int vbeg = min(split * per, nvec), vend = min(vbeg + per, nvec);
+  // main part: warp w takes vectors vbeg + [w*32, w*32+32) + j*512, two per stream and lane per step; the loads
+  // of the next step are issued before this step's entries are looked at
+  constexpr int kStep = 2 * kTopThreads;   // vectors the CTA consumes per step
+  // a lane without a vector holds NaN patterns: they never pass a comparison, so the loop needs no range tests
+  const uint32_t nanw = sizeof(T) == 4 ? 0x7fc00000u : 0x7fc07fc0u;
+  const uint4 nan4 = make_uint4(nanw, nanw, nanw, nanw);
+  auto fetch = [&](int bs, StepRegs& r) {
+    const int v0 = bs + lane, v1 = v0 + kTopThreads;
+    if (v0 < vend) {
+      r.l0 = __ldcs(reinterpret_cast<const uint4*>(hl + (size_t)v0 * NE));
+      r.m0 = __ldcs(reinterpret_cast<const uint4*>(hm + (size_t)v0 * NE));
+    } else {
+      r.l0 = nan4; r.m0 = nan4;
+    }
+    if (v1 < vend) {
+      r.l1 = __ldcs(reinterpret_cast<const uint4*>(hl + (size_t)v1 * NE));
+      r.m1 = __ldcs(reinterpret_cast<const uint4*>(hm + (size_t)v1 * NE));
+    } else {
+      r.l1 = nan4; r.m1 = nan4;
+    }
+  };
+  // all warps run the same number of steps (a warp without vectors offers nothing) so that they can meet at the
+  // steps 1, 7, 31, ... to raise the common threshold to the 32nd value of everything the CTA has seen
+  const int steps = (vend - vbeg + kStep - 1) / kStep;
+  int next_sync = 1;
+  // one step: the loads run two steps ahead (`refill`), the arithmetic looks at `use`.  Hot part: one fused
+  // multiply-add and one compare per entry; only a warp in which some entry reaches the threshold goes on.
+  auto step = [&](int it, const StepRegs& use, StepRegs& refill) {
+    const int bs = vbeg + warp * 32 + it * kStep;
+    fetch(bs + 2 * kStep, refill);
     float l0[NE], m0[NE], l1[NE], m1[NE];
-    const bool ok0 = v0 < nvec, ok1 = v1 < nvec;
-    if (ok0) { Vec<T>::load(hl + (size_t)v0 * NE, l0); Vec<T>::load(hm + (size_t)v0 * NE, m0); }
-    if (ok1) { Vec<T>::load(hl + (size_t)v1 * NE, l1); Vec<T>::load(hm + (size_t)v1 * NE, m1); }
-    float h0[NE], h1[NE];
-    float best = kNegInf;
+    Vec<T>::unpack(use.l0, l0); Vec<T>::unpack(use.m0, m0);
+    Vec<T>::unpack(use.l1, l1); Vec<T>::unpack(use.m1, m1);
+    bool hit = false;
 #pragma unroll
     for (int e = 0; e < NE; ++e) {
-      h0[e] = ok0 ? h_cloud(l0[e], m0[e], nbeta) : qnan;
-      h1[e] = ok1 ? h_cloud(l1[e], m1[e], nbeta) : qnan;
-      best = fmaxf(best, fmaxf(h0[e], h1[e]));   // fmaxf drops NaN
+      hit |= fmaf(nbeta, m0[e], l0[e]) >= st.tau;
+      hit |= fmaf(nbeta, m1[e], l1[e]) >= st.tau;
     }
-    if (!__any_sync(kFullMask, best >= st.tau)) continue;
+    if (__any_sync(kFullMask, hit)) {
+      const int v0 = bs + lane, v1 = v0 + kTopThreads;
 #pragma unroll
-    for (int e = 0; e < NE; ++e) offer(st, h0[e], v0 * NE + e, lane);
+      for (int e = 0; e < NE; ++e) offer(st, h_cloud(l0[e], m0[e], nbeta), v0 * NE + e, lane);
 #pragma unroll
-    for (int e = 0; e < NE; ++e) offer(st, h1[e], v1 * NE + e, lane);
+      for (int e = 0; e < NE; ++e) offer(st, h_cloud(l1[e], m1[e], nbeta), v1 * NE + e, lane);
+    }
+    if (it == next_sync && it + 1 < steps) {
+      next_sync = 4 * next_sync + 3;
+      cta_merge(lists, st.key, warp, lane);
+      const u64 last = lists[0][31];
+      if (last) st.tau = fmaxf(st.tau, order_val((uint32_t)(last >> 32)));
+      __syncthreads();   // lists[] is reused by the next merge
+    }
+  };
+  StepRegs ra, rb, rc;
+  fetch(vbeg + warp * 32, ra);
+  fetch(vbeg + warp * 32 + kStep, rb);
+  {
+    // Bootstrap of the threshold: every lane's maximum over its first entries is an entry of the row, so the
+    // 32nd largest of the CTA's 512 lane maxima has at least 32 entries at or above it.  Step 0 then starts with a
+    // threshold almost as tight as the exact one and only a few dozen entries per CTA take the insertion path.
+    float l0[NE], m0[NE], l1[NE], m1[NE];
+    Vec<T>::unpack(ra.l0, l0); Vec<T>::unpack(ra.m0, m0);
+    Vec<T>::unpack(ra.l1, l1); Vec<T>::unpack(ra.m1, m1);
+    float lm = kNegInf;
+#pragma unroll
+    for (int e = 0; e < NE; ++e) lm = fmaxf(lm, fmaxf(h_cloud(l0[e], m0[e], nbeta), h_cloud(l1[e], m1[e], nbeta)));
+    const u64 mk = bitonic_sort_desc((u64)order_key(lm) << 32, lane);
+    cta_merge(lists, mk, warp, lane);
+    st.tau = order_val((uint32_t)(lists[0][31] >> 32));
+    __syncthreads();
   }
-  // what the vectors did not cover (the tail, or the whole row when it is not 16-byte aligned)
-  for (int base = nvec * NE + warp * 32; base < p.V; base += kTopThreads) {
-    const int v = base + lane;
-    const float h = v < p.V ? h_cloud(load_logit<T>(hl, v), load_logit<T>(hm, v), nbeta) : qnan;
-    offer(st, h, v, lane);
+#pragma unroll 1
+  for (int it = 0; it < steps; ++it) {
+    step(it, ra, rc);
+    ra = rb;   // rotate: sixteen register moves per step keep the loop body single (it is large)
+    rb = rc;
   }
-  lists[warp][lane] = st.key;
-  __syncthreads();
+  // what the vectors did not cover (the tail, or the whole row when it is not 16-byte aligned): last slice
+  if (split == S - 1) {
+    for (int bs = nvec * NE + warp * 32; bs < p.V; bs += kTopThreads) {
+      const int v = bs + lane;
+      const float h = v < p.V ? h_cloud(load_logit<T>(hl, v), load_logit<T>(hm, v), nbeta) : qnan;
+      offer(st, h, v, lane);
+    }
+  }
+  cta_merge(lists, st.key, warp, lane);
   if (warp != 0) return;
-  for (int w = 1; w < kTopWarps; ++w) {
-    const u64 nk = lists[w][lane];
-    const u64 last = __shfl_sync(kFullMask, st.key, 31);
-    unsigned cand = __ballot_sync(kFullMask, nk > last);   // an empty slot (0) never beats anything
-    while (cand) {
-      const int src = __ffs(cand) - 1;
-      cand &= cand - 1;
-      warp_insert(st.key, __shfl_sync(kFullMask, nk, src), lane);
+  st.key = lists[0][lane];
+  if (S > 1) {
+    u64* mine = lists_ws + ((size_t)b * S + split) * 32;
+    mine[lane] = st.key;
+    __threadfence();
+    __syncwarp();
+    if (lane == 0) is_last = (atomicAdd(count_ws + b, 1) == S - 1) ? 1 : 0;
+    __syncwarp();
+    if (!is_last) return;
+    __threadfence();
+    for (int s2 = 0; s2 < S; ++s2) {
+      if (s2 == split) continue;
+      st.key = merge_top32(st.key, __ldcg(lists_ws + ((size_t)b * S + s2) * 32 + (31 - lane)), lane);
     }
+    if (lane == 0) count_ws[b] = 0;
   }
   if (lane < k) {
     const bool have = st.key != 0ull;
@@ -216,9 +335,32 @@ __global__ void __launch_bounds__(32) edge_resample_kernel(const RoundParams p, 
   }
 }
 
-cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_idx, float* topk_val, cudaStream_t s) {
-  if (dtype == SPECSTEER_F32) cloud_topk_kernel<float><<<p.B, kTopThreads, 0, s>>>(p, k, topk_idx, topk_val);
-  else cloud_topk_kernel<uint16_t><<<p.B, kTopThreads, 0, s>>>(p, k, topk_idx, topk_val);
+cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_idx, float* topk_val,
+                              void* lists_ws, int* count_ws, int sm_count, cudaStream_t s) {
+  // Two CTAs fit on an SM.  Few requests: split each row over as many CTAs as still fit at once (one wave), but
+  // keep at least 4096 vectors (64 KB per stream) per slice.  Many requests: split so that the last wave is full.
+  const int nvec = p.V / (dtype == SPECSTEER_F32 ? 4 : 8);
+  const int slots = 2 * sm_count;
+  int s_cap = nvec / 4096 > 1 ? nvec / 4096 : 1;
+  if (s_cap > kTopkMaxSplit) s_cap = kTopkMaxSplit;
+  int S = 1;
+  if (p.B * 2 <= slots) {
+    S = slots / p.B;
+  } else if (p.B > slots) {
+    double best = 1e30;
+    for (int c = 1; c <= 4; ++c) {
+      const int items = p.B * c, waves = (items + slots - 1) / slots;
+      const double cost = (double)waves * slots / items + 0.03 * (c - 1);   // idle share of the last wave + split overhead
+      if (cost < best) { best = cost; S = c; }
+    }
+  }
+  if (S > s_cap) S = s_cap;
+  if (S < 1 || !lists_ws || !count_ws) S = 1;
+  const dim3 grid(p.B, S);
+  if (dtype == SPECSTEER_F32)
+    cloud_topk_kernel<float><<<grid, kTopThreads, 0, s>>>(p, k, topk_idx, topk_val, (u64*)lists_ws, count_ws);
+  else
+    cloud_topk_kernel<uint16_t><<<grid, kTopThreads, 0, s>>>(p, k, topk_idx, topk_val, (u64*)lists_ws, count_ws);
   return cudaGetLastError();
 }
 
