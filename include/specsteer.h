@@ -157,6 +157,33 @@ specsteer_status specsteer_cloud_topk(specsteer_ctx *ctx, const specsteer_round_
 specsteer_status specsteer_edge_resample(specsteer_ctx *ctx, const specsteer_round_desc *desc, int32_t k,
                                          const int32_t *topk_idx, const float *topk_val, void *cuda_stream);
 
+/* Vocabulary-sharded rounds: the logits arrive split along V over n_shards GPUs (a tensor-parallel LM head), GPU g
+ * holding [B][K+1][V_g] for the global token ids [vocab_offset_g, vocab_offset_g + V_g).  The paper runs its
+ * Generalist and the public Specialist copy side by side on the cloud (deployment appendix) and says nothing about
+ * sharding them; this is the same round (Algorithm 1 phases 2 and 3, Eq. 7 / Eq. 6, Eq. 8) with one exchange step:
+ *   1. specsteer_shard_verify_local on every GPU: streams the local shard and writes, for every row, a 64-byte
+ *      partial (largest exponent and float64 sum of the four normalisers over the shard, and the drafted token's
+ *      three logits if the token lies in the shard) into row_partials [B][K+1][64 bytes] (device).
+ *   2. the caller all-gathers the partials into gathered [n_shards][B][K+1][64 bytes] on every GPU (NCCL).
+ *   3. specsteer_shard_verify_combine on every GPU: identical arithmetic everywhere; writes every output
+ *      specsteer_verify_round writes.  desc is the LOCAL descriptor (V = V_g); draft_tokens hold GLOBAL ids.
+ *   4. specsteer_shard_recover_local on every GPU: all GPUs place the CDF target among the shards from the
+ *      gathered partials; the owner samples within its shard and writes the global token id, rec_logprob,
+ *      out_tokens, n_out; the others write -1, -inf, the accepted prefix with -1 in the new slot, and accept_len,
+ *      so that an element-wise MAX all-reduce of those four arrays gives every GPU the result.
+ * STEER recovery only; B <= 1024; n_shards <= SPECSTEER_MAX_SHARDS.
+ * Errors: INVALID_ARG, UNSUPPORTED, ORDER (step out of sequence), CUDA. */
+#define SPECSTEER_MAX_SHARDS 32
+#define SPECSTEER_SHARD_PARTIAL_BYTES 64
+specsteer_status specsteer_shard_verify_local(specsteer_ctx *ctx, const specsteer_round_desc *desc, int32_t vocab_offset,
+                                              void *row_partials, void *cuda_stream);
+specsteer_status specsteer_shard_verify_combine(specsteer_ctx *ctx, const specsteer_round_desc *desc, const void *gathered,
+                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                                int32_t vocab_total, void *cuda_stream);
+specsteer_status specsteer_shard_recover_local(specsteer_ctx *ctx, const specsteer_round_desc *desc, const void *gathered,
+                                               int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                               int32_t vocab_total, void *cuda_stream);
+
 /* Whole round from HOST memory: every pointer in `desc` is a HOST pointer (pinned memory makes the copies
  * asynchronous).  Copies inputs to device staging buffers owned by the context (allocated on the first
  * call, sized for the context's maxima: 3*max_B*(max_K+1)*max_V elements of 4 bytes), runs verification and

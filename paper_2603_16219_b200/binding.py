@@ -28,7 +28,10 @@ EXPORTS = (
     "specsteer_ctx_launch_count", "specsteer_status_string", "specsteer_version",
     "specsteer_verify_round_static", "specsteer_ctx_time_streaming",
     "specsteer_cloud_topk", "specsteer_edge_resample",
+    "specsteer_shard_verify_local", "specsteer_shard_verify_combine", "specsteer_shard_recover_local",
 )
+SHARD_PARTIAL_BYTES = 64
+MAX_SHARDS = 32
 TOPK_MAX = 32
 
 
@@ -82,6 +85,12 @@ def load_library(path: Optional[str] = None):
     lib.specsteer_cloud_topk.restype = C.c_int
     lib.specsteer_edge_resample.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p]
     lib.specsteer_edge_resample.restype = C.c_int
+    lib.specsteer_shard_verify_local.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_int32, C.c_void_p, C.c_void_p]
+    lib.specsteer_shard_verify_local.restype = C.c_int
+    for name in ("specsteer_shard_verify_combine", "specsteer_shard_recover_local"):
+        fn = getattr(lib, name)
+        fn.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+        fn.restype = C.c_int
     lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.specsteer_ctx_time_streaming.restype = C.c_int
     lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
@@ -220,6 +229,33 @@ class Context:
         _check(self._lib.specsteer_edge_resample(self._h, C.byref(desc), k, C.c_void_p(topk_idx.data_ptr()),
                                                  C.c_void_p(topk_val.data_ptr()), self._stream(stream)),
                "specsteer_edge_resample")
+
+    def shard_verify_local(self, desc: RoundDesc, vocab_offset: int, row_partials: torch.Tensor, stream=None):
+        """Step 1 of a vocabulary-sharded round: this shard's 64-byte partial per row into row_partials
+        (uint8 [B, K+1, 64])."""
+        if row_partials.dtype != torch.uint8 or tuple(row_partials.shape) != (desc.B, desc.K + 1, SHARD_PARTIAL_BYTES) \
+                or not row_partials.is_contiguous():
+            raise ValueError("row_partials must be a contiguous uint8 tensor [B, K+1, 64]")
+        _check(self._lib.specsteer_shard_verify_local(self._h, C.byref(desc), int(vocab_offset),
+                                                      C.c_void_p(row_partials.data_ptr()), self._stream(stream)),
+               "specsteer_shard_verify_local")
+
+    def _shard_call(self, fn, name, desc, gathered, shard_rank, vocab_offset, vocab_total, stream):
+        if gathered.dtype != torch.uint8 or gathered.dim() != 4 or not gathered.is_contiguous() or \
+                tuple(gathered.shape[1:]) != (desc.B, desc.K + 1, SHARD_PARTIAL_BYTES):
+            raise ValueError("gathered must be a contiguous uint8 tensor [n_shards, B, K+1, 64]")
+        _check(fn(self._h, C.byref(desc), C.c_void_p(gathered.data_ptr()), int(gathered.shape[0]), int(shard_rank),
+                  int(vocab_offset), int(vocab_total), self._stream(stream)), name)
+
+    def shard_verify_combine(self, desc, gathered, shard_rank, vocab_offset, vocab_total, stream=None):
+        """Step 3: acceptance from the gathered partials of all shards (same outputs as verify_round)."""
+        self._shard_call(self._lib.specsteer_shard_verify_combine, "specsteer_shard_verify_combine", desc, gathered,
+                         shard_rank, vocab_offset, vocab_total, stream)
+
+    def shard_recover_local(self, desc, gathered, shard_rank, vocab_offset, vocab_total, stream=None):
+        """Step 4: the shard that holds the CDF target samples; the others write values a MAX-reduce ignores."""
+        self._shard_call(self._lib.specsteer_shard_recover_local, "specsteer_shard_recover_local", desc, gathered,
+                         shard_rank, vocab_offset, vocab_total, stream)
 
     def round_host(self, desc: RoundDesc, stream=None):
         _check(self._lib.specsteer_round_host(self._h, C.byref(desc), self._stream(stream)), "specsteer_round_host")

@@ -28,6 +28,7 @@ struct specsteer_ctx {
   const void* v_h_llm;
   uint64_t launches;
   bool poisoned;
+  bool shard_streamed;   // specsteer_shard_verify_local ran for the shape in v_*
   // host-round staging
   void* stage;
   size_t stage_bytes;
@@ -219,6 +220,7 @@ specsteer_status specsteer_verify_round(specsteer_ctx* ctx, const specsteer_roun
   if (st != SPECSTEER_OK) return st;
   if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
   ctx->verified = false;
+  ctx->shard_streamed = false;
   if (d->B == 0) { ctx->verified = true; ctx->v_B = 0; ctx->v_K = d->K; ctx->v_V = d->V; ctx->v_dtype = d->dtype; ctx->v_h_llm = d->h_llm; return SPECSTEER_OK; }
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
@@ -240,6 +242,93 @@ specsteer_status specsteer_recover_sample(specsteer_ctx* ctx, const specsteer_ro
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
   return do_recover(ctx, d, (cudaStream_t)cuda_stream);
+}
+
+// ---- vocabulary-sharded path -------------------------------------------------------------------------
+namespace {
+bool same_round(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
+  return ctx->v_B == d->B && ctx->v_K == d->K && ctx->v_V == d->V && ctx->v_dtype == d->dtype && ctx->v_h_llm == d->h_llm;
+}
+void remember_round(specsteer_ctx* ctx, const specsteer_round_desc* d) {
+  ctx->v_B = d->B; ctx->v_K = d->K; ctx->v_V = d->V; ctx->v_dtype = d->dtype; ctx->v_h_llm = d->h_llm;
+}
+specsteer_status check_shard_args(const specsteer_round_desc* d, const void* gathered, int32_t n_shards, int32_t rank,
+                                  int32_t vocab_offset, int32_t vocab_total) {
+  if (!gathered || n_shards < 1 || n_shards > SPECSTEER_MAX_SHARDS || rank < 0 || rank >= n_shards) return SPECSTEER_ERR_INVALID_ARG;
+  if (vocab_offset < 0 || vocab_total < d->V || (int64_t)vocab_offset + d->V > vocab_total) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->B > kMaxSlabB) return SPECSTEER_ERR_UNSUPPORTED;
+  return SPECSTEER_OK;
+}
+}  // namespace
+
+specsteer_status specsteer_shard_verify_local(specsteer_ctx* ctx, const specsteer_round_desc* d, int32_t vocab_offset,
+                                              void* row_partials, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if (!row_partials || vocab_offset < 0 || d->B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  ctx->verified = false;
+  ctx->shard_streamed = false;
+  if (d->B > 0) {
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SPECSTEER_ERR_CUDA;
+    RoundParams p = slab_params(ctx, d, 0, d->B);
+    p.need_p = 1;
+    p.vocab_offset = vocab_offset;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    if (launch_verify_stream(p, d->dtype, rows_aligned(d), ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    if (launch_shard_rows(p, d->dtype, (ShardPartial*)row_partials, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    ctx->launches += 2;
+  }
+  remember_round(ctx, d);
+  ctx->shard_streamed = true;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_shard_verify_combine(specsteer_ctx* ctx, const specsteer_round_desc* d, const void* gathered,
+                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                                int32_t vocab_total, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if ((st = check_shard_args(d, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (!ctx->shard_streamed || !same_round(ctx, d)) return SPECSTEER_ERR_ORDER;
+  if (d->B > 0) {
+    DeviceGuard g(ctx->device);
+    if (!g.ok) return SPECSTEER_ERR_CUDA;
+    RoundParams p = slab_params(ctx, d, 0, d->B);
+    p.need_p = 1;
+    p.shard_parts = (const ShardPartial*)gathered;
+    p.n_shards = n_shards; p.shard_rank = shard_rank;
+    p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;
+    if (launch_epilogue(p, d->dtype, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    ctx->launches += 1;
+  }
+  ctx->verified = true;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_shard_recover_local(specsteer_ctx* ctx, const specsteer_round_desc* d, const void* gathered,
+                                               int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                               int32_t vocab_total, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if ((st = check_shard_args(d, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
+  if (d->recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (!ctx->verified || !ctx->shard_streamed || !same_round(ctx, d)) return SPECSTEER_ERR_ORDER;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  RoundParams p = slab_params(ctx, d, 0, d->B);
+  p.need_p = 1;
+  p.shard_parts = (const ShardPartial*)gathered;
+  p.n_shards = n_shards; p.shard_rank = shard_rank;
+  p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;
+  int nl = 0;
+  if (launch_recover(p, d->dtype, ctx->li, (cudaStream_t)cuda_stream, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += nl;
+  return SPECSTEER_OK;
 }
 
 specsteer_status specsteer_cloud_topk(specsteer_ctx* ctx, const specsteer_round_desc* d, int32_t k, int32_t* topk_idx,

@@ -12,6 +12,17 @@ constexpr int kChunkBF16 = 1024;
 constexpr int kChunkMin = 512;
 constexpr int kMaxSlabB = 1024;  // requests handled by one launch (per-request tables live in shared memory)
 
+// What one vocabulary shard knows about one row (64 bytes; the unit of the all-gather in the sharded path):
+// for the four normalisers the largest exponent and the float64 sum relative to it (value s * 2^m), and the
+// three logits of the drafted token when that token lies in the shard.
+struct ShardPartial {
+  float m[4];
+  double s[4];
+  float tok_logit[3];  // h_LLM, h_SLM+, h_SLM- at the drafted token
+  int has_token;
+};
+static_assert(sizeof(ShardPartial) == 64, "the sharded path exchanges 64 bytes per row and shard");
+
 struct RoundParams {
   int B, K, V;
   long long ld_row, ld_req;  // elements
@@ -37,6 +48,10 @@ struct RoundParams {
   float* lse2;        // [B*(K+1)][4]            base-2 log-normalisers {L,P,M,R}
   int* status_ws;     // [B]                     request status when the caller passes no req_status
   int* dev_error;     // [1]                     set when a bounded wait gave up
+  // vocabulary-sharded path (n_shards == 0: the tensors hold the whole vocabulary)
+  const ShardPartial* shard_parts;  // [n_shards][B][K+1] gathered partials
+  int n_shards, shard_rank;
+  int vocab_offset, vocab_total;    // this shard covers global ids [vocab_offset, vocab_offset + V)
 };
 
 struct LaunchInfo {
@@ -54,6 +69,12 @@ cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_
                               void* lists_ws, int* count_ws, int sm_count, cudaStream_t s);
 cudaError_t launch_edge_resample(const RoundParams& p, int dtype, int k, const int* topk_idx, const float* topk_val,
                                  cudaStream_t s);
+// the streaming kernel alone (partial records into the workspace), no epilogue
+cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s);
+// per-row ShardPartial of this shard from its partial records: out[B][K+1]
+cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out, cudaStream_t s);
+// the per-request epilogue alone (reads p.shard_parts when p.n_shards > 0)
+cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);
 
 }  // namespace specsteer

@@ -16,6 +16,8 @@ struct PickShared {
   double base, target, W;
   int jstar, jlast;
   int tok_min, tok_max_pos;
+  int plan_owner;            // sharded vocabulary: the shard that holds the CDF target, -1 if nothing can be sampled
+  double plan_target, plan_W;  // the target within that shard, and the weight of the whole row
 };
 
 // Exclusive prefix of one double per thread over the CTA, in thread order.
@@ -63,14 +65,20 @@ __device__ __forceinline__ int pick_in_chunk(const double (&w)[PER], int v0, Pic
 // cumulative weight exceeds the target (else the last chunk with positive weight) and the cumulative
 // weight before it.  Each thread owns a contiguous run of chunks; a block-wide scan joins the runs.
 // Every thread must call it; on return sh->{jstar, base, target, W} are set and visible to all.
-__device__ __forceinline__ void find_chunk(const double* cw, int n, double u, PickShared* sh, int tid) {
+// With fixed_target >= 0 (sharded vocabulary) the target and the total are given instead: the search then runs
+// for that absolute target over this shard's chunks, and sh->W is set to W_given.
+__device__ __forceinline__ void find_chunk(const double* cw, int n, double u, PickShared* sh, int tid,
+                                           double fixed_target = -1.0, double W_given = 0.0) {
   const int per = (n + kRecThreads - 1) / kRecThreads;
   const int j0 = min(tid * per, n), j1 = min(j0 + per, n);
   double local = 0.0;
   for (int j = j0; j < j1; ++j) local += cw[j];
   if (tid == 0) { sh->jstar = 0x7fffffff; sh->jlast = -1; }
   const double excl = block_excl_scan(local, sh->warp_tot, tid);  // two barriers inside
-  if (tid == kRecThreads - 1) { sh->W = excl + local; sh->target = u * (excl + local); }
+  if (tid == kRecThreads - 1) {
+    sh->W = fixed_target >= 0.0 ? W_given : excl + local;
+    sh->target = fixed_target >= 0.0 ? fixed_target : u * (excl + local);
+  }
   __syncthreads();
   const double target = sh->target;
   double c = excl;
@@ -141,8 +149,42 @@ __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundP
     cw[j] = (m == kNegInf) ? 0.0 : (double)s * exp2((double)m - lseR);
   }
   if (tid == 0) { sh.tok_min = 0x7fffffff; sh.tok_max_pos = -1; }
+  if (p.n_shards > 0 && tid == 0) {
+    // every rank holds every shard's partial of this row, so all of them place the target identically, without
+    // talking: shard weights in shard order, the target u*W, the first shard whose cumulative weight exceeds it
+    double Wg[32], W = 0.0;
+    for (int g = 0; g < p.n_shards; ++g) {
+      const ShardPartial& sp = p.shard_parts[((long long)g * p.B + b) * K1 + st.n];
+      Wg[g] = (sp.m[Q_R] == kNegInf) ? 0.0 : sp.s[Q_R] * exp2((double)sp.m[Q_R] - lseR);
+      W += Wg[g];
+    }
+    const double target = (double)p.u_recover[b] * W;
+    double c = 0.0, base = 0.0, base_last = 0.0;
+    int owner = -1, last = -1;
+    for (int g = 0; g < p.n_shards; ++g) {
+      if (Wg[g] > 0.0) { last = g; base_last = c; }
+      if (c + Wg[g] > target) { owner = g; base = c; break; }
+      c += Wg[g];
+    }
+    if (owner < 0) { owner = last; base = base_last; }
+    sh.plan_owner = (W > 0.0 && W == W) ? owner : -1;
+    sh.plan_target = target - base;
+    sh.plan_W = W;
+  }
   __syncthreads();
-  find_chunk(cw, p.n_chunks, (double)p.u_recover[b], &sh, tid);
+  if (p.n_shards > 0) {
+    if (sh.plan_owner != p.shard_rank) {   // another shard (or nobody) samples: leave values a MAX-reduce ignores
+      if (tid == 0) {
+        if (p.rec_token) p.rec_token[b] = -1;
+        if (p.rec_logprob) p.rec_logprob[b] = sh.plan_owner < 0 ? __int_as_float(0x7fc00000) : kNegInf;
+        if (p.n_out) p.n_out[b] = st.n;
+      }
+      return;
+    }
+    find_chunk(cw, p.n_chunks, 0.0, &sh, tid, fmax(sh.plan_target, 0.0), sh.plan_W);
+  } else {
+    find_chunk(cw, p.n_chunks, (double)p.u_recover[b], &sh, tid);
+  }
 
   const T* hl = reinterpret_cast<const T*>(p.h_llm);
   const T* hp = reinterpret_cast<const T*>(p.h_plus);
@@ -165,9 +207,9 @@ __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundP
   }
   const int tok = pick_in_chunk(w, v0, &sh, tid);
   if (tok >= v0 && tok < v0 + kPerThread) {
-    if (p.rec_token) p.rec_token[b] = tok;
+    if (p.rec_token) p.rec_token[b] = tok + p.vocab_offset;
     if (p.rec_logprob) p.rec_logprob[b] = (float)(y2[tok - v0] * 0.6931471805599453 - log(sh.W));
-    if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
+    if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok + p.vocab_offset;
     if (p.n_out) p.n_out[b] = st.n + 1;
   }
   if (tok < 0 && tid == 0) {  // no positive weight anywhere in the chunk: nothing can be sampled

@@ -379,28 +379,15 @@ __device__ __forceinline__ double exp_nonpos(double x) {
   return __hiloint2double(__double2hiint(q) + ((int)k << 20), __double2loint(q));
 }
 
-// One warp: combine the partial records of `row` (exact power-of-two rescale, sums in double) and, for a
-// drafted row, the log-probabilities, alpha and the accept decision.
-template <typename T>
-__device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float beta, float lam, float c, int lane,
-                             RowResult* out) {
-  const int K = p.K, K1 = K + 1;
-  const long long row = (long long)b * K1 + t;
-  const float* rec = p.part + row * p.n_chunks * 8;
-  // the drafted token's three logits: issued first so that their latency overlaps the record passes
-  int y = -1;
-  float gl = 0.f, gp = 0.f, gm = 0.f;
-  if (t < len) {
-    y = p.draft_tokens[(long long)b * K + t];
-    if (y >= 0 && y < p.V) {
-      const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
-      gl = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
-      gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
-      gm = load_logit<T>(reinterpret_cast<const T*>(p.h_minus), off);
-    }
-  }
-  pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
-  // pass 1: the largest exponent per normaliser; pass 2 (the same lines, now in L1): sums relative to it
+// 2^d in double for an integer-valued d <= 0; 0 below 2^-1000.
+__device__ __forceinline__ double pow2_nonpos_int_d(float d) {
+  return (d < -1000.f) ? 0.0 : __hiloint2double(((int)d + 1023) << 20, 0);
+}
+
+// One warp: the largest exponent per normaliser over the row's records and the float64 sums relative to it
+// (pass 2 finds the lines of pass 1 in L1); every lane gets the results.
+__device__ __forceinline__ void row_sums_from_records(const RoundParams& p, const float* rec, int lane, float (&M)[4],
+                                                      double (&S)[4]) {
   float Ml[4] = {kNegInf, kNegInf, kNegInf, kNegInf};
 #pragma unroll 4
   for (int ch = lane; ch < p.n_chunks; ch += 32) {
@@ -409,10 +396,8 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
     Ml[0] = fmaxf(Ml[0], x.x); Ml[1] = fmaxf(Ml[1], x.z); Ml[2] = fmaxf(Ml[2], z.x); Ml[3] = fmaxf(Ml[3], z.z);
   }
   const float mine = warp_reduce4<true>(Ml, lane);
-  float M[4];
 #pragma unroll
-  for (int q = 0; q < 4; ++q) M[q] = __shfl_sync(kFullMask, mine, 8 * q);
-  double S[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int q = 0; q < 4; ++q) { M[q] = __shfl_sync(kFullMask, mine, 8 * q); S[q] = 0.0; }
 #pragma unroll 4
   for (int ch = lane; ch < p.n_chunks; ch += 32) {
     const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
@@ -429,6 +414,61 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
   for (int q = 0; q < 4; ++q) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) S[q] += __shfl_xor_sync(kFullMask, S[q], o);
+  }
+}
+
+// One warp: combine the partial records of `row` (exact power-of-two rescale, sums in double) and, for a
+// drafted row, the log-probabilities, alpha and the accept decision.
+template <typename T>
+__device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float beta, float lam, float c, int lane,
+                             RowResult* out) {
+  const int K = p.K, K1 = K + 1;
+  const long long row = (long long)b * K1 + t;
+  const float* rec = p.part + row * p.n_chunks * 8;
+  // the drafted token's three logits: issued first so that their latency overlaps the record passes
+  int y = -1;
+  float gl = 0.f, gp = 0.f, gm = 0.f;
+  if (t < len) {
+    y = p.draft_tokens[(long long)b * K + t];
+    if (p.n_shards == 0 && y >= 0 && y < p.V) {
+      const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
+      gl = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
+      gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
+      gm = load_logit<T>(reinterpret_cast<const T*>(p.h_minus), off);
+    }
+  }
+  pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
+  float M[4];
+  double S[4];
+  if (p.n_shards > 0) {
+    // sharded vocabulary: lane g holds shard g's partial of this row; the token's logits come from its owner
+    const bool have = lane < p.n_shards;
+    ShardPartial sp;
+    if (have) sp = p.shard_parts[((long long)lane * p.B + b) * K1 + t];
+    float Ml[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) Ml[q] = have ? sp.m[q] : kNegInf;
+    const float mine = warp_reduce4<true>(Ml, lane);
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      M[q] = __shfl_sync(kFullMask, mine, 8 * q);
+      double w = 0.0;
+      if (have && sp.m[q] != kNegInf) w = (M[q] == -kNegInf) ? 0.0 : sp.s[q] * pow2_nonpos_int_d(sp.m[q] - M[q]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) w += __shfl_xor_sync(kFullMask, w, o);
+      S[q] = w;
+    }
+    const unsigned owners = __ballot_sync(kFullMask, have && sp.has_token != 0);
+    if (t < len && y >= 0 && y < p.vocab_total && owners) {
+      const int src = __ffs(owners) - 1;
+      gl = __shfl_sync(kFullMask, sp.tok_logit[0], src);
+      gp = __shfl_sync(kFullMask, sp.tok_logit[1], src);
+      gm = __shfl_sync(kFullMask, sp.tok_logit[2], src);
+    } else if (t < len) {
+      y = -1;   // outside the global vocabulary, or no shard delivered it
+    }
+  } else {
+    row_sums_from_records(p, rec, lane, M, S);
   }
   // lanes 0..3 take the logarithm of one sum each, lane 4 that of lambda
   const double arg = lane == 0 ? S[0] : (lane == 1 ? S[1] : (lane == 2 ? S[2] : (lane == 3 ? S[3] : (double)lam)));
@@ -450,7 +490,7 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
         make_float4((float)r.lse[0], (float)r.lse[1], (float)r.lse[2], (float)r.lse[3]);
   if (fin && t < len) {
     const long long i = (long long)b * K + t;
-    if (y >= 0 && y < p.V) {
+    if (y >= 0 && y < (p.n_shards > 0 ? p.vocab_total : p.V)) {
       const double cd = (double)c;
       const double l = (double)gl, pp = (double)gp, m = (double)gm;
       const double rr = l + (double)beta * (pp - m);  // Eq. 8
@@ -771,24 +811,63 @@ static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cud
   return cudaGetLastError();
 }
 
-cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
-                          int* n_launches, cudaEvent_t ev_begin, cudaEvent_t ev_end) {
-  *n_launches = 2;
-  cudaError_t e;
-  if (ev_begin && (e = cudaEventRecord(ev_begin, s)) != cudaSuccess) return e;
+// ---- vocabulary-sharded path: this shard's view of every row ---------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kEpiWarps * 32) shard_rows_kernel(const RoundParams p, ShardPartial* out) {
+  const int b = blockIdx.x, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int K = p.K, K1 = K + 1;
+  int len = p.draft_len[b];
+  if (len < 0 || len > K) len = 0;
+  const int R = len + ((p.flags & SPECSTEER_FLAG_BONUS) ? 1 : 0);
+  pdl_wait();
+  for (int t = warp; t <= K; t += kEpiWarps) {
+    ShardPartial sp;
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { sp.m[q] = kNegInf; sp.s[q] = 0.0; }
+    sp.tok_logit[0] = sp.tok_logit[1] = sp.tok_logit[2] = 0.f;
+    sp.has_token = 0;
+    if (t < R) {
+      const long long row = (long long)b * K1 + t;
+      float M[4];
+      double S[4];
+      row_sums_from_records(p, p.part + row * p.n_chunks * 8, lane, M, S);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) { sp.m[q] = M[q]; sp.s[q] = S[q]; }
+      if (t < len) {
+        const int y = p.draft_tokens[(long long)b * K + t] - p.vocab_offset;   // id within this shard
+        if (y >= 0 && y < p.V) {
+          const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
+          sp.tok_logit[0] = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
+          sp.tok_logit[1] = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
+          sp.tok_logit[2] = load_logit<T>(reinterpret_cast<const T*>(p.h_minus), off);
+          sp.has_token = 1;
+        }
+      }
+    }
+    if (lane == 0) out[(long long)b * K1 + t] = sp;
+  }
+}
+
+cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out, cudaStream_t s) {
+  if (dtype == SPECSTEER_F32) shard_rows_kernel<float><<<p.B, kEpiWarps * 32, 0, s>>>(p, out);
+  else shard_rows_kernel<uint16_t><<<p.B, kEpiWarps * 32, 0, s>>>(p, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s) {
   const bool np = p.need_p != 0;
   if (dtype == SPECSTEER_F32) {
-    e = aligned ? (np ? launch_stream<float, kChunkF32, 16, 16, 4, true, true>(p, li, s)
-                      : launch_stream<float, kChunkF32, 16, 16, 4, true, false>(p, li, s))
-                : launch_stream<float, kChunkF32, 16, 16, 4, false, true>(p, li, s);
-  } else {
-    e = aligned ? (np ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, true>(p, li, s)
-                      : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, false>(p, li, s))
-                : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, true>(p, li, s);
+    return aligned ? (np ? launch_stream<float, kChunkF32, 16, 16, 4, true, true>(p, li, s)
+                         : launch_stream<float, kChunkF32, 16, 16, 4, true, false>(p, li, s))
+                   : launch_stream<float, kChunkF32, 16, 16, 4, false, true>(p, li, s);
   }
-  if (e != cudaSuccess) return e;
-  if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;
-  // programmatic dependent launch: the epilogue reads its inputs while the streaming kernel drains
+  return aligned ? (np ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, true>(p, li, s)
+                       : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, false>(p, li, s))
+                 : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, true>(p, li, s);
+}
+
+cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s) {
+  // programmatic dependent launch: the epilogue reads its inputs while the kernel before it drains
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.B);
   cfg.blockDim = dim3(kEpiWarps * 32);
@@ -801,6 +880,16 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
   cfg.numAttrs = 1;
   if (dtype == SPECSTEER_F32) return cudaLaunchKernelEx(&cfg, epilogue_kernel<float>, p);
   return cudaLaunchKernelEx(&cfg, epilogue_kernel<uint16_t>, p);
+}
+
+cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
+                          int* n_launches, cudaEvent_t ev_begin, cudaEvent_t ev_end) {
+  *n_launches = 2;
+  cudaError_t e;
+  if (ev_begin && (e = cudaEventRecord(ev_begin, s)) != cudaSuccess) return e;
+  if ((e = launch_verify_stream(p, dtype, aligned, li, s)) != cudaSuccess) return e;
+  if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;
+  return launch_epilogue(p, dtype, s);
 }
 
 }  // namespace specsteer

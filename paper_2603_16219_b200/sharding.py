@@ -4,6 +4,10 @@ Requests of a round are independent, so the path shards by request: every rank v
 contiguous block and no collective touches the logits.  These helpers hold the shard arithmetic and the
 two tiny collectives a job needs around the kernels (gathering per-request results, and the
 max-over-ranks of a timing).  They work with any torch.distributed backend (NCCL on GPUs, gloo in tests).
+
+When the logits arrive split along the vocabulary instead (a tensor-parallel LM head), `sharded_vocab_round`
+runs the round with one exchange step: an all-gather of 64 bytes per row and rank, and a MAX all-reduce of the
+per-request results.  The arithmetic stays in the library's kernels; only the two collectives live here.
 """
 from __future__ import annotations
 
@@ -44,3 +48,47 @@ def max_over_ranks(value: float, device, dist) -> float:
     t = torch.tensor([float(value)], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def vocab_range(V: int, rank: int, world: int, align: int = 8) -> Tuple[int, int]:
+    """Contiguous block [lo, hi) of the V token ids owned by `rank`: equal blocks rounded up to `align` ids
+    (16-byte rows for 16-bit logits), the last rank taking what is left."""
+    if world <= 0 or not (0 <= rank < world) or V < 0 or align <= 0:
+        raise ValueError("bad shard arguments")
+    per = -(-V // world)
+    per = -(-per // align) * align
+    lo = min(rank * per, V)
+    return lo, min(lo + per, V)
+
+
+def gather_partials(row_partials: torch.Tensor, dist) -> torch.Tensor:
+    """All-gather the [B, K+1, 64] uint8 partials of every rank into [world, B, K+1, 64], rank-major."""
+    world = dist.get_world_size()
+    out = torch.empty((world,) + tuple(row_partials.shape), dtype=row_partials.dtype, device=row_partials.device)
+    dist.all_gather(list(out.unbind(0)), row_partials.contiguous())
+    return out
+
+
+def reduce_recovered(outputs: Dict[str, torch.Tensor], dist) -> None:
+    """Element-wise MAX over ranks of the four arrays the owning shard fills (in place)."""
+    for name in ("rec_token", "rec_logprob", "out_tokens", "n_out"):
+        t = outputs.get(name)
+        if t is not None:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+
+
+def sharded_vocab_round(ctx, desc, outputs: Dict[str, torch.Tensor], vocab_offset: int, vocab_total: int, dist,
+                        stream=None) -> torch.Tensor:
+    """One verify + recover round over a vocabulary split across the ranks of `dist`.
+
+    `desc` describes this rank's shard (V = local width; draft_tokens hold global ids) and points at `outputs`.
+    Returns the gathered partials.  Every rank ends with identical outputs.
+    """
+    rank = dist.get_rank()
+    parts = torch.empty((desc.B, desc.K + 1, 64), dtype=torch.uint8, device=outputs["accept_len"].device)
+    ctx.shard_verify_local(desc, vocab_offset, parts, stream)
+    gathered = gather_partials(parts, dist)
+    ctx.shard_verify_combine(desc, gathered, rank, vocab_offset, vocab_total, stream)
+    ctx.shard_recover_local(desc, gathered, rank, vocab_offset, vocab_total, stream)
+    reduce_recovered(outputs, dist)
+    return gathered

@@ -64,3 +64,54 @@ def test_request_range_covers_every_request_once():
             assert got == list(range(B))
     with pytest.raises(ValueError):
         sharding.request_range(4, 2, 2)
+
+
+def _vocab_worker(rank, world, port, q):
+    import torch.distributed as dist
+    from paper_2603_16219_b200 import sharding
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    try:
+        B, K1 = 3, 4
+        parts = torch.full((B, K1, 64), rank + 1, dtype=torch.uint8)
+        parts[:, :, 0] = torch.arange(B * K1, dtype=torch.uint8).reshape(B, K1)
+        gathered = sharding.gather_partials(parts, dist)
+        ok = tuple(gathered.shape) == (world, B, K1, 64)
+        for r in range(world):                                  # rank-major, every rank sees the same thing
+            ok = ok and bool((gathered[r, :, :, 1:] == r + 1).all()) and bool((gathered[r, :, :, 0] == parts[:, :, 0]).all())
+        # the owner of each request's target fills the results, the others leave -1 / -inf / the accepted length
+        outs = {"rec_token": torch.tensor([7 if rank == 0 else -1, 9 if rank == 1 else -1, -1], dtype=torch.int32),
+                "rec_logprob": torch.tensor([-0.5 if rank == 0 else float("-inf"), -2.0 if rank == 1 else float("-inf"),
+                                             float("-inf")]),
+                "out_tokens": torch.tensor([[3, 7 if rank == 0 else -1], [9 if rank == 1 else -1, -1], [-1, -1]], dtype=torch.int32),
+                "n_out": torch.tensor([2 if rank == 0 else 1, 1 if rank == 1 else 0, 0], dtype=torch.int32)}
+        sharding.reduce_recovered(outs, dist)
+        ok = ok and outs["rec_token"].tolist() == [7, 9, -1] and outs["n_out"].tolist() == [2, 1, 0]
+        ok = ok and outs["out_tokens"].tolist() == [[3, 7], [9, -1], [-1, -1]]
+        ok = ok and outs["rec_logprob"][:2].tolist() == [-0.5, -2.0]
+        q.put((rank, ok))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_vocab_shard_collectives_on_two_ranks():
+    """The two collectives of the vocabulary-sharded round (all-gather of row partials, MAX all-reduce of results)."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_vocab_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+    assert res == [(0, True), (1, True)]
+
+
+def test_vocab_range_covers_every_id_once():
+    from paper_2603_16219_b200 import sharding
+    for V, world, align in ((151936, 8, 8), (4096, 7, 1024), (10, 4, 8), (128256, 3, 8), (5, 2, 1)):
+        spans = [sharding.vocab_range(V, r, world, align) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][1] == V
+        assert all(spans[i][1] == spans[i + 1][0] for i in range(world - 1))
+        assert all(lo % align == 0 for lo, hi in spans if hi > lo)
