@@ -855,12 +855,13 @@ cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out
 }
 
 cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s) {
-  // producer warps: two for float32, four for 16-bit logits (measured: 6.43 against 6.15 TB/s on the float32
-  // serving shape with two, 5.87 against 5.64 TB/s on the largest bf16 shape with four)
+  // Ring shape per logit type, from sweeps on the two largest benchmark shapes: float32 is bound by memory and
+  // runs best with 144 KB in flight (12 stages, 6 consumer pairs, 3 producers: 0.350 ms against 0.379 ms for
+  // 16/16/4 on 2.33 GB); 16-bit logits need the arithmetic of 8 pairs and 4 producers (12/12/3 is 12 % slower).
   const bool np = p.need_p != 0;
   if (dtype == SPECSTEER_F32) {
-    return aligned ? (np ? launch_stream<float, kChunkF32, 16, 16, 2, true, true>(p, li, s)
-                         : launch_stream<float, kChunkF32, 16, 16, 2, true, false>(p, li, s))
+    return aligned ? (np ? launch_stream<float, kChunkF32, 12, 12, 3, true, true>(p, li, s)
+                         : launch_stream<float, kChunkF32, 12, 12, 3, true, false>(p, li, s))
                    : launch_stream<float, kChunkF32, 16, 16, 4, false, true>(p, li, s);
   }
   return aligned ? (np ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, true>(p, li, s)
