@@ -190,6 +190,18 @@ def test_outliers_after_the_first_batch_of_a_chunk(env, dtype):
         P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, 1, P.TOL[L.dtype])
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_extreme_temperatures(env, dtype):
+    """Very low temperatures stretch a row over thousands of binades (nearly every chunk overflows its first
+    attempt and is redone with per-batch tests); very high ones flatten it.  Logits of ordinary size."""
+    spec, inputs = _small(env["synth"], 6, 3, 7000, dtype, seed=23, beta_choices=(0.5, 1.0, 2.0))
+    inputs["temperature"] = torch.tensor([0.02, 0.05, 0.1, 5.0, 50.0, 1.0], dtype=torch.float32, device="cuda")
+    tol = P.TOL[inputs["h_llm"].dtype]
+    for am, rm in ((0, 0), (1, 1)):
+        gpu = P.run_gpu(env["ctx"], inputs, am, rm, 1)
+        P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, 1, tol)
+
+
 def test_many_requests_cross_the_slab_limit(env):
     spec, inputs = _small(env["synth"], 5000, 2, 64, "bf16", seed=6, ragged=True)
     gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
