@@ -1,19 +1,25 @@
 // Verification: one streaming pass over the three logit tensors, then a small per-request epilogue.
 //
-// Streaming kernel.  Work unit: a tile = one chunk of TILE vocabulary entries of one used row, all
-// three streams.  A persistent CTA per SM owns a ring of shared-memory stages.  One producer thread
-// fills stages with 1-D bulk (TMA) copies signalled on mbarriers; each consumer warp owns whole tiles
-// (two stages per warp, so that one loads while the other is reduced), keeps four running
-// (reference exponent, scaled sum) pairs per lane, and writes one 32-byte partial record per tile.
-// Epilogue kernel.  One CTA per request: each warp combines the records of one row in chunk order and
-// forms the log-probabilities and alpha; the accept flags are then scanned for accept_len
-// (Algorithm 1 Phase 2; Eq. 6 / Eq. 7).
+// Streaming kernel.  Work unit: a tile = two chunks of vocabulary entries of one used row, all three
+// streams (12 KB).  A persistent CTA per SM owns a ring of shared-memory stages.  A few producer threads
+// fill stages with 1-D bulk (TMA) copies signalled on mbarriers; the consumer warps work in pairs, each
+// pair owns two stages (one loads while the other is reduced) and each warp of the pair reduces one chunk:
+// four (reference exponent, sum) pairs, the references uniform over the warp, and writes one 32-byte partial
+// record per chunk.  A full chunk is first tried without any test inside it; an overflow sends it through
+// the variant that tests every batch.
+// Epilogue kernel.  One CTA per request: each warp combines the records of one row and forms the
+// log-probabilities and alpha; the accept flags are then scanned for accept_len
+// (Algorithm 1 Phase 2; Eq. 6 / Eq. 7).  With a sharded vocabulary the rows come from the shards' gathered
+// partials instead of the records.
 #include "common.cuh"
 #include "internal.h"
 #include "specsteer.h"
 
 namespace specsteer {
 
+// How many of the four pairs per batch of the h_SLM- stream take the FMA-pipe polynomial instead of ex2.approx
+// for 16-bit logits (all outputs / without the h_SLM+ normaliser).  0: measured no faster at any setting,
+// because the polynomial costs as many issue slots as it frees on the special-function unit.
 #ifndef SPECSTEER_POLY_PAIRS_BF16
 #define SPECSTEER_POLY_PAIRS_BF16 0
 #endif
@@ -22,7 +28,7 @@ constexpr int kPolyPairsBF16 = SPECSTEER_POLY_PAIRS_BF16;
 #define SPECSTEER_POLY_PAIRS_BF16_LEAN 0
 #endif
 constexpr int kPolyPairsBF16Lean = SPECSTEER_POLY_PAIRS_BF16_LEAN;
-constexpr float kSlack = 16.f;  // a lane's reference exponent may lag its running maximum by this much
+constexpr float kSlack = 16.f;  // careful path: the reference exponent may lag the running maximum by this much
 
 struct TileMeta {
   int row, tile, n_valid;  // padded row index b*(K+1)+t, tile within the row, valid entries in the tile
