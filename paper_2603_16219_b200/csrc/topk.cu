@@ -338,22 +338,14 @@ __global__ void __launch_bounds__(32) edge_resample_kernel(const RoundParams p, 
 cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_idx, float* topk_val,
                               void* lists_ws, int* count_ws, int sm_count, cudaStream_t s) {
   // Two CTAs fit on an SM.  Few requests: split each row over as many CTAs as still fit at once (one wave), but
-  // keep at least 4096 vectors (64 KB per stream) per slice.  Many requests: split so that the last wave is full.
+  // keep at least 4096 vectors (64 KB per stream) per slice.  Otherwise one CTA per row: splitting further only
+  // multiplies the fixed work per CTA (measured on 512 rows of 256000 bf16 entries: 98 us unsplit, 135 us split in 4).
   const int nvec = p.V / (dtype == SPECSTEER_F32 ? 4 : 8);
   const int slots = 2 * sm_count;
   int s_cap = nvec / 4096 > 1 ? nvec / 4096 : 1;
   if (s_cap > kTopkMaxSplit) s_cap = kTopkMaxSplit;
   int S = 1;
-  if (p.B * 2 <= slots) {
-    S = slots / p.B;
-  } else if (p.B > slots) {
-    double best = 1e30;
-    for (int c = 1; c <= 4; ++c) {
-      const int items = p.B * c, waves = (items + slots - 1) / slots;
-      const double cost = (double)waves * slots / items + 0.03 * (c - 1);   // idle share of the last wave + split overhead
-      if (cost < best) { best = cost; S = c; }
-    }
-  }
+  if (p.B * 2 <= slots) S = slots / p.B;
   if (S > s_cap) S = s_cap;
   if (S < 1 || !lists_ws || !count_ws) S = 1;
   const dim3 grid(p.B, S);
