@@ -312,7 +312,38 @@ def test_error_codes_on_device(env):
         fresh.verify_round(desc)
     assert e.value.code == b.ERR_INVALID_ARG
     assert fresh.launch_count == 0 and fresh.workspace_bytes > 0
+    # the timing hook wants both events or none
+    ev = torch.cuda.Event(enable_timing=True)
+    ev.record()
+    with pytest.raises(b.SpecSteerError) as e:
+        fresh.time_streaming(ev, None)
+    assert e.value.code == b.ERR_INVALID_ARG
     small_ctx.close(); fresh.close()
+
+
+def test_streaming_kernel_timing_hook(env):
+    """The event pair the library records around the streaming kernel gives a positive time below the whole call's,
+    and switching the hook off leaves the events untouched."""
+    spec, inputs = _small(env["synth"], 8, 3, 50000, "f32", seed=12)
+    b = env["binding"]
+    outs = b.alloc_outputs(8, 3, "cuda")
+    desc = b.make_desc(inputs, outs, flags=1)
+    e0, e1, a, z = (torch.cuda.Event(enable_timing=True) for _ in range(4))
+    for ev in (e0, e1):
+        ev.record()
+    torch.cuda.synchronize()
+    env["ctx"].time_streaming(e0, e1)
+    a.record()
+    env["ctx"].verify_round(desc)
+    env["ctx"].recover_sample(desc)
+    z.record()
+    env["ctx"].time_streaming(None, None)
+    torch.cuda.synchronize()
+    inner, outer = e0.elapsed_time(e1), a.elapsed_time(z)
+    assert 0 < inner < outer
+    env["ctx"].verify_round(desc)          # hook off: e0/e1 keep their times
+    torch.cuda.synchronize()
+    assert e0.elapsed_time(e1) == inner
 
 
 def test_host_round_matches_device_round(env):
