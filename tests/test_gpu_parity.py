@@ -202,6 +202,21 @@ def test_extreme_temperatures(env, dtype):
         P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, 1, tol)
 
 
+@pytest.mark.parametrize("K", [20, 70])
+def test_long_drafts(env, K):
+    """More draft positions than the usual handful; beyond 64 rows a request's epilogue runs in several passes."""
+    b = env["binding"]
+    spec = env["synth"].RoundSpec("long_drafts", 3, K, 900, "f32", ragged=True)
+    inputs = env["synth"].make_round(spec, device="cuda", seed=K)
+    inputs["draft_len"] = torch.tensor([K, K // 2, 1], dtype=torch.int32, device="cuda")
+    inputs["lam"][:] = 0.05                                  # accept almost everything so that late rows matter
+    ctx = b.Context(max_B=3, max_K=K, max_V=900)
+    for am, rm, fl in ((0, 0, 1), (1, 1, 0)):
+        gpu = P.run_gpu(ctx, inputs, am, rm, fl)
+        P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), am, rm, fl, 1e-4)
+    ctx.close()
+
+
 def test_many_requests_cross_the_slab_limit(env):
     spec, inputs = _small(env["synth"], 5000, 2, 64, "bf16", seed=6, ragged=True)
     gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
