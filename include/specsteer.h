@@ -95,7 +95,8 @@ typedef struct {
    * Algorithm 1 itself needs three normalisers per row (h_LLM and h_SLM- for Eq. 7, h_rec for Eq. 8).  The
    * fourth, of h_SLM+, is formed only when something asks for it: a non-NULL logp_plus or log_z, EXACT_Z
    * acceptance or RESIDUAL recovery.  Leaving logp_plus and log_z NULL in RATIO + STEER mode therefore saves a
-   * quarter of the exponentials (it matters for 16-bit logits, where they bind before the memory does). */
+   * quarter of the exponentials (it matters for 16-bit logits, where they bind before the memory does).  The other
+   * outputs then keep their decisions and tokens; their floating-point values may differ in the last bits. */
   int32_t *accept_len;   /* [B]      drafts accepted before the first rejection */
   uint8_t *accept_flags; /* [B][K]   1 where u <= alpha (every drafted position, also after the first rejection) */
   float *alpha;          /* [B][K]   acceptance probability; 0 beyond draft_len */
