@@ -29,6 +29,7 @@ struct specsteer_ctx {
   uint64_t launches;
   bool poisoned;
   bool shard_streamed;   // specsteer_shard_verify_local ran for the shape in v_*
+  bool v_two_phase;      // the last verify_round left the recovery rows unread (see two_phase())
   // host-round staging
   void* stage;
   size_t stage_bytes;
@@ -94,8 +95,9 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
   p.B = nb; p.K = K; p.V = d->V;
   p.ld_row = d->ld_row; p.ld_req = d->ld_req;
   p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
-  p.need_p = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
-              d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? 1 : 0;
+  p.sums = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
+            d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? SUM_ALL : (SUM_L | SUM_M | SUM_R);
+  p.row_mode = ROWS_ALL;
   p.tile = tile_of(d->dtype);
   p.n_chunks = n_chunks_of(d->V, p.tile);
   auto lg = [&](const void* base) { return (const void*)((const char*)base + (size_t)b0 * d->ld_req * es); };
@@ -125,11 +127,21 @@ bool rows_aligned(const specsteer_round_desc* d) {
          ((size_t)d->ld_req * es) % 16 == 0;
 }
 
+// Verification needs the normalisers of h_LLM and h_SLM- only (Eq. 7); when nobody asks for a quantity of the
+// fused target on the drafted rows, the h_SLM+ tensor is left unread there and the recovery call forms the
+// normalisers of its one row itself (Eq. 8 on the row of the first rejection).
+bool two_phase(const specsteer_round_desc* d) {
+  return d->accept_mode == SPECSTEER_ACCEPT_RATIO && d->recover_mode == SPECSTEER_RECOVER_STEER && !d->logp_plus &&
+         !d->logp_star && !d->log_z && rows_aligned(d);
+}
+
 specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
   const bool aligned = rows_aligned(d);
+  const bool lean = two_phase(d);
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
     RoundParams p = slab_params(ctx, d, b0, nb);
+    if (lean) { p.sums = SUM_L | SUM_M; p.row_mode = ROWS_DRAFTED; }
     int nl = 0;
     const bool first = b0 == 0, last = b0 + nb >= d->B;
     if (launch_verify(p, d->dtype, aligned, ctx->li, s, &nl, first ? ctx->ev_stream_begin : nullptr,
@@ -141,10 +153,18 @@ specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cu
 }
 
 specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
+  const bool lean = ctx->v_two_phase;   // what the verification of this round did, not what this descriptor says
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
     RoundParams p = slab_params(ctx, d, b0, nb);
     int nl = 0;
+    if (lean) {   // the recovery rows have no records yet: one more streaming pass over them alone
+      p.sums = SUM_ALL;
+      p.row_mode = ROWS_RECOVERY;
+      if (launch_verify_stream(p, d->dtype, true, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+      if (launch_recovery_row_lse(p, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+      ctx->launches += 2;
+    }
     if (launch_recover(p, d->dtype, ctx->li, s, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
     ctx->launches += nl;
   }
@@ -226,6 +246,7 @@ specsteer_status specsteer_verify_round(specsteer_ctx* ctx, const specsteer_roun
   if (!g.ok) return SPECSTEER_ERR_CUDA;
   st = do_verify(ctx, d, (cudaStream_t)cuda_stream);
   if (st != SPECSTEER_OK) return st;
+  ctx->v_two_phase = two_phase(d);
   ctx->verified = true;
   ctx->v_B = d->B; ctx->v_K = d->K; ctx->v_V = d->V; ctx->v_dtype = d->dtype; ctx->v_h_llm = d->h_llm;
   return SPECSTEER_OK;
@@ -273,7 +294,7 @@ specsteer_status specsteer_shard_verify_local(specsteer_ctx* ctx, const specstee
     DeviceGuard g(ctx->device);
     if (!g.ok) return SPECSTEER_ERR_CUDA;
     RoundParams p = slab_params(ctx, d, 0, d->B);
-    p.need_p = 1;
+    p.sums = SUM_ALL;
     p.vocab_offset = vocab_offset;
     cudaStream_t s = (cudaStream_t)cuda_stream;
     if (launch_verify_stream(p, d->dtype, rows_aligned(d), ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
@@ -297,13 +318,14 @@ specsteer_status specsteer_shard_verify_combine(specsteer_ctx* ctx, const specst
     DeviceGuard g(ctx->device);
     if (!g.ok) return SPECSTEER_ERR_CUDA;
     RoundParams p = slab_params(ctx, d, 0, d->B);
-    p.need_p = 1;
+    p.sums = SUM_ALL;
     p.shard_parts = (const ShardPartial*)gathered;
     p.n_shards = n_shards; p.shard_rank = shard_rank;
     p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;
     if (launch_epilogue(p, d->dtype, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
     ctx->launches += 1;
   }
+  ctx->v_two_phase = false;
   ctx->verified = true;
   return SPECSTEER_OK;
 }
@@ -321,7 +343,7 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx* ctx, const specste
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
   RoundParams p = slab_params(ctx, d, 0, d->B);
-  p.need_p = 1;
+  p.sums = SUM_ALL;
   p.shard_parts = (const ShardPartial*)gathered;
   p.n_shards = n_shards; p.shard_rank = shard_rank;
   p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;

@@ -23,12 +23,21 @@ struct ShardPartial {
 };
 static_assert(sizeof(ShardPartial) == 64, "the sharded path exchanges 64 bytes per row and shard");
 
+enum { SUM_L = 1, SUM_P = 2, SUM_M = 4, SUM_R = 8, SUM_ALL = 15 };  // bit q = normaliser Q_q
+enum {
+  ROWS_ALL = 0,       // rows 0 .. draft_len (the last one only with FLAG_BONUS)
+  ROWS_DRAFTED = 1,   // rows 0 .. draft_len - 1: verification alone
+  ROWS_RECOVERY = 2   // row accept_len of the requests that sample (after the epilogue has run)
+};
+
 struct RoundParams {
   int B, K, V;
   long long ld_row, ld_req;  // elements
   int accept_mode, recover_mode;
   unsigned flags;
-  int need_p;    // the normaliser of h_SLM+ is wanted (logp_plus, log_z, EXACT_Z or RESIDUAL); Algorithm 1 itself is not
+  int sums;      // SUM_* bits: which of the four normalisers the streaming pass forms (Algorithm 1 needs L, M and,
+                 // on the recovery row, R; the one of h_SLM+ only serves logp_plus, log_z, EXACT_Z and RESIDUAL)
+  int row_mode;  // ROWS_*: which rows of a request the streaming pass reads
   int tile;      // vocabulary entries per chunk (kChunkF32 or kChunkBF16)
   int n_chunks;  // ceil(V / tile)
   const void *h_llm, *h_plus, *h_minus;
@@ -71,6 +80,8 @@ cudaError_t launch_edge_resample(const RoundParams& p, int dtype, int k, const i
                                  cudaStream_t s);
 // the streaming kernel alone (partial records into the workspace), no epilogue
 cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s);
+// log-normalisers of row accept_len of every sampling request from its records (after a ROWS_RECOVERY pass)
+cudaError_t launch_recovery_row_lse(const RoundParams& p, cudaStream_t s);
 // per-row ShardPartial of this shard from its partial records: out[B][K+1]
 cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out, cudaStream_t s);
 // the per-request epilogue alone (reads p.shard_parts when p.n_shards > 0)

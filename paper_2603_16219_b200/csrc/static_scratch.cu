@@ -89,8 +89,9 @@ extern "C" specsteer_status specsteer_verify_round_static(const specsteer_round_
   p.B = d->B; p.K = d->K; p.V = d->V;
   p.ld_row = d->ld_row; p.ld_req = d->ld_req;
   p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
-  p.need_p = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
-              d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? 1 : 0;
+  p.sums = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
+            d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? SUM_ALL : (SUM_L | SUM_M | SUM_R);
+  p.row_mode = ROWS_ALL;
   p.tile = tile; p.n_chunks = n_chunks;
   p.h_llm = d->h_llm; p.h_plus = d->h_slm_plus; p.h_minus = d->h_slm_minus;
   p.draft_tokens = d->draft_tokens; p.draft_len = d->draft_len;

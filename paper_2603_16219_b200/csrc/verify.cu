@@ -183,7 +183,7 @@ __device__ __forceinline__ void exp_sum8(f32x2& s2, const f32x2 (&x)[4], f32x2 c
 }
 
 // Eight vocabulary entries per lane of the three streams: r = l + beta (p - m)  (Eq. 8), then the four sums.
-template <bool MASKED, bool FIRST>
+template <bool MASKED, bool FIRST, int SUMS>
 __device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32x2 (&m)[4], f32x2 beta2, f32x2 c2,
                                        float c, float inv_c, unsigned vmask, int lane) {
   f32x2 r[4];
@@ -202,17 +202,19 @@ __device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32
       }
     }
   }
-  const float bm[4] = {max8(l), max8(p), max8(m), max8(r)};  // order of Q_L, Q_P, Q_M, Q_R
+  // order of Q_L, Q_P, Q_M, Q_R; a normaliser that is not wanted never leaves -inf
+  const float bm[4] = {(SUMS & SUM_L) ? max8(l) : kNegInf, (SUMS & SUM_P) ? max8(p) : kNegInf,
+                       (SUMS & SUM_M) ? max8(m) : kNegInf, (SUMS & SUM_R) ? max8(r) : kNegInf};
   if (FIRST) {
     acc_start(a, bm, c, inv_c, lane);
   } else {
     const bool upd = (bm[0] > a.thr[0]) | (bm[1] > a.thr[1]) | (bm[2] > a.thr[2]) | (bm[3] > a.thr[3]);
     if (__any_sync(kFullMask, upd)) acc_raise(a, bm, c, inv_c, lane);
   }
-  exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-  exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-  exp_sum8<0>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-  exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+  if (SUMS & SUM_L) exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+  if (SUMS & SUM_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+  if (SUMS & SUM_M) exp_sum8<0>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+  if (SUMS & SUM_R) exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
 }
 
 // ---- one chunk (half a tile) from shared memory, one warp ---------------------------------------
@@ -253,7 +255,7 @@ template <> struct Batch<uint16_t> {
   }
 };
 
-template <typename T, int CHUNK, bool MASKED>
+template <typename T, int CHUNK, bool MASKED, int SUMS>
 __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, const T* sm, int lane, int n_valid,
                                            float beta, float c, float inv_c) {
   const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
@@ -262,11 +264,12 @@ __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, con
     if (MASKED && it > 0 && it * 256 >= n_valid) break;  // warp-uniform: nothing left for any lane
     f32x2 l[4], p[4], m[4];
     Batch<T>::load(sl, it, lane, l);
-    Batch<T>::load(sp, it, lane, p);
+    if (SUMS & (SUM_P | SUM_R)) Batch<T>::load(sp, it, lane, p);   // otherwise the h_SLM+ slot was never filled
+    else p[0] = p[1] = p[2] = p[3] = 0ull;
     Batch<T>::load(sm, it, lane, m);
     const unsigned vmask = MASKED ? Batch<T>::mask(it, lane, n_valid) : 0xffu;
-    if (it == 0) accum8<MASKED, true>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
-    else accum8<MASKED, false>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
+    if (it == 0) accum8<MASKED, true, SUMS>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
+    else accum8<MASKED, false, SUMS>(a, l, p, m, beta2, c2, c, inv_c, vmask, lane);
   }
 }
 
@@ -278,39 +281,45 @@ __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, con
 // chunk_pass, which tests every batch.
 constexpr float kBias = 60.f;
 
-template <typename T, int CHUNK, int POLY_N, bool NEED_P>
+template <typename T, int CHUNK, int POLY_N, int SUMS>
 __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, const T* sm, int lane, float beta,
                                            float c, float inv_c) {
   const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
   float run_m = kNegInf;  // running maximum of the stream that takes the polynomial
+  constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;   // the h_SLM+ slot is filled and read
   {
     f32x2 l[4], p[4], m[4], r[4];
     Batch<T>::load(sl, 0, lane, l);
-    Batch<T>::load(sp, 0, lane, p);
+    if (kPlus) Batch<T>::load(sp, 0, lane, p);
     Batch<T>::load(sm, 0, lane, m);
+    if (SUMS & SUM_R) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
-    const float bm[4] = {max8(l), NEED_P ? max8(p) : kNegInf, max8(m), max8(r)};
+      for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
+    }
+    const float bm[4] = {(SUMS & SUM_L) ? max8(l) : kNegInf, (SUMS & SUM_P) ? max8(p) : kNegInf,
+                         (SUMS & SUM_M) ? max8(m) : kNegInf, (SUMS & SUM_R) ? max8(r) : kNegInf};
     acc_start(a, bm, c, inv_c, lane, kBias);
     run_m = bm[Q_M];
-    exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    if (NEED_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-    exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-    exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+    if (SUMS & SUM_L) exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+    if (SUMS & SUM_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (SUMS & SUM_M) exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+    if (SUMS & SUM_R) exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
 #pragma unroll 1
   for (int it = 1; it < CHUNK / 256; ++it) {
     f32x2 l[4], p[4], m[4], r[4];
     Batch<T>::load(sl, it, lane, l);
-    Batch<T>::load(sp, it, lane, p);
+    if (kPlus) Batch<T>::load(sp, it, lane, p);
     Batch<T>::load(sm, it, lane, m);
+    if (SUMS & SUM_R) {
 #pragma unroll
-    for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
-    if (POLY_N > 0) run_m = fmaxf(run_m, max8(m));
-    exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    if (NEED_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-    exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-    exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+      for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
+    }
+    if (POLY_N > 0 && (SUMS & SUM_M)) run_m = fmaxf(run_m, max8(m));
+    if (SUMS & SUM_L) exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+    if (SUMS & SUM_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (SUMS & SUM_M) exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+    if (SUMS & SUM_R) exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
   const float kBig = 1.329227995784916e36f;  // 2^120
   bool bad = false;
@@ -320,7 +329,7 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     unpack2(a.s2[q], s0, s1);
     bad |= !(s0 + s1 < kBig);
   }
-  if (POLY_N > 0) {
+  if (POLY_N > 0 && (SUMS & SUM_M)) {
     float n0, n1;
     unpack2(a.nref2[Q_M], n0, n1);
     bad |= !(fmaf(run_m, c, n0) < 120.f);
@@ -484,7 +493,7 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
     r.lse[q] = (double)M[q] + __shfl_sync(kFullMask, lg, q);
-    if (q != Q_P || p.need_p) fin = fin && isfinite(r.lse[q]);
+    if (p.sums & (1 << q)) fin = fin && isfinite(r.lse[q]);
   }
   const double ln2 = 0.6931471805599453;
   const double log_lam = __shfl_sync(kFullMask, lg, 4) * ln2;
@@ -529,7 +538,7 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
   const bool params_ok = isfinite(Tmp) && Tmp > 0.f && isfinite(lam) && lam > 0.f && isfinite(beta);
   if (len < 0 || len > K) { status |= SPECSTEER_REQ_BAD_LEN; len = 0; }
   const bool bonus = (p.flags & SPECSTEER_FLAG_BONUS) != 0;
-  const int R = params_ok ? len + (bonus ? 1 : 0) : 0;
+  const int R = params_ok ? len + ((bonus && p.row_mode != ROWS_DRAFTED) ? 1 : 0) : 0;  // rows with records
   const float c = kLog2e / Tmp;
   const float qnan = __int_as_float(0x7fc00000);
 
@@ -599,12 +608,13 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 // producer thread that owns the stages congruent to its index modulo NPW (one thread cannot issue tiles
 // fast enough for a whole SM).  Every stage is always consumed by the same pair of warps, so a waiting
 // warp is never a whole barrier phase ahead of the data.
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, bool NEED_P>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
   constexpr int TILE = 2 * CHUNK;
   // 16-bit logits carry half the bytes per power of two, so there the special-function unit binds before
   // HBM does: the h_SLM- stream takes the FMA-pipe polynomial for POLY_N of its four pairs per batch
-  constexpr int POLY_N = sizeof(T) == 2 ? (NEED_P ? kPolyPairsBF16 : kPolyPairsBF16Lean) : 0;
+  constexpr int POLY_N = sizeof(T) == 2 ? ((SUMS & SUM_P) ? kPolyPairsBF16 : kPolyPairsBF16Lean) : 0;
+  constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;  // h_SLM+ is read at all
   constexpr int NPAIR = NCW / 2;
   static_assert(NCW % 2 == 0 && STAGES % NPAIR == 0, "each stage belongs to one fixed pair of consumer warps");
   static_assert(STAGES % NPW == 0, "each producer owns a fixed subset of the stages");
@@ -619,6 +629,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   float* beta_s = reinterpret_cast<float*>(row_start + p.B + 1);  // [B]
   float* c_s = beta_s + p.B;                                      // [B]  log2(e) / T_b
   float* ic_s = c_s + p.B;                                        // [B]  T_b / log2(e)
+  int* first_s = reinterpret_cast<int*>(ic_s + p.B);              // [B]  first row of the request that is read
 
   pdl_launch_dependents();  // the epilogue's CTAs may take over SMs as this grid's CTAs retire
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -637,7 +648,17 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   for (int b = tid; b < p.B; b += nthreads) {
     int len = p.draft_len[b];
     if (len < 0 || len > K) len = 0;
-    row_start[b + 1] = len + (bonus ? 1 : 0);
+    int cnt = len + (bonus ? 1 : 0), first = 0;
+    if (p.row_mode == ROWS_DRAFTED) {
+      cnt = len;
+    } else if (p.row_mode == ROWS_RECOVERY) {   // the epilogue has run: one row for a request that samples
+      const int n = p.accept_len[b];
+      const bool bad = (p.status_ws[b] & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+      cnt = (!bad && n >= 0 && n <= len && (n < len || bonus)) ? 1 : 0;
+      first = n;
+    }
+    row_start[b + 1] = cnt;
+    first_s[b] = first;
     beta_s[b] = p.beta[b];
     c_s[b] = kLog2e / p.temperature[b];
     ic_s[b] = p.temperature[b] * kLn2;
@@ -685,20 +706,21 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
             break;
           }
           while (row_start[b + 1] <= cr) ++b;  // cr < row_start[B], so b stays below B
-          const int t = cr - row_start[b];
+          const int t = first_s[b] + cr - row_start[b];
           const int n_valid = min(TILE, p.V - tr * TILE);
           const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)tr * TILE;
           T* dst = tiles + (size_t)stage * 3 * TILE;
           meta[stage] = TileMeta{b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b]};
           const int n_bulk = (int)(((size_t)n_valid * sizeof(T)) & ~(size_t)15) / (int)sizeof(T);
           for (int e = n_bulk; e < n_valid; ++e) {  // ragged end of the last tile: < 16 bytes per stream
-            dst[e] = hl[off + e]; dst[TILE + e] = hp[off + e]; dst[2 * TILE + e] = hm[off + e];
+            dst[e] = hl[off + e]; dst[2 * TILE + e] = hm[off + e];
+            if (kPlus) dst[TILE + e] = hp[off + e];
           }
           const uint32_t bytes = (uint32_t)(n_bulk * sizeof(T));
           if (bytes) {
-            mbar_arrive_expect_tx(&full[stage], 3 * bytes);
+            mbar_arrive_expect_tx(&full[stage], (kPlus ? 3 : 2) * bytes);
             bulk_g2s(dst, hl + off, bytes, &full[stage]);
-            bulk_g2s(dst + TILE, hp + off, bytes, &full[stage]);
+            if (kPlus) bulk_g2s(dst + TILE, hp + off, bytes, &full[stage]);
             bulk_g2s(dst + 2 * TILE, hm + off, bytes, &full[stage]);
           } else {
             mbar_arrive(&full[stage]);
@@ -728,7 +750,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
           break;
         }
         while (row_start[b + 1] <= cr) ++b;
-        const int t = cr - row_start[b];
+        const int t = first_s[b] + cr - row_start[b];
         const int n_valid = min(TILE, p.V - tr * TILE);
         const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)tr * TILE;
         T* dst = tiles + (size_t)stage * 3 * TILE;
@@ -762,9 +784,9 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       const T* sl = tiles + (size_t)stage * 3 * TILE + half * CHUNK;
       Acc a;
       if (nv >= CHUNK) {
-        if (!chunk_fast<T, CHUNK, POLY_N, NEED_P>(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.beta, mt.c, mt.inv_c))
-          chunk_pass<T, CHUNK, false>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
-      } else if (nv > 0) chunk_pass<T, CHUNK, true>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
+        if (!chunk_fast<T, CHUNK, POLY_N, SUMS>(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.beta, mt.c, mt.inv_c))
+          chunk_pass<T, CHUNK, false, SUMS>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
+      } else if (nv > 0) chunk_pass<T, CHUNK, true, SUMS>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);  // the stage may be refilled while we reduce
       if (nv > 0) {
@@ -799,21 +821,62 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
 }
 
 // ---- launch -------------------------------------------------------------------------------------------
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, bool NEED_P>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
   const size_t fixed = (size_t)STAGES * 3 * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
                        STAGES * sizeof(TileMeta) + 16;
-  const size_t smem = fixed + (size_t)(4 * p.B + 1) * sizeof(int);
-  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, NEED_P>;
+  const size_t smem = fixed + (size_t)(5 * p.B + 1) * sizeof(int);
+  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS>;
   static bool attr_set_dev[64] = {};  // per instantiation and device; sized for the largest slab
   bool& attr_set = attr_set_dev[li.device & 63];
   if (!attr_set) {
-    const size_t smem_max = fixed + (size_t)(4 * kMaxSlabB + 1) * sizeof(int);
+    const size_t smem_max = fixed + (size_t)(5 * kMaxSlabB + 1) * sizeof(int);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   kern<<<li.sm_count, (NCW + NPW) * 32, smem, s>>>(p);
+  return cudaGetLastError();
+}
+
+// ---- normalisers of the recovery rows alone ------------------------------------------------------------
+// When verification read only h_LLM and h_SLM- (the two tensors Eq. 7 needs), the streaming kernel is run once
+// more over row accept_len of the requests that sample, all four normalisers; this kernel turns that row's
+// records into its log-normalisers for the recovery kernel and flags a non-finite row.
+__global__ void __launch_bounds__(32) recovery_row_lse_kernel(const RoundParams p) {
+  const int b = blockIdx.x, lane = threadIdx.x;
+  const int K1 = p.K + 1;
+  pdl_launch_dependents();
+  pdl_wait();
+  int len = p.draft_len[b];
+  if (len < 0 || len > p.K) len = 0;
+  const int n = p.accept_len[b], status = p.status_ws[b];
+  const bool bad = (status & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+  if (bad || !(n < len || (p.flags & SPECSTEER_FLAG_BONUS))) return;
+  const long long row = (long long)b * K1 + n;
+  float M[4];
+  double S[4];
+  row_sums_from_records(p, p.part + row * p.n_chunks * 8, lane, M, S);
+  const double lg = log2_pos(lane == 0 ? S[0] : (lane == 1 ? S[1] : (lane == 2 ? S[2] : S[3])));
+  bool fin = true;
+  float lse[4];
+#pragma unroll
+  for (int q = 0; q < 4; ++q) {
+    const double v = (double)M[q] + __shfl_sync(kFullMask, lg, q);
+    fin = fin && isfinite(v);
+    lse[q] = (float)v;
+  }
+  if (lane == 0) {
+    *reinterpret_cast<float4*>(p.lse2 + row * 4) = make_float4(lse[0], lse[1], lse[2], lse[3]);
+    if (!fin) {
+      p.status_ws[b] = status | SPECSTEER_REQ_NONFINITE;
+      if (p.req_status) p.req_status[b] = status | SPECSTEER_REQ_NONFINITE;
+    }
+  }
+}
+
+cudaError_t launch_recovery_row_lse(const RoundParams& p, cudaStream_t s) {
+  recovery_row_lse_kernel<<<p.B, 32, 0, s>>>(p);
   return cudaGetLastError();
 }
 
@@ -864,15 +927,20 @@ cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, 
   // Ring shape per logit type, from sweeps on the two largest benchmark shapes: float32 is bound by memory and
   // runs best with 144 KB in flight (12 stages, 6 consumer pairs, 3 producers: 0.350 ms against 0.379 ms for
   // 16/16/4 on 2.33 GB); 16-bit logits need the arithmetic of 8 pairs and 4 producers (12/12/3 is 12 % slower).
-  const bool np = p.need_p != 0;
+  // the three sets of normalisers that occur: all four; without h_SLM+'s; h_LLM and h_SLM- alone (then the
+  // h_SLM+ tensor is not read at all).  Rows that are not 16-byte aligned always take the full set.
+  constexpr int kNoPlus = SUM_L | SUM_M | SUM_R, kRatio = SUM_L | SUM_M;
+  const int sums = !aligned ? SUM_ALL : ((p.sums & SUM_P) ? SUM_ALL : ((p.sums & SUM_R) ? kNoPlus : kRatio));
   if (dtype == SPECSTEER_F32) {
-    return aligned ? (np ? launch_stream<float, kChunkF32, 12, 12, 3, true, true>(p, li, s)
-                         : launch_stream<float, kChunkF32, 12, 12, 3, true, false>(p, li, s))
-                   : launch_stream<float, kChunkF32, 16, 16, 4, false, true>(p, li, s);
+    if (!aligned) return launch_stream<float, kChunkF32, 16, 16, 4, false, SUM_ALL>(p, li, s);
+    if (sums == SUM_ALL) return launch_stream<float, kChunkF32, 12, 12, 3, true, SUM_ALL>(p, li, s);
+    if (sums == kNoPlus) return launch_stream<float, kChunkF32, 12, 12, 3, true, kNoPlus>(p, li, s);
+    return launch_stream<float, kChunkF32, 12, 12, 3, true, kRatio>(p, li, s);
   }
-  return aligned ? (np ? launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, true>(p, li, s)
-                       : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, false>(p, li, s))
-                 : launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, true>(p, li, s);
+  if (!aligned) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, SUM_ALL>(p, li, s);
+  if (sums == SUM_ALL) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL>(p, li, s);
+  if (sums == kNoPlus) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kNoPlus>(p, li, s);
+  return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kRatio>(p, li, s);
 }
 
 cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s) {

@@ -141,6 +141,55 @@ def test_outputs_not_requested_skip_the_plus_normaliser(env, dtype):
     P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), 0, 0, 1, P.TOL[inputs["h_llm"].dtype])
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, 1])
+def test_algorithm1_outputs_only_leave_h_slm_plus_unread_in_verification(env, dtype, flags):
+    """RATIO + STEER with none of logp_plus, logp_star, log_z requested: verification reads h_LLM and h_SLM- alone
+    (Eq. 7 needs nothing else; to prove it h_SLM+ is poisoned on every row that is not a recovery row) and
+    the recovery call forms the normalisers of its one row.  Decisions and tokens must match the oracle."""
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], 9, 4, 9004 if dtype == "f32" else 12288, dtype, seed=31, ragged=True,
+                          beta_choices=(0.5, 1.0, 2.0), temp_choices=(0.7, 1.0))
+    inputs["draft_len"][0] = 0
+    inputs["u_accept"][1] = 0.0                      # everything accepted: the bonus row (or nothing) is recovered
+    inputs["h_llm"][2, 1, 17] = float("nan")         # a non-finite drafted row
+    inputs["lam"][3] = 1e30                          # rejected at once, and row 0 is non-finite only through h_SLM+:
+    inputs["h_slm_plus"][3, 0, 5] = float("inf")     # verification cannot see it, the recovery of that row does
+    skip = ("logp_plus", "logp_star", "log_z")
+    ora = P.run_oracle(env["oracle"], P.to_np_inputs(inputs), 0, 0, flags)
+    # poison h_SLM+ wherever Algorithm 1 does not need it: all rows but row accept_len of a sampling request
+    poisoned = dict(inputs)
+    hp = inputs["h_slm_plus"].clone()
+    keep = torch.zeros(hp.shape[:2], dtype=torch.bool, device="cuda")
+    for r in range(spec.B):
+        n, ln = int(ora["accept_len"][r]), int(inputs["draft_len"][r])
+        if n < ln or flags:
+            keep[r, n] = True
+    hp[~keep] = float("nan")
+    poisoned["h_slm_plus"] = hp
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in skip}
+    d = b.make_desc(poisoned, outs, flags=flags)
+    before = env["ctx"].launch_count
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0
+    assert env["ctx"].launch_count - before == 5      # stream + epilogue; recovery rows' stream + their normalisers + sampling
+    gpu = {k: v.cpu().numpy() for k, v in outs.items()}
+    safe = (ora["accept_margin"] > P.MARGIN).all(axis=1) & (ora["cdf_margin"] > P.MARGIN)
+    assert safe.sum() >= spec.B - 1
+    for k in ("accept_len", "rec_token", "n_out", "req_status", "out_tokens"):
+        assert np.array_equal(gpu[k][safe], ora[k][safe]), k
+    assert gpu["req_status"][3] == b.REQ_NONFINITE and gpu["rec_token"][3] == -1 and gpu["accept_len"][3] == 0
+    safe[3] = False      # its per-position diagnostics differ by design: the oracle reads h_SLM+ on drafted rows
+    tol = P.TOL[inputs["h_llm"].dtype]
+    assert np.array_equal(gpu["accept_flags"][safe], ora["accept_flags"][safe])
+    for k in ("alpha", "logp_llm", "logp_minus", "rec_logprob"):
+        fin = np.isfinite(ora[k]) & (safe[:, None] if ora[k].ndim == 2 else safe)
+        assert np.array_equal(np.isnan(gpu[k][safe]), np.isnan(ora[k][safe])), k
+        assert np.abs(gpu[k][fin] - ora[k][fin]).max(initial=0.0) <= tol, k
+
+
 def test_draft_length_extremes_and_no_bonus(env):
     """len 0 (with and without the bonus row: a request that reads nothing), len K, ragged in between."""
     spec, inputs = _small(env["synth"], 9, 4, 3000, "f32", seed=3)
