@@ -184,11 +184,14 @@ def run_cuda(args, rank, world, local_rank):
     rows = synth.used_rows(spec, inputs["draft_len"], bonus=True)
     positions = int(inputs["draft_len"].sum().item())
     logit_bytes = spec.logit_bytes(rows)
+    if args.lean:   # the timed streaming launch reads two tensors over the drafted rows only
+        logit_bytes = 2 * positions * spec.V * spec.elem_bytes
     ctx = binding.Context(spec.B, spec.K, spec.V, device=local_rank)
     outs = binding.alloc_outputs(spec.B, spec.K, dev)
-    if args.lean:   # only what Algorithm 1 needs: without these two the normaliser of h_SLM+ is not formed
-        outs.pop("logp_plus")
-        outs.pop("log_z")
+    if args.lean:   # only what Algorithm 1 needs: verification then reads h_LLM and h_SLM- alone (Eq. 7) over the drafted
+        # rows, and the recovery call streams its one row per request (Eq. 8)
+        for name in ("logp_plus", "logp_star", "log_z"):
+            outs.pop(name)
     desc = binding.make_desc(inputs, outs, flags=flags)
     stream = torch.cuda.current_stream(dev)
 
@@ -300,8 +303,8 @@ def run_cuda(args, rank, world, local_rank):
     host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
     host_out = binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True)
     if args.lean:
-        host_out.pop("logp_plus")
-        host_out.pop("log_z")
+        for name in ("logp_plus", "logp_star", "log_z"):
+            host_out.pop(name)
     hdesc = binding.make_desc(host_in, host_out, flags=flags)
     h2d = sum(v.numel() * v.element_size() for v in host_in.values())
     d2h = sum(v.numel() * v.element_size() for v in host_out.values())
@@ -362,7 +365,7 @@ def run_cuda(args, rank, world, local_rank):
         "config": {"workload": spec.name, "B": spec.B, "K": spec.K, "V": spec.V, "logit_dtype": spec.dtype,
                    "requests_per_gpu": spec.B, "rows_read_per_gpu": rows, "positions_per_step_per_gpu": positions,
                    "accept_mode": "ratio", "recover_mode": "steer", "bonus_row": True, "lambda": spec.lam,
-                   "outputs": "Algorithm 1 only (no logp_plus, log_z)" if args.lean else "all",
+                   "outputs": "Algorithm 1 only (no logp_plus, logp_star, log_z)" if args.lean else "all",
                    "acceptance_rate": float(outs["accept_len"].sum().item()) / max(1, positions),
                    "l2": ("inputs %.2f GB per step exceed L2" % (logit_bytes / 1e9)) if n_sets == 1 else
                          ("rotating %d input sets (%.2f GB) to exceed L2" % (n_sets, n_sets * logit_bytes / 1e9)),
@@ -389,7 +392,7 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--requests", type=int, default=0, help="override B (reduced batch for profiler captures)")
     ap.add_argument("--lean", action="store_true",
-                    help="request only the outputs Algorithm 1 needs (no logp_plus, log_z): three normalisers per row")
+                    help="request only the outputs Algorithm 1 needs (no logp_plus, logp_star, log_z)")
     ap.add_argument("--topk", type=int, default=0,
                     help="with --kernels-only: also time the top-k split recovery (cloud + edge kernels) with this k")
     ap.add_argument("--kernels-only", action="store_true",

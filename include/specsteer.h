@@ -92,11 +92,16 @@ typedef struct {
   const float *u_recover;                       /* [B]      uniform in [0,1) for the recovery sample */
 
   /* ---- outputs (caller-allocated; any may be NULL except accept_len) ----
-   * Algorithm 1 itself needs three normalisers per row (h_LLM and h_SLM- for Eq. 7, h_rec for Eq. 8).  The
-   * fourth, of h_SLM+, is formed only when something asks for it: a non-NULL logp_plus or log_z, EXACT_Z
-   * acceptance or RESIDUAL recovery.  Leaving logp_plus and log_z NULL in RATIO + STEER mode therefore saves a
-   * quarter of the exponentials (it matters for 16-bit logits, where they bind before the memory does).  The other
-   * outputs then keep their decisions and tokens; their floating-point values may differ in the last bits. */
+   * What is requested decides what is read.  Algorithm 1 itself needs the normalisers of h_LLM and h_SLM- on the
+   * drafted rows (Eq. 7) and that of h_rec on the one row it recovers from (Eq. 8).
+   *   - RATIO + STEER with logp_plus, logp_star and log_z all NULL (and 16-byte aligned rows): verification reads
+   *     h_LLM and h_SLM- alone, over the drafted rows; specsteer_recover_sample then streams row accept_len of the
+   *     requests that sample, all three tensors.  About a fifth fewer bytes per round.  A non-finite entry of
+   *     h_SLM+ on a drafted row is then not seen (REQ_NONFINITE is raised for it only on the recovery row).
+   *   - logp_star wanted, logp_plus and log_z NULL: one pass over all three tensors and all rows, but the
+   *     normaliser of h_SLM+ is not formed (a quarter fewer exponentials; it matters for 16-bit logits).
+   *   - otherwise (logp_plus or log_z wanted, EXACT_Z, RESIDUAL): all four normalisers on every row.
+   * Decisions and tokens are the same in all three; floating-point outputs may differ in the last bits. */
   int32_t *accept_len;   /* [B]      drafts accepted before the first rejection */
   uint8_t *accept_flags; /* [B][K]   1 where u <= alpha (every drafted position, also after the first rejection) */
   float *alpha;          /* [B][K]   acceptance probability; 0 beyond draft_len */
