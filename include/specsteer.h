@@ -61,7 +61,10 @@ typedef enum { SPECSTEER_ACCEPT_RATIO = 0, SPECSTEER_ACCEPT_EXACT_Z = 1 } specst
 typedef enum { SPECSTEER_RECOVER_STEER = 0, SPECSTEER_RECOVER_RESIDUAL = 1 } specsteer_recover_mode;
 
 enum {
-  SPECSTEER_FLAG_BONUS = 1u /* when all drafts are accepted, also sample one token (STEER) from row draft_len */
+  SPECSTEER_FLAG_BONUS = 1u,    /* when all drafts are accepted, also sample one token (STEER) from row draft_len */
+  SPECSTEER_FLAG_TWO_PHASE = 2u /* take the two-phase round (see the outputs below) whenever it is eligible, however
+                                   small the batch; without it the library takes it from 128 MB of logits upwards,
+                                   below which its two extra launches cost more than the bytes it saves */
 };
 
 /* bits of req_status[b] */
@@ -96,7 +99,8 @@ typedef struct {
    * drafted rows (Eq. 7) and that of h_rec on the one row it recovers from (Eq. 8).
    *   - RATIO + STEER with logp_plus, logp_star and log_z all NULL (and 16-byte aligned rows): verification reads
    *     h_LLM and h_SLM- alone, over the drafted rows; specsteer_recover_sample then streams row accept_len of the
-   *     requests that sample, all three tensors.  About a fifth fewer bytes per round.  A non-finite entry of
+   *     requests that sample, all three tensors: the two-phase round, about a fifth fewer bytes (taken automatically
+   *     for large batches, see SPECSTEER_FLAG_TWO_PHASE).  A non-finite entry of
    *     h_SLM+ on a drafted row is then not seen (REQ_NONFINITE is raised for it only on the recovery row).
    *   - logp_star wanted, logp_plus and log_z NULL: one pass over all three tensors and all rows, but the
    *     normaliser of h_SLM+ is not formed (a quarter fewer exponentials; it matters for 16-bit logits).

@@ -20,6 +20,7 @@ F32, BF16 = 0, 1
 ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
 RECOVER_STEER, RECOVER_RESIDUAL = 0, 1
 FLAG_BONUS = 1
+FLAG_TWO_PHASE = 2
 REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1, 2, 4, 8, 16
 
 EXPORTS = (

@@ -71,7 +71,7 @@ specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc
     return SPECSTEER_ERR_INVALID_ARG;
   if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL)
     return SPECSTEER_ERR_INVALID_ARG;
-  if (d->flags & ~(uint32_t)SPECSTEER_FLAG_BONUS) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
   if (d->B > 0) {
     if (!d->h_llm || !d->h_slm_plus || !d->h_slm_minus || !d->draft_len || !d->lambda || !d->beta ||
         !d->temperature || !d->u_recover || !d->accept_len)
@@ -131,8 +131,13 @@ bool rows_aligned(const specsteer_round_desc* d) {
 // fused target on the drafted rows, the h_SLM+ tensor is left unread there and the recovery call forms the
 // normalisers of its one row itself (Eq. 8 on the row of the first rejection).
 bool two_phase(const specsteer_round_desc* d) {
-  return d->accept_mode == SPECSTEER_ACCEPT_RATIO && d->recover_mode == SPECSTEER_RECOVER_STEER && !d->logp_plus &&
-         !d->logp_star && !d->log_z && rows_aligned(d);
+  const bool eligible = d->accept_mode == SPECSTEER_ACCEPT_RATIO && d->recover_mode == SPECSTEER_RECOVER_STEER &&
+                        !d->logp_plus && !d->logp_star && !d->log_z && rows_aligned(d);
+  if (!eligible) return false;
+  if (d->flags & SPECSTEER_FLAG_TWO_PHASE) return true;
+  // two more launches (about 10 us) against a fifth of the bytes: worth it from roughly 128 MB of logits upwards
+  const double bytes = 3.0 * d->B * (d->K + 1) * (double)d->V * (d->dtype == SPECSTEER_F32 ? 4 : 2);
+  return bytes >= 128.0 * 1024 * 1024;
 }
 
 specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {

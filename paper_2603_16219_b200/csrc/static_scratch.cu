@@ -66,7 +66,7 @@ extern "C" specsteer_status specsteer_verify_round_static(const specsteer_round_
     return SPECSTEER_ERR_INVALID_ARG;
   if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL)
     return SPECSTEER_ERR_INVALID_ARG;
-  if (d->flags & ~(uint32_t)SPECSTEER_FLAG_BONUS) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
   const int tile = d->dtype == SPECSTEER_F32 ? kChunkF32 : kChunkBF16;
   const int n_chunks = (d->V + tile - 1) / tile;
   const long long rows = (long long)d->B * (d->K + 1);

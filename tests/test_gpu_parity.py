@@ -168,7 +168,7 @@ def test_algorithm1_outputs_only_leave_h_slm_plus_unread_in_verification(env, dt
     hp[~keep] = float("nan")
     poisoned["h_slm_plus"] = hp
     outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in skip}
-    d = b.make_desc(poisoned, outs, flags=flags)
+    d = b.make_desc(poisoned, outs, flags=flags | b.FLAG_TWO_PHASE)
     before = env["ctx"].launch_count
     env["ctx"].verify_round(d)
     env["ctx"].recover_sample(d)
