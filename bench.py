@@ -300,6 +300,35 @@ def run_cuda(args, rank, world, local_rank):
             dist.barrier()
             dist.destroy_process_group()
         return
+    # ---- beside the headline: the same batch with only the outputs Algorithm 1 needs (the two-phase round for
+    # large batches: h_LLM and h_SLM- over the drafted rows, then one recovery row per request)
+    alg1 = None
+    if not args.lean:
+        lean_outs = {k: v for k, v in binding.alloc_outputs(spec.B, spec.K, dev).items()
+                     if k not in ("logp_plus", "logp_star", "log_z")}
+        lean_sets = [binding.make_desc(si, lean_outs, flags=flags) for si, _ in sets]
+        n_lean = min(args.steps, 200)
+        for i in range(3):
+            ctx.verify_round(lean_sets[i % n_sets], stream)
+            ctx.recover_sample(lean_sets[i % n_sets], stream)
+        barrier()
+        l0, l1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.perf_counter()
+        l0.record(stream)
+        for i in range(n_lean):
+            ctx.verify_round(lean_sets[i % n_sets], stream)
+            ctx.recover_sample(lean_sets[i % n_sets], stream)
+        l1.record(stream)
+        barrier()
+        sampler.window(w0, time.perf_counter())
+        lean_ms = l0.elapsed_time(l1) / n_lean
+        if dist is not None:
+            t = torch.tensor([lean_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            lean_ms = float(t.item())
+        same = torch.equal(lean_outs["accept_len"], outs["accept_len"]) and torch.equal(lean_outs["rec_token"], outs["rec_token"])
+        alg1 = {"value": world * positions / (lean_ms * 1e-3), "unit": UNIT, "ms_per_step": lean_ms, "steps": n_lean,
+                "outputs": "no logp_plus, logp_star, log_z", "same_accept_len_and_tokens_as_headline": bool(same)}
     # ---- end to end: pinned host buffers in, pinned host results out, copies inside the timed region
     host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
     host_out = binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True)
@@ -375,6 +404,7 @@ def run_cuda(args, rank, world, local_rank):
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "api": "specsteer_round_host (pinned host buffers)"},
+        "algorithm1_outputs_only": alg1,
         "gpu_launches": int(gpu_launches),
         "clocks": sampler.summary(),
     }
