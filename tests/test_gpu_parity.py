@@ -293,6 +293,16 @@ def test_many_requests_cross_the_slab_limit(env):
     sel = np.unique(sel)
     npin = P.to_np_inputs(inputs, torch.as_tensor(sel, device="cuda"))
     P.compare(env["oracle"], gpu, npin, 0, 0, 1, 2e-3, sel=sel)
+    # the two-phase round over the same slabs: same decisions and tokens
+    b = env["binding"]
+    lean = {k: v for k, v in b.alloc_outputs(5000, 2, "cuda").items() if k not in ("logp_plus", "logp_star", "log_z")}
+    d = b.make_desc(inputs, lean, flags=b.FLAG_BONUS | b.FLAG_TWO_PHASE)
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0
+    for k in ("accept_len", "accept_flags", "rec_token", "out_tokens", "n_out", "req_status"):
+        assert np.array_equal(lean[k].cpu().numpy(), gpu[k]), k
 
 
 def test_zero_requests_and_zero_drafts(env):
