@@ -73,13 +73,27 @@ def test_config_full_size_sampled_parity(env, cfg):
     env["ctx"].verify_round(d)
     env["ctx"].recover_sample(d)
     torch.cuda.synchronize()
-    for k, v in lean.items():
-        got = v.cpu().numpy()
-        if got.dtype.kind in "iu":
-            assert np.array_equal(got, full[k]), k
-        else:
-            assert np.array_equal(np.isnan(got), np.isnan(full[k])), k
-            assert np.nanmax(np.abs(got - full[k]), initial=0.0) <= 1e-5, k
+    def same_as_full(got_outs):
+        for k, v in got_outs.items():
+            got = v.cpu().numpy()
+            if got.dtype.kind in "iu":
+                assert np.array_equal(got, full[k]), k
+            else:
+                assert np.array_equal(np.isnan(got), np.isnan(full[k])), k
+                assert np.nanmax(np.abs(got - full[k]), initial=0.0) <= 1e-5, k
+
+    same_as_full(lean)
+    # and the two-phase round `bench.py --lean` times (these batches are large enough for it to be automatic):
+    # h_LLM and h_SLM- over the drafted rows, then one recovery row per request
+    alg1 = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items()
+            if k not in ("logp_plus", "logp_star", "log_z")}
+    d = b.make_desc(inputs, alg1, flags=1)
+    before = env["ctx"].launch_count
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].launch_count - before == 5
+    same_as_full(alg1)
 
 
 # ------------------------------------------------------------------ shapes, tails, strides
