@@ -22,12 +22,15 @@ def env(oracle_mod):
     ctx.close()
 
 
-def _run(env, inputs, k, flags, V=None):
+def _run(env, inputs, k, flags, V=None, cloud_only_verification=False):
     b, o = env["binding"], env["oracle"]
     hl = inputs["h_llm"]
     B, K = hl.shape[0], hl.shape[1] - 1
     outs = b.alloc_outputs(B, K, "cuda")
-    desc = b.make_desc(inputs, outs, flags=flags, V=V)
+    if cloud_only_verification:      # verification that never reads h_SLM+, as on the paper's cloud
+        for name in ("logp_plus", "logp_star", "log_z"):
+            outs.pop(name)
+    desc = b.make_desc(inputs, outs, flags=flags | (b.FLAG_TWO_PHASE if cloud_only_verification else 0), V=V)
     idx = torch.full((B, k), -7, dtype=torch.int32, device="cuda")
     val = torch.full((B, k), 123.0, dtype=torch.float32, device="cuda")
     env["ctx"].verify_round(desc)
@@ -41,7 +44,7 @@ def _run(env, inputs, k, flags, V=None):
     if V is not None:
         npin = {k_: (v[..., :V] if k_.startswith("h_") else v) for k_, v in npin.items()}
         npin = {k_: (np.ascontiguousarray(v) if k_.startswith("h_") else v) for k_, v in npin.items()}
-    ora = P.run_oracle(o, npin, 0, 0, flags)
+    ora = P.run_oracle(o, npin, 0, 0, flags & 1)
     safe = (ora["accept_margin"] > P.MARGIN).all(axis=1)
     assert np.array_equal(gpu["accept_len"][safe], ora["accept_len"][safe])
     top = o.topk_recover_round(npin["h_llm"], npin["h_slm_plus"], npin["h_slm_minus"], npin["draft_len"], npin["beta"],
@@ -116,6 +119,16 @@ def test_topk_on_benchmark_shapes(env, cfg):
     inputs = env["synth"].make_round(spec, device="cuda", seed=cfg)
     gpu, top = _run(env, inputs, 32, 1)
     assert (gpu["rec_token"] >= 0).all()
+
+
+def test_topk_after_verification_without_h_slm_plus(env):
+    """The deployment the appendix describes: the cloud verifies with h_LLM and h_SLM- alone and truncates, the edge
+    adds its private term.  h_SLM+ is read by the edge kernel only."""
+    spec = env["synth"].RoundSpec("topk_cloud", 7, 4, 16384, "bf16", ragged=True, beta_choices=(0.5, 1.0, 2.0))
+    inputs = env["synth"].make_round(spec, device="cuda", seed=41)
+    before = env["ctx"].launch_count
+    _run(env, inputs, 32, 1, cloud_only_verification=True)
+    assert env["ctx"].launch_count - before == 4      # streaming (two tensors) + epilogue, cloud_topk, edge_resample
 
 
 def test_topk_argument_checks(env):
