@@ -146,7 +146,12 @@ specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cu
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
     RoundParams p = slab_params(ctx, d, b0, nb);
-    if (lean) { p.sums = SUM_L | SUM_M; p.row_mode = ROWS_DRAFTED; }
+    if (lean) {   // two tensors over the drafted rows, in the larger chunks of that launch shape
+      p.sums = SUM_L | SUM_M;
+      p.row_mode = ROWS_DRAFTED;
+      p.tile = d->dtype == SPECSTEER_F32 ? kChunkRatioF32 : kChunkRatioBF16;
+      p.n_chunks = n_chunks_of(d->V, p.tile);
+    }
     int nl = 0;
     const bool first = b0 == 0, last = b0 + nb >= d->B;
     if (launch_verify(p, d->dtype, aligned, ctx->li, s, &nl, first ? ctx->ev_stream_begin : nullptr,

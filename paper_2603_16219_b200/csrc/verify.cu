@@ -619,7 +619,9 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   static_assert(NCW % 2 == 0 && STAGES % NPAIR == 0, "each stage belongs to one fixed pair of consumer warps");
   static_assert(STAGES % NPW == 0, "each producer owns a fixed subset of the stages");
   extern __shared__ __align__(128) unsigned char smem_raw[];
-  constexpr int kStageBytes = 3 * TILE * (int)sizeof(T);
+  constexpr int NSLOT = kPlus ? 3 : 2;                   // streams held per stage
+  constexpr int MSLOT = NSLOT - 1;                       // slot of h_SLM-
+  constexpr int kStageBytes = NSLOT * TILE * (int)sizeof(T);
   T* tiles = reinterpret_cast<T*>(smem_raw);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem_raw + (size_t)STAGES * kStageBytes);
   uint64_t* empty = full + STAGES;
@@ -709,11 +711,11 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
           const int t = first_s[b] + cr - row_start[b];
           const int n_valid = min(TILE, p.V - tr * TILE);
           const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)tr * TILE;
-          T* dst = tiles + (size_t)stage * 3 * TILE;
+          T* dst = tiles + (size_t)stage * NSLOT * TILE;
           meta[stage] = TileMeta{b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b]};
           const int n_bulk = (int)(((size_t)n_valid * sizeof(T)) & ~(size_t)15) / (int)sizeof(T);
           for (int e = n_bulk; e < n_valid; ++e) {  // ragged end of the last tile: < 16 bytes per stream
-            dst[e] = hl[off + e]; dst[2 * TILE + e] = hm[off + e];
+            dst[e] = hl[off + e]; dst[MSLOT * TILE + e] = hm[off + e];
             if (kPlus) dst[TILE + e] = hp[off + e];
           }
           const uint32_t bytes = (uint32_t)(n_bulk * sizeof(T));
@@ -721,7 +723,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
             mbar_arrive_expect_tx(&full[stage], (kPlus ? 3 : 2) * bytes);
             bulk_g2s(dst, hl + off, bytes, &full[stage]);
             if (kPlus) bulk_g2s(dst + TILE, hp + off, bytes, &full[stage]);
-            bulk_g2s(dst + 2 * TILE, hm + off, bytes, &full[stage]);
+            bulk_g2s(dst + MSLOT * TILE, hm + off, bytes, &full[stage]);
           } else {
             mbar_arrive(&full[stage]);
           }
@@ -781,12 +783,12 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       }
       const TileMeta mt = meta[stage];
       const int nv = mt.n_valid - half * CHUNK;  // valid entries in this warp's chunk
-      const T* sl = tiles + (size_t)stage * 3 * TILE + half * CHUNK;
+      const T* sl = tiles + (size_t)stage * NSLOT * TILE + half * CHUNK;
       Acc a;
       if (nv >= CHUNK) {
-        if (!chunk_fast<T, CHUNK, POLY_N, SUMS>(a, sl, sl + TILE, sl + 2 * TILE, lane, mt.beta, mt.c, mt.inv_c))
-          chunk_pass<T, CHUNK, false, SUMS>(a, sl, sl + TILE, sl + 2 * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
-      } else if (nv > 0) chunk_pass<T, CHUNK, true, SUMS>(a, sl, sl + TILE, sl + 2 * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
+        if (!chunk_fast<T, CHUNK, POLY_N, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, mt.beta, mt.c, mt.inv_c))
+          chunk_pass<T, CHUNK, false, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
+      } else if (nv > 0) chunk_pass<T, CHUNK, true, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
       if (lane == 0) mbar_arrive(&empty[stage]);  // the stage may be refilled while we reduce
       if (nv > 0) {
@@ -823,7 +825,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
 // ---- launch -------------------------------------------------------------------------------------------
 template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
-  const size_t fixed = (size_t)STAGES * 3 * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
+  const size_t fixed = (size_t)STAGES * ((SUMS & (SUM_P | SUM_R)) ? 3 : 2) * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
                        STAGES * sizeof(TileMeta) + 16;
   const size_t smem = fixed + (size_t)(5 * p.B + 1) * sizeof(int);
   auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS>;
@@ -935,12 +937,12 @@ cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, 
     if (!aligned) return launch_stream<float, kChunkF32, 16, 16, 4, false, SUM_ALL>(p, li, s);
     if (sums == SUM_ALL) return launch_stream<float, kChunkF32, 12, 12, 3, true, SUM_ALL>(p, li, s);
     if (sums == kNoPlus) return launch_stream<float, kChunkF32, 12, 12, 3, true, kNoPlus>(p, li, s);
-    return launch_stream<float, kChunkF32, 12, 12, 3, true, kRatio>(p, li, s);
+    return launch_stream<float, kChunkRatioF32, 12, 12, 3, true, kRatio>(p, li, s);
   }
   if (!aligned) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, SUM_ALL>(p, li, s);
   if (sums == SUM_ALL) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL>(p, li, s);
   if (sums == kNoPlus) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kNoPlus>(p, li, s);
-  return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kRatio>(p, li, s);
+  return launch_stream<uint16_t, kChunkRatioBF16, 16, 16, 4, true, kRatio>(p, li, s);
 }
 
 cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s) {
