@@ -25,6 +25,8 @@ if ROOT not in sys.path:
 METRIC = "verified_draft_positions_per_sec"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0
+N_SM = 148
+EX2_PER_CLK_PER_SM = 16
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per used row of the streaming kernel, from the ncu captures summarised under
 # profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows), keyed by
@@ -373,6 +375,15 @@ def run_cuda(args, rank, world, local_rank):
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "whole_step_gbs": logit_bytes / (ms_per_step * 1e-3) / 1e9,
     }
+    # The second ceiling of the streaming kernel: one ex2 per normaliser and vocabulary entry on the
+    # special-function unit (16 results per clock and SM: 4 per sub-partition), at the clock sampled under load.
+    clk = sampler.summary()
+    if not args.lean and clk.get("sm_mhz"):
+        n_ex2 = 4.0 * rows * spec.V
+        sfu_peak = N_SM * EX2_PER_CLK_PER_SM * clk["sm_mhz"] * 1e6
+        roofline["sfu"] = {"ex2_per_launch": n_ex2, "achieved": n_ex2 / (kernel_ms * 1e-3), "peak": sfu_peak,
+                           "unit": "ex2/s", "frac": n_ex2 / (kernel_ms * 1e-3) / sfu_peak,
+                           "peak_source": "derived: 16 ex2 per clock per SM x 148 SMs x median SM clock under load"}
     cpu = None
     if world == 1:
         import oracle

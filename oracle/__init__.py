@@ -23,7 +23,7 @@ _SRC_TOPK = os.path.join(_HERE, "specsteer_oracle_topk.c")
 _HDR = os.path.join(_HERE, "specsteer_oracle.h")
 _LIB = os.path.join(_HERE, "libspecsteer_oracle.so")
 
-DTYPE_F32, DTYPE_BF16 = 0, 1
+DTYPE_F32, DTYPE_BF16, DTYPE_F64 = 0, 1, 2
 ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
 RECOVER_STEER, RECOVER_RESIDUAL = 0, 1
 FLAG_BONUS = 1
@@ -98,7 +98,9 @@ def _logits(a):
         return a, DTYPE_F32
     if a.dtype == np.uint16:
         return a, DTYPE_BF16
-    raise TypeError("logits must be float32 or uint16 (bf16 bit patterns), got %s" % a.dtype)
+    if a.dtype == np.float64:
+        return a, DTYPE_F64
+    raise TypeError("logits must be float32, float64 or uint16 (bf16 bit patterns), got %s" % a.dtype)
 
 
 def _p(a):
@@ -169,7 +171,7 @@ def cloud_topk_row(h_llm, h_minus, beta, k):
     """Cloud half of the top-k split recovery on one row: (ids[k] int32, values[k] float32)."""
     hl, dt = _logits(h_llm)
     hm, dt2 = _logits(h_minus)
-    assert dt == dt2 and hl.ndim == 1 and hl.shape == hm.shape
+    assert dt == dt2 and dt != DTYPE_F64 and hl.ndim == 1 and hl.shape == hm.shape
     idx = np.empty(k, np.int32)
     val = np.empty(k, np.float32)
     rc = lib().specsteer_oracle_cloud_topk_row(hl.shape[0], dt, _p(hl), _p(hm), float(beta), int(k), _p(idx), _p(val))
@@ -181,6 +183,7 @@ def cloud_topk_row(h_llm, h_minus, beta, k):
 def edge_resample_row(h_plus, beta, temperature, idx, val, u):
     """Edge half on one row: dict(token, logprob, probs[k], cdf_margin)."""
     hp, dt = _logits(h_plus)
+    assert dt != DTYPE_F64
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     val = np.ascontiguousarray(val, dtype=np.float32)
     k = idx.shape[0]
@@ -214,3 +217,29 @@ def topk_recover_round(h_llm, h_slm_plus, h_slm_minus, draft_len, beta, temperat
         out["topk_idx"][b], out["topk_val"][b] = idx, val
         out["rec_token"][b], out["rec_logprob"][b], out["cdf_margin"][b] = r["token"], r["logprob"], r["cdf_margin"]
     return out
+
+
+# ---- the LM head in front of the round ------------------------------------------------------------------
+def bf16_to_f64(bits):
+    """Exact values of bf16 bit patterns (the upper half of an IEEE float32), as float64."""
+    bits = np.ascontiguousarray(bits, dtype=np.uint16)
+    return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def lmhead_logits(x_bits, w_bits):
+    """h = x W^T: the logits an LM head gives for hidden states x [..., d] and head weights W [V, d] (the h_LLM and
+    h_SLM of Algorithm 1's verification and recovery steps), both bf16, every product and sum in float64."""
+    x = bf16_to_f64(x_bits)
+    w = bf16_to_f64(w_bits)
+    assert x.shape[-1] == w.shape[1]
+    return np.matmul(x, w.T)
+
+
+def lmhead_verify_recover_round(x_llm, w_llm, x_plus, w_plus, x_minus, w_minus, draft_tokens, draft_len, lam, beta,
+                                temperature, u_accept, u_recover, **kw):
+    """The round of Algorithm 1 on logits that are first formed from hidden states [B, K+1, d] and head weights
+    [V, d]: float64 logits, then `verify_recover_round` as it stands."""
+    hl = lmhead_logits(x_llm, w_llm)
+    hp = lmhead_logits(x_plus, w_plus)
+    hm = lmhead_logits(x_minus, w_minus)
+    return verify_recover_round(hl, hp, hm, draft_tokens, draft_len, lam, beta, temperature, u_accept, u_recover, **kw)

@@ -42,6 +42,8 @@
 static double logit_at(const void *base, int dtype, int64_t idx) {
   if (dtype == ORACLE_DTYPE_F32) {
     return (double)((const float *)base)[idx];
+  } else if (dtype == ORACLE_DTYPE_F64) { /* logits that were themselves computed in double (the LM-head path) */
+    return ((const double *)base)[idx];
   } else { /* bf16: the upper 16 bits of an IEEE float32 */
     uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
     float f;

@@ -11,7 +11,7 @@
 extern "C" {
 #endif
 
-enum { ORACLE_DTYPE_F32 = 0, ORACLE_DTYPE_BF16 = 1 };
+enum { ORACLE_DTYPE_F32 = 0, ORACLE_DTYPE_BF16 = 1, ORACLE_DTYPE_F64 = 2 };
 enum { ORACLE_ACCEPT_RATIO = 0 /* Eq. 7 */, ORACLE_ACCEPT_EXACT_Z = 1 /* Eq. 6 */ };
 enum { ORACLE_RECOVER_STEER = 0 /* Eq. 8 softmax */, ORACLE_RECOVER_RESIDUAL = 1 };
 enum { ORACLE_FLAG_BONUS = 1u };
