@@ -194,6 +194,32 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx *ctx, const specste
                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
                                                int32_t vocab_total, void *cuda_stream);
 
+/* The round with the three LM heads fused in front of it.  Algorithm 1's verification and recovery steps read the
+ * logits of three forward passes, h = x W^T: the Generalist (h_LLM), and the Specialist with and without the private
+ * context (h_SLM+, h_SLM-; the same model, hence usually the same head).  This entry point takes the hidden states and
+ * the head weights instead of the logits and never stores a logit: the products are formed tile by tile on the tensor
+ * cores (tcgen05, float32 accumulation in tensor memory), each tile is reduced at once to the per-chunk partial sums
+ * the round needs, and the recovery step (Eq. 8) recomputes the 128 logits of the one chunk it samples from.
+ *   - round: as for specsteer_verify_round + specsteer_recover_sample, except that h_llm, h_slm_plus, h_slm_minus,
+ *     ld_row, ld_req and dtype are ignored.  Every output may be requested; every row of every request is computed.
+ *   - x_*: DEVICE, bf16, [B][K+1][d] dense; w_*: DEVICE, bf16, [V][d] dense (row v = the head's weights of token v);
+ *     all 16-byte aligned, d_llm and d_slm multiples of 8.  w_slm_plus and w_slm_minus may be the same pointer.
+ *   - RATIO or EXACT_Z acceptance, STEER recovery (RESIDUAL: UNSUPPORTED).
+ *   - The first call allocates a second workspace for the context's maxima
+ *     (max_B*(max_K+1)*(16 + 32*ceil(max_V/128)) bytes); later calls allocate nothing.
+ *   - Accuracy: the logits carry the rounding of a float32 accumulation over d bf16 products, so decisions may
+ *     differ from exact arithmetic where their margin is below about 1e-4.
+ * Three launches; stream-ordered; specsteer_ctx_time_streaming brackets the tensor-core kernel.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, TIMEOUT, CUDA. */
+typedef struct {
+  specsteer_round_desc round;
+  const void *x_llm, *w_llm;             /* [B][K+1][d_llm], [V][d_llm] */
+  const void *x_slm_plus, *w_slm_plus;   /* [B][K+1][d_slm], [V][d_slm] */
+  const void *x_slm_minus, *w_slm_minus; /* [B][K+1][d_slm], [V][d_slm] */
+  int32_t d_llm, d_slm;
+} specsteer_lmhead_desc;
+specsteer_status specsteer_lmhead_round(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc, void *cuda_stream);
+
 /* Whole round from HOST memory: every pointer in `desc` is a HOST pointer (pinned memory makes the copies
  * asynchronous).  Copies inputs to device staging buffers owned by the context (allocated on the first
  * call, sized for the context's maxima: 3*max_B*(max_K+1)*max_V elements of 4 bytes), runs verification and

@@ -30,6 +30,7 @@ EXPORTS = (
     "specsteer_verify_round_static", "specsteer_ctx_time_streaming",
     "specsteer_cloud_topk", "specsteer_edge_resample",
     "specsteer_shard_verify_local", "specsteer_shard_verify_combine", "specsteer_shard_recover_local",
+    "specsteer_lmhead_round",
 )
 SHARD_PARTIAL_BYTES = 64
 MAX_SHARDS = 32
@@ -51,6 +52,17 @@ class RoundDesc(C.Structure):
         ("logp_star", C.c_void_p), ("log_z", C.c_void_p),
         ("rec_token", C.c_void_p), ("rec_logprob", C.c_void_p), ("out_tokens", C.c_void_p),
         ("n_out", C.c_void_p), ("req_status", C.c_void_p),
+    ]
+
+
+class LmheadDesc(C.Structure):
+    """Mirror of ``specsteer_lmhead_desc``."""
+    _fields_ = [
+        ("round", RoundDesc),
+        ("x_llm", C.c_void_p), ("w_llm", C.c_void_p),
+        ("x_slm_plus", C.c_void_p), ("w_slm_plus", C.c_void_p),
+        ("x_slm_minus", C.c_void_p), ("w_slm_minus", C.c_void_p),
+        ("d_llm", C.c_int32), ("d_slm", C.c_int32),
     ]
 
 
@@ -92,6 +104,8 @@ def load_library(path: Optional[str] = None):
         fn = getattr(lib, name)
         fn.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         fn.restype = C.c_int
+    lib.specsteer_lmhead_round.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p]
+    lib.specsteer_lmhead_round.restype = C.c_int
     lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.specsteer_ctx_time_streaming.restype = C.c_int
     lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
@@ -178,6 +192,52 @@ def make_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor],
     return d
 
 
+def make_lmhead_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor], *, accept_mode=ACCEPT_RATIO,
+                     flags=0) -> LmheadDesc:
+    """Descriptor of a round on hidden states and head weights: inputs hold x_llm [B, K+1, d_llm], w_llm [V, d_llm],
+    x_slm_plus / x_slm_minus [B, K+1, d_slm], w_slm_plus / w_slm_minus [V, d_slm] (bf16, contiguous) and the
+    per-request tensors of ``make_desc``."""
+    xl, wl = inputs["x_llm"], inputs["w_llm"]
+    xp, wp, xm, wm = inputs["x_slm_plus"], inputs["w_slm_plus"], inputs["x_slm_minus"], inputs["w_slm_minus"]
+    for t in (xl, wl, xp, wp, xm, wm):
+        if t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError("hidden states and head weights must be contiguous bfloat16 tensors")
+    B, K1, dL = xl.shape
+    V, dS = wp.shape
+    if wl.shape != (V, dL) or xp.shape != (B, K1, dS) or xm.shape != (B, K1, dS) or wm.shape != (V, dS):
+        raise ValueError("operand shapes do not agree")
+    K = K1 - 1
+    ld = LmheadDesc()
+    d = ld.round
+    d.B, d.K, d.V = B, K, V
+    d.ld_row, d.ld_req, d.dtype = V, K1 * V, F32
+    d.accept_mode, d.recover_mode, d.flags = int(accept_mode), RECOVER_STEER, int(flags)
+
+    def ptr(t, dt, n):
+        if t.dtype != dt or not t.is_contiguous() or t.numel() != n:
+            raise ValueError("bad auxiliary tensor: dtype %s, numel %d (want %s, %d)" % (t.dtype, t.numel(), dt, n))
+        return t.data_ptr() if n else None
+
+    d.draft_tokens = ptr(inputs["draft_tokens"], torch.int32, B * K)
+    d.draft_len = ptr(inputs["draft_len"], torch.int32, B)
+    d.lam = ptr(inputs["lam"], torch.float32, B)
+    d.beta = ptr(inputs["beta"], torch.float32, B)
+    d.temperature = ptr(inputs["temperature"], torch.float32, B)
+    d.u_accept = ptr(inputs["u_accept"], torch.float32, B * K)
+    d.u_recover = ptr(inputs["u_recover"], torch.float32, B)
+    for name, (dt, shp) in _OUT_SPECS.items():
+        t = outputs.get(name)
+        n = B
+        for s in shp(K):
+            n *= s
+        setattr(d, name, ptr(t, dt, n) if t is not None else None)
+    ld.x_llm, ld.w_llm = xl.data_ptr(), wl.data_ptr()
+    ld.x_slm_plus, ld.w_slm_plus = xp.data_ptr(), wp.data_ptr()
+    ld.x_slm_minus, ld.w_slm_minus = xm.data_ptr(), wm.data_ptr()
+    ld.d_llm, ld.d_slm = dL, dS
+    return ld
+
+
 def _check_topk(desc, topk_idx, topk_val) -> int:
     if topk_idx.dtype != torch.int32 or topk_val.dtype != torch.float32 or topk_idx.shape != topk_val.shape or \
             topk_idx.dim() != 2 or topk_idx.shape[0] != desc.B or not topk_idx.is_contiguous() or \
@@ -216,6 +276,10 @@ class Context:
     def recover_sample(self, desc: RoundDesc, stream=None):
         _check(self._lib.specsteer_recover_sample(self._h, C.byref(desc), self._stream(stream)),
                "specsteer_recover_sample")
+
+    def lmhead_round(self, desc: LmheadDesc, stream=None):
+        """Verification and recovery with the three LM heads fused in front: no logit tensor is ever stored."""
+        _check(self._lib.specsteer_lmhead_round(self._h, C.byref(desc), self._stream(stream)), "specsteer_lmhead_round")
 
     def cloud_topk(self, desc: RoundDesc, topk_idx: torch.Tensor, topk_val: torch.Tensor, stream=None):
         """Cloud half of the top-k split recovery: fills topk_idx [B, k] int32 and topk_val [B, k] float32."""

@@ -38,6 +38,10 @@ struct specsteer_ctx {
   bool host_ready;
   // optional timing hooks around the streaming kernel (caller-owned events)
   cudaEvent_t ev_stream_begin, ev_stream_end;
+  // fused LM-head path: records at 128 entries per chunk and the drafted tokens' logits (allocated on first use)
+  void* lm_ws;
+  float* lm_part;
+  float* lm_tok;
 };
 
 static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
@@ -240,6 +244,7 @@ specsteer_status specsteer_ctx_destroy(specsteer_ctx* ctx) {
     cudaStreamDestroy(ctx->copy_stream);
   }
   if (ctx->stage) cudaFree(ctx->stage);
+  if (ctx->lm_ws) cudaFree(ctx->lm_ws);
   if (ctx->ws) cudaFree(ctx->ws);
   delete ctx;
   return SPECSTEER_OK;
@@ -360,6 +365,68 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx* ctx, const specste
   int nl = 0;
   if (launch_recover(p, d->dtype, ctx->li, (cudaStream_t)cuda_stream, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += nl;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, void* cuda_stream) {
+  if (!ctx || !ld) return SPECSTEER_ERR_INVALID_ARG;
+  const specsteer_round_desc* d = &ld->round;
+  if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
+  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
+  if (ld->d_llm <= 0 || ld->d_slm <= 0) return SPECSTEER_ERR_INVALID_ARG;
+  if (ld->d_llm % 8 || ld->d_slm % 8) return SPECSTEER_ERR_UNSUPPORTED;   // rows of the operands must be 16-byte multiples
+  if (d->B > 0) {
+    if (!ld->x_llm || !ld->w_llm || !ld->x_slm_plus || !ld->w_slm_plus || !ld->x_slm_minus || !ld->w_slm_minus ||
+        !d->draft_len || !d->lambda || !d->beta || !d->temperature || !d->u_recover || !d->accept_len)
+      return SPECSTEER_ERR_INVALID_ARG;
+    if (d->K > 0 && (!d->draft_tokens || !d->u_accept)) return SPECSTEER_ERR_INVALID_ARG;
+    const void* ops[6] = {ld->x_llm, ld->w_llm, ld->x_slm_plus, ld->w_slm_plus, ld->x_slm_minus, ld->w_slm_minus};
+    for (const void* o : ops)
+      if ((uintptr_t)o & 15u) return SPECSTEER_ERR_UNSUPPORTED;
+  }
+  if (d->B > ctx->max_B || d->K > ctx->max_K || d->V > ctx->max_V) return SPECSTEER_ERR_UNSUPPORTED;
+  if ((size_t)(ld->d_llm + 2 * ld->d_slm) * 2 + (size_t)n_chunks_of(d->V, kLmheadChunk) * 8 + 64 > 200 * 1024)
+    return SPECSTEER_ERR_UNSUPPORTED;   // the recovery kernel keeps the row's hidden states and chunk weights in shared memory
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  ctx->verified = false;
+  ctx->shard_streamed = false;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  const int K1 = d->K + 1;
+  if (!ctx->lm_ws) {   // sized for the context's maxima, once
+    const size_t rows = (size_t)ctx->max_B * (ctx->max_K + 1);
+    const size_t part_bytes = align_up(rows * (size_t)n_chunks_of(ctx->max_V, kLmheadChunk) * 32, 256);
+    const size_t tok_bytes = align_up(rows * 16, 256);
+    if (cudaMalloc(&ctx->lm_ws, part_bytes + tok_bytes) != cudaSuccess) { ctx->lm_ws = nullptr; return SPECSTEER_ERR_WORKSPACE; }
+    ctx->lm_part = (float*)ctx->lm_ws;
+    ctx->lm_tok = (float*)((char*)ctx->lm_ws + part_bytes);
+    ctx->ws_bytes += part_bytes + tok_bytes;
+  }
+  specsteer_round_desc dd = *d;
+  dd.dtype = SPECSTEER_F32; dd.ld_row = d->V; dd.ld_req = (int64_t)K1 * d->V;   // no logit tensor exists
+  RoundParams p = slab_params(ctx, &dd, 0, d->B);
+  p.h_llm = p.h_plus = p.h_minus = nullptr;
+  p.sums = SUM_ALL;
+  p.row_mode = ROWS_ALL;
+  p.tile = kLmheadChunk;
+  p.n_chunks = n_chunks_of(d->V, kLmheadChunk);
+  p.part = ctx->lm_part;
+  p.tok_logits = ctx->lm_tok;
+  LmheadOperands op;
+  op.x_llm = (const uint16_t*)ld->x_llm; op.w_llm = (const uint16_t*)ld->w_llm;
+  op.x_plus = (const uint16_t*)ld->x_slm_plus; op.w_plus = (const uint16_t*)ld->w_slm_plus;
+  op.x_minus = (const uint16_t*)ld->x_slm_minus; op.w_minus = (const uint16_t*)ld->w_slm_minus;
+  op.d_llm = ld->d_llm; op.d_slm = ld->d_slm;
+  if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_lmhead(p, op, ctx->lm_tok, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_epilogue(p, SPECSTEER_F32, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_lmhead_recover(p, op, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 3;
   return SPECSTEER_OK;
 }
 

@@ -65,6 +65,17 @@ struct RoundParams {
   const ShardPartial* shard_parts;  // [n_shards][B][K+1] gathered partials
   int n_shards, shard_rank;
   int vocab_offset, vocab_total;    // this shard covers global ids [vocab_offset, vocab_offset + V)
+  // fused LM-head path: the logit tensors do not exist; the drafted tokens' logits were left here instead
+  const float* tok_logits;          // [B*(K+1)][4] {h_LLM, h_SLM+, h_SLM-, unused} of the row's drafted token, or null
+};
+
+// The LM heads in front of the round: h = x W^T, all operands bf16, row-major, dense.
+constexpr int kLmheadChunk = 128;   // vocabulary entries per partial record on that path (one tensor-core tile)
+struct LmheadOperands {
+  const uint16_t *x_llm, *w_llm;      // [B*(K+1)][d_llm], [V][d_llm]
+  const uint16_t *x_plus, *w_plus;    // [B*(K+1)][d_slm], [V][d_slm]
+  const uint16_t *x_minus, *w_minus;  // [B*(K+1)][d_slm], [V][d_slm]
+  int d_llm, d_slm;
 };
 
 struct LaunchInfo {
@@ -76,6 +87,11 @@ struct LaunchInfo {
 // ev_begin / ev_end, when not null, are recorded on `s` just before and just after the streaming kernel.
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
                           int* n_launches, cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
+// The tensor-core pass: partial records of every row at kLmheadChunk entries per chunk, and tok_logits.
+cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, const LaunchInfo& li,
+                          cudaStream_t s);
+// Recovery (Eq. 8) from those records; the logits of the one chunk that holds the CDF target are recomputed.
+cudaError_t launch_lmhead_recover(const RoundParams& p, const LmheadOperands& op, cudaStream_t s);
 constexpr int kTopkMaxSplit = 16;  // CTAs that may share one row in specsteer_cloud_topk
 // lists_ws: [B][kTopkMaxSplit][32] 64-bit keys; count_ws: [B] counters, zero between launches
 cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_idx, float* topk_val,

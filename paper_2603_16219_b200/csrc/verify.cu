@@ -445,7 +445,7 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
   float gl = 0.f, gp = 0.f, gm = 0.f;
   if (t < len) {
     y = p.draft_tokens[(long long)b * K + t];
-    if (p.n_shards == 0 && y >= 0 && y < p.V) {
+    if (p.n_shards == 0 && !p.tok_logits && y >= 0 && y < p.V) {
       const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
       gl = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
       gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
@@ -453,6 +453,10 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
     }
   }
   pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
+  if (p.tok_logits && y >= 0 && y < p.V) {  // fused LM-head path: the tensor-core pass left them in the workspace
+    const float4 g = ld_cg_f4(p.tok_logits + row * 4);
+    gl = g.x; gp = g.y; gm = g.z;
+  }
   float M[4];
   double S[4];
   if (p.n_shards > 0) {

@@ -151,6 +151,74 @@ def make_round(spec: RoundSpec, device="cpu", seed: int = 0) -> Dict[str, torch.
     }
 
 
+def make_lmhead_round(spec: RoundSpec, d_llm: int, d_slm: int, device="cpu", seed: int = 0) -> Dict[str, torch.Tensor]:
+    """Inputs of one round on hidden states and LM heads instead of logits (bf16), deterministic for
+    (spec, d_llm, d_slm, seed, device type); needs d_slm < d_llm.
+
+    The three logit tensors x W^T have the structure of ``make_round``'s: the Specialist's head is the first d_slm
+    columns of the Generalist's, the Generalist's hidden state is the Specialist's clean state s followed by extra
+    dimensions, and the Specialist's two states are s plus noise (twice as much with the context as without).  The
+    first hidden dimension is the constant 1 and carries a per-token bias with the Zipf profile over one random
+    permutation of the vocabulary.  Draft tokens are sampled from Softmax(h_SLM+ / T) formed with a float32 product.
+    """
+    dev = torch.device(device)
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(seed)
+    cgen = torch.Generator(device="cpu")
+    cgen.manual_seed(seed + 1)
+    B, K, V = spec.B, spec.K, spec.V
+    K1 = K + 1
+    if spec.beta_uniform is not None:
+        lo, hi = spec.beta_uniform
+        beta = lo + (hi - lo) * torch.rand(B, generator=cgen)
+    else:
+        beta = torch.tensor(spec.beta_choices)[torch.randint(len(spec.beta_choices), (B,), generator=cgen)]
+    temp = torch.tensor(spec.temp_choices)[torch.randint(len(spec.temp_choices), (B,), generator=cgen)]
+    lam = torch.full((B,), spec.lam)
+    if spec.ragged:
+        draft_len = torch.randint(1, K + 1, (B,), generator=cgen, dtype=torch.int32)
+    else:
+        draft_len = torch.full((B,), K, dtype=torch.int32)
+    u_accept = torch.rand(B, K, generator=cgen, dtype=torch.float32)
+    u_recover = torch.rand(B, generator=cgen, dtype=torch.float32)
+    sigma = _sigma_per_request(spec).to(dev)          # noise of h_SLM+ in logit units; h_SLM- gets half
+
+    # heads: entries N(0, g^2 / d_slm) on the shared columns, so that s W^T has standard deviation g for |s_i| ~ 1
+    w_llm = torch.randn(V, d_llm, generator=gen, device=dev) * (GAUSS_G / d_slm ** 0.5)
+    w_llm[:, d_slm:] *= 0.3 * (d_slm / max(1, d_llm - d_slm)) ** 0.5   # the extra dimensions add a tenth of the variance
+    rank = torch.argsort(torch.rand(V, generator=gen, device=dev)).to(torch.float32) + 1.0
+    w_llm[:, 0] = -ZIPF_S * torch.log(rank)
+    w_llm = w_llm.to(torch.bfloat16)
+    w_slm = w_llm[:, :d_slm].contiguous()
+    s = torch.randn(B, K1, d_slm, generator=gen, device=dev)
+    s[..., 0] = 1.0
+    extra = torch.randn(B, K1, d_llm - d_slm, generator=gen, device=dev)
+    x_llm = torch.cat([s, extra], dim=2).to(torch.bfloat16)
+    sg = (sigma / GAUSS_G)[:, None, None]
+    x_plus = s + sg * torch.randn(B, K1, d_slm, generator=gen, device=dev)
+    x_minus = s + 0.5 * sg * torch.randn(B, K1, d_slm, generator=gen, device=dev)
+    x_plus[..., 0] = 1.0
+    x_minus[..., 0] = 1.0
+    x_plus, x_minus = x_plus.to(torch.bfloat16), x_minus.to(torch.bfloat16)
+
+    draft = torch.zeros(B, K, dtype=torch.int32, device=dev)
+    wf = w_slm.to(torch.float32)
+    for b0 in range(0, B, 32):
+        b1 = min(B, b0 + 32)
+        hp = torch.matmul(x_plus[b0:b1, :K].to(torch.float32), wf.t())
+        q = torch.softmax(hp.to(torch.float64) / temp[b0:b1, None, None].to(dev).to(torch.float64), dim=2)
+        if K > 0:
+            draft[b0:b1] = torch.multinomial(q.view(-1, V), 1, generator=gen).view(b1 - b0, K).to(torch.int32)
+        del hp, q
+    return {
+        "x_llm": x_llm, "w_llm": w_llm, "x_slm_plus": x_plus, "w_slm_plus": w_slm, "x_slm_minus": x_minus,
+        "w_slm_minus": w_slm,
+        "draft_tokens": draft, "draft_len": draft_len.to(dev),
+        "lam": lam.to(dev), "beta": beta.to(torch.float32).to(dev), "temperature": temp.to(torch.float32).to(dev),
+        "u_accept": u_accept.to(dev), "u_recover": u_recover.to(dev),
+    }
+
+
 def used_rows(spec: RoundSpec, draft_len: torch.Tensor, bonus: bool) -> int:
     """Rows the round must read: the drafted rows plus, with the bonus flag, the row after them."""
     return int(draft_len.to(torch.int64).sum().item()) + (spec.B if bonus else 0)

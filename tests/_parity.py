@@ -21,12 +21,12 @@ def to_np_inputs(inputs, sel=None):
     return out
 
 
-def run_oracle(oracle, npin, accept_mode, recover_mode, flags, V=None, force=None, nthreads=8):
+def run_oracle(oracle, npin, accept_mode, recover_mode, flags, V=None, force=None, nthreads=8, margin=MARGIN):
     return oracle.verify_recover_round(
         npin["h_llm"], npin["h_slm_plus"], npin["h_slm_minus"], npin["draft_tokens"], npin["draft_len"],
         npin["lam"], npin["beta"], npin["temperature"], npin["u_accept"], npin["u_recover"],
         accept_mode=accept_mode, recover_mode=recover_mode, flags=flags, force_accept=force,
-        margin_tol=MARGIN, nthreads=nthreads, V=V)
+        margin_tol=margin, nthreads=nthreads, V=V)
 
 
 def run_gpu(ctx, inputs, accept_mode, recover_mode, flags, V=None):
@@ -42,10 +42,13 @@ def _slice(npin, b):
     return {k: v[b:b + 1] for k, v in npin.items()}
 
 
-def compare(oracle, gpu, npin, accept_mode, recover_mode, flags, tol, V=None, sel=None):
+def compare(oracle, gpu, npin, accept_mode, recover_mode, flags, tol, V=None, sel=None, margin=MARGIN):
     """Assert parity of GPU outputs (dict of numpy, all requests) with the oracle on the requests `sel`
-    (indices into the GPU batch; npin holds exactly those requests, in order).  Returns statistics."""
-    ora = run_oracle(oracle, npin, accept_mode, recover_mode, flags, V=V)
+    (indices into the GPU batch; npin holds exactly those requests, in order).  Returns statistics.
+    `margin` is the width below which a decision may differ (then it is forced in the oracle and the rest
+    of the request is compared on that branch)."""
+    MARGIN = margin
+    ora = run_oracle(oracle, npin, accept_mode, recover_mode, flags, V=V, margin=margin)
     B = npin["draft_len"].shape[0]
     K = npin["draft_tokens"].shape[1]
     sel = np.arange(B) if sel is None else np.asarray(sel)
@@ -68,7 +71,8 @@ def compare(oracle, gpu, npin, accept_mode, recover_mode, flags, tol, V=None, se
                 force = np.full((1, K), -1, np.int8)
             force[0, t] = int(g["accept_flags"][b][t])
             stats["excused_accept"] += 1
-            one = run_oracle(oracle, _slice(npin, b), accept_mode, recover_mode, flags, V=V, force=force, nthreads=1)
+            one = run_oracle(oracle, _slice(npin, b), accept_mode, recover_mode, flags, V=V, force=force, nthreads=1,
+                             margin=margin)
             ob = {k: v[0] for k, v in one.items()}
         assert g["accept_len"][b] == ob["accept_len"]
         assert g["req_status"][b] == ob["req_status"], (b, g["req_status"][b], ob["req_status"])
