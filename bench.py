@@ -25,6 +25,7 @@ if ROOT not in sys.path:
 METRIC = "verified_draft_positions_per_sec"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0   # sustained, under the power cap
 N_SM = 148
 EX2_PER_CLK_PER_SM = 16
 NOMINAL_HBM_GBS = 8000.0
@@ -425,6 +426,119 @@ def run_cuda(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def _tensor_peak():
+    """Measured dense bf16 throughput (TFLOP/s): the sustained figure, since the kernel runs inside a long step."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            d = json.load(f)
+        return float(d.get("bf16_tflops_sustained") or d["bf16_tflops"]), "measured (sustained)"
+    except Exception:
+        return FALLBACK_BF16_TFLOPS, "fallback"
+
+
+def run_lmhead(args, local_rank):
+    """The round with the LM heads fused in front (1 GPU): the hidden states and head weights of the benchmark
+    shape go in, no logit is stored.  Beside it, the same work unfused: three library products into float32 logit
+    tensors followed by the streaming round.  One short JSON line."""
+    import dataclasses
+    import torch
+    from paper_2603_16219_b200 import binding, build, synth
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    build.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    spec = synth.CONFIGS[args.config]
+    if args.requests:
+        spec = dataclasses.replace(spec, B=args.requests, name="%s_first%d" % (spec.name, args.requests))
+    dL, dS = args.d_llm, args.d_slm
+    inputs = synth.make_lmhead_round(spec, dL, dS, device=dev, seed=0)
+    B, K, V = spec.B, spec.K, spec.V
+    rows = B * (K + 1)
+    positions = int(inputs["draft_len"].sum().item())
+    ctx = binding.Context(B, K, V, device=local_rank)
+    outs = binding.alloc_outputs(B, K, dev)
+    desc = binding.make_lmhead_desc(inputs, outs, flags=binding.FLAG_BONUS)
+    stream = torch.cuda.current_stream(dev)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    steps = min(args.steps, 50)
+    for _ in range(max(3, min(args.warmup, 5))):
+        ctx.lmhead_round(desc, stream)
+    torch.cuda.synchronize(dev)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(min(steps, 16))]
+    for a, b in evs:
+        a.record(stream)
+        b.record(stream)
+    stride = max(1, steps // len(evs))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = ctx.launch_count
+    torch.cuda.synchronize(dev)
+    w0 = time.perf_counter()
+    e0.record(stream)
+    used = 0
+    for i in range(steps):
+        if i % stride == 0 and used < len(evs):
+            ctx.time_streaming(*evs[used])
+            ctx.lmhead_round(desc, stream)
+            ctx.time_streaming(None, None)
+            used += 1
+        else:
+            ctx.lmhead_round(desc, stream)
+    e1.record(stream)
+    torch.cuda.synchronize(dev)
+    w1 = time.perf_counter()
+    sampler.window(w0, w1)
+    assert ctx.device_error() == 0
+    fused_ms = e0.elapsed_time(e1) / steps
+    kernel_ms = sum(a.elapsed_time(b) for a, b in evs[:used]) / used
+    gpu_launches = ctx.launch_count - launches0
+    fused_out = {k: v.clone() for k, v in outs.items()}
+
+    # ---- the same work unfused: library products into float32 logits, then the streaming round
+    h = {n: torch.empty(B, K + 1, V, dtype=torch.float32, device=dev) for n in ("h_llm", "h_slm_plus", "h_slm_minus")}
+    li = {k: inputs[k] for k in ("draft_tokens", "draft_len", "lam", "beta", "temperature", "u_accept", "u_recover")}
+    li.update(h)
+    d2 = binding.make_desc(li, outs, flags=binding.FLAG_BONUS)
+    pairs = (("h_llm", "x_llm", "w_llm"), ("h_slm_plus", "x_slm_plus", "w_slm_plus"), ("h_slm_minus", "x_slm_minus", "w_slm_minus"))
+
+    def unfused():
+        for hn, xn, wn in pairs:
+            h[hn].view(rows, V).copy_(torch.matmul(inputs[xn].view(rows, -1), inputs[wn].t()))
+        ctx.verify_round(d2, stream)
+        ctx.recover_sample(d2, stream)
+
+    for _ in range(3):
+        unfused()
+    torch.cuda.synchronize(dev)
+    u0, u1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_un = min(steps, 20)
+    u0.record(stream)
+    for _ in range(n_un):
+        unfused()
+    u1.record(stream)
+    torch.cuda.synchronize(dev)
+    unfused_ms = u0.elapsed_time(u1) / n_un
+    same = float(((fused_out["accept_len"] == outs["accept_len"]) & (fused_out["rec_token"] == outs["rec_token"])).float().mean().item())
+    sampler.stop()
+    peak, peak_kind = _tensor_peak()
+    flops = 2.0 * rows * V * (dL + 2 * dS)
+    achieved = flops / (kernel_ms * 1e-3) / 1e12
+    line = {
+        "workload": "%s_lmhead_dllm%d_dslm%d" % (spec.name, dL, dS), "metric": METRIC,
+        "value": positions / (fused_ms * 1e-3), "unit": UNIT, "ms_per_step": fused_ms, "steps": steps, "dtype": "bf16",
+        "roofline": {"bound": "tensor", "kernel": "lmhead_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                     "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": None,
+                     "algorithmic_flops_per_launch": flops, "kernel_ms": kernel_ms},
+        "unfused": {"ms_per_step": unfused_ms, "what": "three torch.matmul (library GEMM) products from the same bf16 operands, "
+                    "copied into float32 logit tensors (bf16 product rounded once), then verify_round + recover_sample",
+                    "requests_with_same_accept_len_and_token": same},
+        "logit_bytes_never_stored": 3 * rows * V * 4,
+        "gpu_launches": int(gpu_launches), "clocks": sampler.summary(),
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -439,6 +553,10 @@ def main():
                     help="with --kernels-only: also time the top-k split recovery (cloud + edge kernels) with this k")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the device-resident steps and print a short line (profiling aid)")
+    ap.add_argument("--lmhead", action="store_true",
+                    help="time the round with the LM heads fused in front (hidden states and head weights in, 1 GPU)")
+    ap.add_argument("--d-llm", type=int, default=5120, help="with --lmhead: hidden width of the Generalist")
+    ap.add_argument("--d-slm", type=int, default=2048, help="with --lmhead: hidden width of the Specialist")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -451,6 +569,9 @@ def main():
         sys.exit(subprocess.call(cmd))
     if args.impl == "reference":
         run_reference(args, rank, world)
+    elif args.lmhead:
+        if rank == 0:
+            run_lmhead(args, local_rank)
     else:
         run_cuda(args, rank, world, local_rank)
 

@@ -188,3 +188,40 @@ def test_agrees_with_the_streaming_round_on_materialised_logits(env):
     assert same.mean() > 0.9
     ok = same[:, None] & np.isfinite(streamed["logp_llm"])
     assert np.abs(fused["logp_llm"][ok] - streamed["logp_llm"][ok]).max() < TOL
+
+
+def test_full_size_sampled_requests():
+    """The benchmark shape (256 requests, K = 4, V = 151936, hidden widths 5120 and 2048) in the launch the bench
+    times; 6 requests spread over the batch are checked against the oracle, whose logits are formed 16384
+    vocabulary entries at a time (each logit is still one float64 dot product)."""
+    import oracle as o
+    from paper_2603_16219_b200 import binding as b, build, synth
+    o.build()
+    build.build()
+    spec = synth.CONFIGS[3]
+    inputs = synth.make_lmhead_round(spec, 5120, 2048, device="cuda", seed=0)
+    ctx = b.Context(spec.B, spec.K, spec.V, device=0)
+    try:
+        outs = b.alloc_outputs(spec.B, spec.K, "cuda")
+        desc = b.make_lmhead_desc(inputs, outs, flags=1)
+        ctx.lmhead_round(desc)
+        torch.cuda.synchronize()
+        assert ctx.device_error() == 0
+        gpu = {k: v.cpu().numpy() for k, v in outs.items()}
+    finally:
+        ctx.close()
+    P.invariants(gpu, {"draft_tokens": inputs["draft_tokens"], "draft_len": inputs["draft_len"]}, 1, TOL)
+    sel = np.linspace(0, spec.B - 1, 6).astype(int)
+    selt = torch.as_tensor(sel, device="cuda")
+
+    def logits(xn, wn):
+        x = _bits(inputs[xn][selt])
+        w = _bits(inputs[wn])
+        return np.concatenate([o.lmhead_logits(x, w[v0:v0 + 16384]) for v0 in range(0, spec.V, 16384)], axis=2)
+
+    npin = {"h_llm": logits("x_llm", "w_llm"), "h_slm_plus": logits("x_slm_plus", "w_slm_plus"),
+            "h_slm_minus": logits("x_slm_minus", "w_slm_minus")}
+    for k in ("draft_tokens", "draft_len", "lam", "beta", "temperature", "u_accept", "u_recover"):
+        npin[k] = inputs[k][selt].cpu().numpy()
+    stats = P.compare(o, gpu, npin, 0, 0, 1, TOL, sel=sel, margin=MARGIN)
+    assert stats["requests"] == 6
