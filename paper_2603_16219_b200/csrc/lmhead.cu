@@ -24,15 +24,19 @@ constexpr int kBM = kLmheadChunk;  // rows of hidden states per tile = lanes of 
 constexpr int kBN = kLmheadChunk;  // vocabulary entries per tile = one partial record
 constexpr int kBK = 64;            // hidden entries per stage: 128 bytes of bf16, one swizzle row
 constexpr int kUmmaK = 16;         // hidden entries per tcgen05.mma of kind::f16
-constexpr int kStages = 6;
 constexpr int kTileBytes = kBM * kBK * 2;   // 16 KB, one operand tile
-constexpr int kStageBytes = 2 * kTileBytes;
+// The operand ring is made of groups of four tiles.  A group holds either two steps of one product ({x, W} twice) or
+// one step of both Specialist products when they share a head ({x+, x-, W}).  Each step has its own "full" barrier,
+// the group one "empty" barrier: one tcgen05.commit per group (a commit costs about as much as an MMA).
+constexpr int kGroups = 3;
+constexpr int kGroupBytes = 4 * kTileBytes;
 constexpr int kThreads = 192;
 constexpr uint32_t kTmemCols = 512;         // 4 accumulators of 128 columns: {L even, P, M, L odd}
-constexpr int kSmemBytes = kStages * kStageBytes + 1024 /* alignment */ + 256 /* barriers */;
+constexpr int kSmemBytes = kGroups * kGroupBytes + 1024 /* alignment */ + 512 /* barriers */;
 
 struct LmKernelParams {
   int R, V, K, d_llm, d_slm, n_chunks;
+  int shared_head;    // h_SLM+ and h_SLM- use the same head: its tile is loaded once for both products
   const int* draft_tokens;
   const int* draft_len;
   const float* beta;
@@ -100,7 +104,7 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
 constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
 
 struct LmShared {
-  uint64_t full[kStages], empty[kStages];
+  uint64_t full[kGroups][2], empty[kGroups];
   uint64_t tmem_full, tmem_empty, drain;
   uint32_t tmem_slot;
   int abort_flag;
@@ -158,14 +162,14 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
               const __grid_constant__ CUtensorMap tm_xm, const __grid_constant__ CUtensorMap tm_wm, const LmKernelParams p) {
   extern __shared__ unsigned char smem_raw[];
   const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // operand tiles need 1024-byte alignment
-  LmShared* sh = reinterpret_cast<LmShared*>(smem_raw + (smem0 - smem_u32(smem_raw)) + kStages * kStageBytes);
+  LmShared* sh = reinterpret_cast<LmShared*>(smem_raw + (smem0 - smem_u32(smem_raw)) + kGroups * kGroupBytes);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int mb_count = (p.R + kBM - 1) / kBM, nb_count = (p.V + kBN - 1) / kBN;
   const int n_tiles = mb_count * nb_count;
   const int nkL = (p.d_llm + kBK - 1) / kBK, nkS = (p.d_slm + kBK - 1) / kBK;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+    for (int s = 0; s < kGroups; ++s) { mbar_init(&sh->full[s][0], 1); mbar_init(&sh->full[s][1], 1); mbar_init(&sh->empty[s], 1); }
     mbar_init(&sh->tmem_full, 1);
     mbar_init(&sh->tmem_empty, 4);
     mbar_init(&sh->drain, 1);
@@ -181,57 +185,109 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
   if (warp == 0) {
     // ================= TMA producer =================
     if (lane == 0) {
-      int it = 0;
+      int grp = 0;  // groups issued so far: group i lives in slot i % kGroups
       bool ok = true;
+      uint32_t base = 0;
+      int gs = 0;
+      auto begin_group = [&]() {
+        gs = grp % kGroups;
+        const uint32_t ph = (uint32_t)((grp / kGroups) & 1);
+        if (aborted(sh) || !mbar_wait(&sh->empty[gs], ph ^ 1u)) { set_abort(sh, p.dev_error); ok = false; return; }
+        base = smem0 + gs * kGroupBytes;
+        ++grp;
+      };
+      // two steps of x W^T (the second one missing at an odd end): tiles {x, W, x, W}
+      auto pair_steps = [&](const CUtensorMap* ta, const CUtensorMap* tb, int m0, int n0, int nk) {
+        for (int kb = 0; kb < nk && ok; kb += 2) {
+          begin_group();
+          if (!ok) break;
+#pragma unroll
+          for (int j = 0; j < 2; ++j) {
+            if (kb + j < nk) {
+              mbar_arrive_expect_tx(&sh->full[gs][j], 2 * kTileBytes);
+              tma_load_2d(base + j * 2 * kTileBytes, ta, (kb + j) * kBK, m0, &sh->full[gs][j]);
+              tma_load_2d(base + j * 2 * kTileBytes + kTileBytes, tb, (kb + j) * kBK, n0, &sh->full[gs][j]);
+            } else {
+              mbar_arrive(&sh->full[gs][j]);  // unused this time: keep its phase in step with the group's
+            }
+          }
+        }
+      };
       for (int g = blockIdx.x; g < n_tiles && ok; g += gridDim.x) {
         const int mb = g % mb_count, nb = g / mb_count;  // row blocks fastest: CTAs running together share W tiles in L2
-        for (int seg = 0; seg < 3 && ok; ++seg) {
-          const CUtensorMap* ta = seg == 0 ? &tm_xl : (seg == 1 ? &tm_xp : &tm_xm);
-          const CUtensorMap* tb = seg == 0 ? &tm_wl : (seg == 1 ? &tm_wp : &tm_wm);
-          const int nk = seg == 0 ? nkL : nkS;
-          for (int kb = 0; kb < nk; ++kb, ++it) {
-            const int s = it % kStages;
-            const uint32_t ph = (uint32_t)((it / kStages) & 1);
-            if (aborted(sh) || !mbar_wait(&sh->empty[s], ph ^ 1u)) { set_abort(sh, p.dev_error); ok = false; break; }
-            const uint32_t a = smem0 + s * kStageBytes;
-            mbar_arrive_expect_tx(&sh->full[s], kStageBytes);
-            tma_load_2d(a, ta, kb * kBK, mb * kBM, &sh->full[s]);
-            tma_load_2d(a + kTileBytes, tb, kb * kBK, nb * kBN, &sh->full[s]);
+        const int m0 = mb * kBM, n0 = nb * kBN;
+        pair_steps(&tm_xl, &tm_wl, m0, n0, nkL);
+        if (p.shared_head) {
+          for (int kb = 0; kb < nkS && ok; ++kb) {   // one step of both products: tiles {x+, x-, W}
+            begin_group();
+            if (!ok) break;
+            mbar_arrive_expect_tx(&sh->full[gs][0], 3 * kTileBytes);
+            tma_load_2d(base, &tm_xp, kb * kBK, m0, &sh->full[gs][0]);
+            tma_load_2d(base + kTileBytes, &tm_xm, kb * kBK, m0, &sh->full[gs][0]);
+            tma_load_2d(base + 2 * kTileBytes, &tm_wp, kb * kBK, n0, &sh->full[gs][0]);
+            mbar_arrive(&sh->full[gs][1]);
           }
+        } else {
+          pair_steps(&tm_xp, &tm_wp, m0, n0, nkS);
+          pair_steps(&tm_xm, &tm_wm, m0, n0, nkS);
         }
       }
       if (!ok) {  // copies already issued may still be landing: wait for them (bounded) before the CTA exits
-        for (int i = it > kStages ? it - kStages : 0; i < it; ++i)
-          mbar_wait(&sh->full[i % kStages], (uint32_t)((i / kStages) & 1));
+        for (int i = grp > kGroups ? grp - kGroups : 0; i < grp; ++i) {
+          mbar_wait(&sh->full[i % kGroups][0], (uint32_t)((i / kGroups) & 1));
+          mbar_wait(&sh->full[i % kGroups][1], (uint32_t)((i / kGroups) & 1));
+        }
       }
     }
   } else if (warp == 1) {
     // ================= tensor-core issuer =================
     if (lane == 0) {
-      int it = 0, ti = 0;
+      int grp = 0, ti = 0;
       bool ok = true;
-      for (int g = blockIdx.x; g < n_tiles && ok; g += gridDim.x, ++ti) {
-        for (int seg = 0; seg < 3 && ok; ++seg) {
-          // h_LLM alternates between two accumulators, so its long K loop of the next tile runs while the
-          // epilogue drains this one; h_SLM+ and h_SLM- wait for the epilogue of the tile before
-          const uint32_t col = seg == 0 ? ((ti & 1) ? 384u : 0u) : (seg == 1 ? 128u : 256u);
-          if (seg == 1 && ti > 0) {
-            if (aborted(sh) || !mbar_wait(&sh->tmem_empty, (uint32_t)((ti - 1) & 1))) { set_abort(sh, p.dev_error); ok = false; break; }
-            tc_fence_after();
-          }
-          const int nk = seg == 0 ? nkL : nkS;
-          for (int kb = 0; kb < nk; ++kb, ++it) {
-            const int s = it % kStages;
-            const uint32_t ph = (uint32_t)((it / kStages) & 1);
-            if (aborted(sh) || !mbar_wait(&sh->full[s], ph)) { set_abort(sh, p.dev_error); ok = false; break; }
-            tc_fence_after();
-            const uint32_t a = smem0 + s * kStageBytes;
-            const uint64_t ad = smem_desc_sw128(a), bd = smem_desc_sw128(a + kTileBytes);
+      // one step of 64 hidden entries: four tcgen05.mma, 32 bytes further along the swizzled row each
+      auto product = [&](uint32_t col, uint32_t a, uint32_t b, int kb) {
+        const uint64_t ad = smem_desc_sw128(a), bd = smem_desc_sw128(b);
 #pragma unroll
-            for (int k = 0; k < kBK / kUmmaK; ++k)  // 32 bytes further along the swizzled row per step
-              umma_bf16(tmem_base + col, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), kIdesc, (kb | k) != 0);
-            umma_commit(&sh->empty[s]);  // the stage is free once these have read it
+        for (int k = 0; k < kBK / kUmmaK; ++k)
+          umma_bf16(tmem_base + col, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), kIdesc, (kb | k) != 0);
+      };
+      auto landed = [&](int gs, int j, uint32_t ph) {
+        if (aborted(sh) || !mbar_wait(&sh->full[gs][j], ph)) { set_abort(sh, p.dev_error); ok = false; return; }
+        tc_fence_after();
+      };
+      auto pair_steps = [&](uint32_t col, int nk) {
+        for (int kb = 0; kb < nk && ok; kb += 2, ++grp) {
+          const int gs = grp % kGroups;
+          const uint32_t ph = (uint32_t)((grp / kGroups) & 1);
+          const uint32_t base = smem0 + gs * kGroupBytes;
+          for (int j = 0; j < 2 && kb + j < nk && ok; ++j) {
+            landed(gs, j, ph);
+            if (ok) product(col, base + j * 2 * kTileBytes, base + j * 2 * kTileBytes + kTileBytes, kb + j);
           }
+          if (ok) umma_commit(&sh->empty[gs]);  // the group is free once these have read it
+        }
+      };
+      for (int g = blockIdx.x; g < n_tiles && ok; g += gridDim.x, ++ti) {
+        // h_LLM alternates between two accumulators, so its long K loop of the next tile runs while the
+        // epilogue drains this one; h_SLM+ and h_SLM- wait for the epilogue of the tile before
+        pair_steps((ti & 1) ? 384u : 0u, nkL);
+        if (ok && ti > 0) {
+          if (aborted(sh) || !mbar_wait(&sh->tmem_empty, (uint32_t)((ti - 1) & 1))) { set_abort(sh, p.dev_error); ok = false; }
+          tc_fence_after();
+        }
+        if (p.shared_head) {
+          for (int kb = 0; kb < nkS && ok; ++kb, ++grp) {
+            const int gs = grp % kGroups;
+            const uint32_t base = smem0 + gs * kGroupBytes;
+            landed(gs, 0, (uint32_t)((grp / kGroups) & 1));
+            if (!ok) break;
+            product(128u, base, base + 2 * kTileBytes, kb);
+            product(256u, base + kTileBytes, base + 2 * kTileBytes, kb);
+            umma_commit(&sh->empty[gs]);
+          }
+        } else {
+          pair_steps(128u, nkS);
+          pair_steps(256u, nkS);
         }
         if (ok) umma_commit(&sh->tmem_full);
       }
@@ -352,6 +408,7 @@ __device__ __forceinline__ double block_excl_scan256(double v, double* warp_tot,
 // dot product of a hidden state held in shared memory with one row of the head, 8 entries per lane and step
 __device__ __forceinline__ float warp_dot_bf16(const uint16_t* x_sh, const uint16_t* w_row, int d, int lane) {
   float acc = 0.f;
+#pragma unroll 4
   for (int i = lane * 8; i < d; i += 256) {  // d is a multiple of 8
     const uint4 wv = __ldg(reinterpret_cast<const uint4*>(w_row + i));
     const uint4 xv = *reinterpret_cast<const uint4*>(x_sh + i);
@@ -523,6 +580,7 @@ cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float*
   k.R = R; k.V = p.V; k.K = p.K; k.d_llm = op.d_llm; k.d_slm = op.d_slm; k.n_chunks = p.n_chunks;
   k.draft_tokens = p.draft_tokens; k.draft_len = p.draft_len; k.beta = p.beta; k.temperature = p.temperature;
   k.part = p.part; k.tok_logits = tok_logits; k.dev_error = p.dev_error;
+  k.shared_head = (op.w_plus == op.w_minus) ? 1 : 0;
   static bool attr_set[64] = {};
   if (li.device < 64 && !attr_set[li.device]) {
     cudaError_t e = cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
