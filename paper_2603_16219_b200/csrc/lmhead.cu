@@ -382,14 +382,14 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
 }
 
 // ---- recovery ------------------------------------------------------------------------------------------
-constexpr int kRecT = 256;
+constexpr int kRecT = 1024;  // 32 warps: recomputing the chunk is a chain of dependent loads per warp, so many warps
 struct LmRecShared {
   double warp_tot[kRecT / 32];
   double base, target, W;
   int jstar, jlast, tok_min, tok_last;
 };
 
-__device__ __forceinline__ double block_excl_scan256(double v, double* warp_tot, int tid) {
+__device__ __forceinline__ double block_excl_scan_rec(double v, double* warp_tot, int tid) {
   const int lane = tid & 31, warp = tid >> 5;
   double inc = v;
 #pragma unroll
@@ -471,7 +471,7 @@ __global__ void __launch_bounds__(kRecT) lmhead_recover_kernel(const RoundParams
   const int j0 = min(tid * per, p.n_chunks), j1 = min(j0 + per, p.n_chunks);
   double local = 0.0;
   for (int j = j0; j < j1; ++j) local += cw[j];
-  const double excl = block_excl_scan256(local, sh.warp_tot, tid);
+  const double excl = block_excl_scan_rec(local, sh.warp_tot, tid);
   if (tid == kRecT - 1) { sh.W = excl + local; sh.target = (double)p.u_recover[b] * (excl + local); }
   __syncthreads();
   const double target = sh.target;
@@ -515,7 +515,7 @@ __global__ void __launch_bounds__(kRecT) lmhead_recover_kernel(const RoundParams
     y2 = ((double)lg[0][tid] + beta * ((double)lg[1][tid] - (double)lg[2][tid])) * cd - lseR;  // log2 Softmax(h_rec)(v)
     w = exp2(y2);
   }
-  const double before = block_excl_scan256(w, sh.warp_tot, tid);
+  const double before = block_excl_scan_rec(w, sh.warp_tot, tid);
   if (tid < kBN && w > 0.0) {
     atomicMax(&sh.tok_last, v);
     if (sh.base + before + w > sh.target) atomicMin(&sh.tok_min, v);
