@@ -86,3 +86,37 @@ def test_product_has_no_cpu_fallback_and_never_imports_the_oracle():
             if f.endswith((".py", ".cu", ".cuh", ".h")):
                 txt = open(os.path.join(dirpath, f)).read()
                 assert "oracle" not in txt.replace("the CPU oracle", ""), f
+
+
+def test_lmhead_descriptor_marshalling_rejects_bad_operands():
+    """Host-side checks of the LM-head descriptor builder (no GPU: only shapes, dtypes and pointers are looked at)."""
+    import torch
+    from paper_2603_16219_b200 import binding as b
+    B, K, V, dL, dS = 2, 3, 40, 16, 8
+    bf = torch.bfloat16
+    inputs = {
+        "x_llm": torch.zeros(B, K + 1, dL, dtype=bf), "w_llm": torch.zeros(V, dL, dtype=bf),
+        "x_slm_plus": torch.zeros(B, K + 1, dS, dtype=bf), "w_slm_plus": torch.zeros(V, dS, dtype=bf),
+        "x_slm_minus": torch.zeros(B, K + 1, dS, dtype=bf), "w_slm_minus": torch.zeros(V, dS, dtype=bf),
+        "draft_tokens": torch.zeros(B, K, dtype=torch.int32), "draft_len": torch.zeros(B, dtype=torch.int32),
+        "lam": torch.ones(B), "beta": torch.ones(B), "temperature": torch.ones(B),
+        "u_accept": torch.zeros(B, K), "u_recover": torch.zeros(B),
+    }
+    outs = b.alloc_outputs(B, K, "cpu")
+    d = b.make_lmhead_desc(inputs, outs, flags=b.FLAG_BONUS)
+    assert (d.round.B, d.round.K, d.round.V, d.d_llm, d.d_slm) == (B, K, V, dL, dS)
+    assert d.x_llm == inputs["x_llm"].data_ptr() and d.w_slm_minus == inputs["w_slm_minus"].data_ptr()
+    assert d.round.accept_len == outs["accept_len"].data_ptr() and d.round.flags == b.FLAG_BONUS
+    import pytest
+    for key, bad in (("w_llm", torch.zeros(V, dL)),                       # float32 head
+                     ("x_slm_plus", torch.zeros(B, K + 1, dS + 8, dtype=bf)),  # width differs from its head
+                     ("w_slm_minus", torch.zeros(V + 1, dS, dtype=bf)),        # vocabulary differs
+                     ("x_llm", torch.zeros(B, K + 1, 2 * dL, dtype=bf)[..., ::2])):  # not contiguous
+        broken = dict(inputs)
+        broken[key] = bad
+        with pytest.raises(ValueError):
+            b.make_lmhead_desc(broken, outs)
+    broken = dict(inputs)
+    broken["beta"] = torch.ones(B + 1)
+    with pytest.raises(ValueError):
+        b.make_lmhead_desc(broken, outs)

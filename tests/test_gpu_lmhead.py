@@ -225,3 +225,45 @@ def test_full_size_sampled_requests():
         npin[k] = inputs[k][selt].cpu().numpy()
     stats = P.compare(o, gpu, npin, 0, 0, 1, TOL, sel=sel, margin=MARGIN)
     assert stats["requests"] == 6
+
+
+def test_no_drafts_at_all_and_empty_batch(env):
+    """K = 0: every request has its bonus row only (Eq. 8 with nothing to verify); B = 0: nothing is launched."""
+    b = env["binding"]
+    _, gpu, _ = _case(env, _spec(env, 0, B=9, K=0, V=1500), 128, 64, seed=11)
+    assert (gpu["accept_len"] == 0).all() and (gpu["n_out"] == 1).all()
+    inputs = env["synth"].make_lmhead_round(_spec(env, 0, B=3, K=2, V=700), 128, 64, device="cuda", seed=12)
+    empty = {k: (v[:0].contiguous() if k.startswith("x_") or not k.startswith("w_") else v) for k, v in inputs.items()}
+    outs = b.alloc_outputs(0, 2, "cuda")
+    before = env["ctx"].launch_count
+    env["ctx"].lmhead_round(b.make_lmhead_desc(empty, outs))
+    assert env["ctx"].launch_count == before
+
+
+def test_bad_parameters_are_reported_per_request(env):
+    def mutate(inputs):
+        inputs["temperature"][1] = 0.0
+        inputs["lam"][3] = -1.0
+        inputs["beta"][4] = float("nan")
+    inputs = env["synth"].make_lmhead_round(_spec(env, 0, B=6, K=3, V=2000), 128, 64, device="cuda", seed=13)
+    mutate(inputs)
+    gpu = _run_gpu(env, inputs)
+    for r in (1, 3, 4):
+        assert gpu["req_status"][r] & 16 and gpu["accept_len"][r] == 0 and gpu["rec_token"][r] == -1
+    ok = [0, 2, 5]
+    npin = _np_inputs(env["oracle"], inputs, sel=torch.as_tensor(ok, device="cuda"))
+    P.compare(env["oracle"], gpu, npin, 0, 0, 1, TOL, sel=ok, margin=MARGIN)
+
+
+def test_one_context_serves_both_paths_and_changing_shapes(env):
+    """The fused path has its own workspace: a streaming round in between must not disturb it, and shapes may change
+    from call to call."""
+    b = env["binding"]
+    lm = env["synth"].make_lmhead_round(_spec(env, 0, B=10, K=3, V=3000), 192, 64, device="cuda", seed=14)
+    first = _run_gpu(env, lm)
+    st = env["synth"].make_round(_spec(env, 0, B=4, K=2, V=5000), device="cuda", seed=1)
+    P.run_gpu(env["ctx"], st, 0, 0, 1)
+    _case(env, _spec(env, 1, B=3, K=5, V=9000), 128, 128, seed=15)
+    again = _run_gpu(env, lm)
+    for k in first:
+        assert np.array_equal(first[k], again[k], equal_nan=True), k
