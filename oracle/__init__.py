@@ -25,7 +25,7 @@ _LIB = os.path.join(_HERE, "libspecsteer_oracle.so")
 
 DTYPE_F32, DTYPE_BF16, DTYPE_F64 = 0, 1, 2
 ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
-RECOVER_STEER, RECOVER_RESIDUAL = 0, 1
+RECOVER_STEER, RECOVER_RESIDUAL, RECOVER_ARGMAX = 0, 1, 2
 FLAG_BONUS = 1
 REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1, 2, 4, 8, 16
 

@@ -13,7 +13,8 @@ extern "C" {
 
 enum { ORACLE_DTYPE_F32 = 0, ORACLE_DTYPE_BF16 = 1, ORACLE_DTYPE_F64 = 2 };
 enum { ORACLE_ACCEPT_RATIO = 0 /* Eq. 7 */, ORACLE_ACCEPT_EXACT_Z = 1 /* Eq. 6 */ };
-enum { ORACLE_RECOVER_STEER = 0 /* Eq. 8 softmax */, ORACLE_RECOVER_RESIDUAL = 1 };
+enum { ORACLE_RECOVER_STEER = 0 /* Eq. 8 softmax */, ORACLE_RECOVER_RESIDUAL = 1,
+       ORACLE_RECOVER_ARGMAX = 2 /* greedy decoding: the token of largest h_rec (Eq. 8) */ };
 enum { ORACLE_FLAG_BONUS = 1u };
 enum {
   ORACLE_REQ_BAD_TOKEN = 1, ORACLE_REQ_BAD_LEN = 2, ORACLE_REQ_NONFINITE = 4,

@@ -343,3 +343,90 @@ def test_forced_decisions_and_margins(oracle_mod):
     forced = _round(oracle_mod, L, P, M, tok, u, np.array([0.9], np.float32), lam=1.0,
                     force_accept=np.array([[1, -1]], np.int8))
     assert forced["accept_len"][0] == 2
+
+
+# ---------------------------------------------------------------- greedy recovery (the paper decodes greedily)
+def _grid_rows(rng, B, K, V, q=4, lo=-8, hi=8):
+    """Rows on a grid of 1/q: every h_rec with beta in {0, 0.5, 1, 2} is exact in float32, ties are frequent."""
+    f = lambda: (rng.integers(lo * q, hi * q, size=(B, K + 1, V)) / q).astype(np.float32)
+    return f(), f(), f()
+
+
+@pytest.mark.parametrize("beta", [0.0, 0.5, 1.0, 2.0])
+def test_argmax_recovery_is_the_first_maximiser_of_h_rec(oracle_mod, beta):
+    """Eq. 8 under greedy decoding, by exhaustive search with exact rationals (lowest id among equals); the accept
+    decisions are those of the sampling round."""
+    from fractions import Fraction
+    o = oracle_mod
+    rng = np.random.default_rng(40)
+    B, K, V = 6, 3, 23
+    L, P, M = _grid_rows(rng, B, K, V)
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    ua, ur = rng.random((B, K)).astype(np.float32), rng.random(B).astype(np.float32)
+    g = _round(o, L, P, M, tok, ua, ur, beta=beta, recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
+    s = _round(o, L, P, M, tok, ua, ur, beta=beta, recover_mode=o.RECOVER_STEER, flags=o.FLAG_BONUS)
+    for k in ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "log_z", "req_status"):
+        assert np.array_equal(g[k], s[k], equal_nan=True), k
+    for b in range(B):
+        n = int(g["accept_len"][b])
+        h = [Fraction(float(L[b, n, v])) + Fraction(beta) * (Fraction(float(P[b, n, v])) - Fraction(float(M[b, n, v])))
+             for v in range(V)]
+        want = min(range(V), key=lambda v: (-h[v], v))
+        assert g["rec_token"][b] == want and g["n_out"][b] == n + 1
+        assert g["out_tokens"][b][n] == want and (g["out_tokens"][b][:n] == tok[b][:n]).all()
+        hr = np.array([float(x) for x in h])
+        assert g["rec_logprob"][b] == pytest.approx(sps.log_softmax(hr)[want], abs=1e-12)
+        assert np.isinf(g["cdf_margin"][b])
+
+
+def test_argmax_recovery_with_beta_zero_is_numpy_argmax_of_the_generalist(oracle_mod):
+    o = oracle_mod
+    rng = np.random.default_rng(41)
+    L, P, M = _rand_rows(rng, 5, 2, 4001)
+    tok = rng.integers(0, 4001, (5, 2)).astype(np.int32)
+    g = _round(o, L, P, M, tok, np.ones((5, 2), np.float32), rng.random(5).astype(np.float32), beta=0.0,
+               recover_mode=o.RECOVER_ARGMAX)          # u = 1: the first draft is rejected unless alpha = 1
+    for b in range(5):
+        n = int(g["accept_len"][b])
+        if g["rec_token"][b] >= 0:
+            assert g["rec_token"][b] == int(np.argmax(L[b, n]))
+
+
+def test_argmax_recovery_ignores_the_temperature_but_reports_the_tempered_probability(oracle_mod):
+    o = oracle_mod
+    rng = np.random.default_rng(42)
+    L, P, M = _rand_rows(rng, 4, 1, 999)
+    tok = np.zeros((4, 1), np.int32)
+    ua, ur = np.ones((4, 1), np.float32), np.zeros(4, np.float32)
+    toks = []
+    for T in (0.25, 1.0, 3.0):
+        g = _round(o, L, P, M, tok, ua, ur, beta=1.5, T=T, length=[0, 0, 0, 0], recover_mode=o.RECOVER_ARGMAX,
+                   flags=o.FLAG_BONUS)
+        toks.append(g["rec_token"].copy())
+        for b in range(4):
+            hr = (L[b, 0].astype(np.float64) + 1.5 * (P[b, 0].astype(np.float64) - M[b, 0].astype(np.float64))) / T
+            assert g["rec_logprob"][b] == pytest.approx(sps.log_softmax(hr)[g["rec_token"][b]], abs=1e-9)
+    assert np.array_equal(toks[0], toks[1]) and np.array_equal(toks[1], toks[2])
+
+
+def test_argmax_recovery_decides_on_single_precision_values(oracle_mod):
+    """Two entries whose exact h_rec differ by 2^-30: equal once formed in float32, so the lower id wins (exact
+    arithmetic would pick the other).  A difference float32 does resolve is honoured."""
+    o = oracle_mod
+    L = np.array([[[1.0, 1.0, 0.0]]], np.float32)
+    P = np.array([[[0.0, 2.0 ** -30, 0.0]]], np.float32)
+    M = np.zeros((1, 1, 3), np.float32)
+    kw = dict(tok=np.zeros((1, 0), np.int32), u_acc=np.zeros((1, 0), np.float32), u_rec=np.zeros(1, np.float32),
+              recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
+    assert _round(o, L, P, M, **kw)["rec_token"][0] == 0
+    P[0, 0, 1] = 2.0 ** -20
+    assert _round(o, L, P, M, **kw)["rec_token"][0] == 1
+
+
+def test_argmax_recovery_is_not_defined_for_float64_logits(oracle_mod):
+    o = oracle_mod
+    L = np.zeros((1, 1, 4))
+    with pytest.raises(RuntimeError):
+        o.verify_recover_round(L, L, L, np.zeros((1, 0), np.int32), np.zeros(1, np.int32), np.ones(1, np.float32),
+                               np.ones(1, np.float32), np.ones(1, np.float32), np.zeros((1, 0), np.float32),
+                               np.zeros(1, np.float32), recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
