@@ -58,7 +58,16 @@ typedef enum { SPECSTEER_ACCEPT_RATIO = 0, SPECSTEER_ACCEPT_EXACT_Z = 1 } specst
  *   STEER     y ~ Softmax(h_LLM + beta (h_SLM+ - h_SLM-))                   (Eq. 8; Algorithm 1 Phase 3)
  *   RESIDUAL  y ~ normalise(max(0, Softmax(h_rec) - P_SLM+)), the speculative-sampling residual of the
  *             fused target; not in the paper, offered so that EXACT_Z + RESIDUAL emits exactly P*. */
-typedef enum { SPECSTEER_RECOVER_STEER = 0, SPECSTEER_RECOVER_RESIDUAL = 1 } specsteer_recover_mode;
+typedef enum {
+  SPECSTEER_RECOVER_STEER = 0,    /* y ~ Softmax(h_rec / T), Eq. 8 (Algorithm 1 as printed) */
+  SPECSTEER_RECOVER_RESIDUAL = 1, /* y ~ norm(max(0, Softmax(h_rec / T) - P_SLM+)), an extension */
+  SPECSTEER_RECOVER_ARGMAX = 2    /* greedy decoding, the paper's experimental setting: y = the token of largest h_rec
+                                     (Eq. 8), lowest id among equals, on the rejection row and on the bonus row;
+                                     h_rec is compared as float32 forms it, fl(h_LLM + beta * fl(h_SLM+ - h_SLM-)) with
+                                     one fused multiply-add; u_recover is not used; rec_logprob is its log-probability
+                                     under Softmax(h_rec / T).  One more pass over row accept_len of every request
+                                     that takes a token.  Not available in the sharded and LM-head rounds. */
+} specsteer_recover_mode;
 
 enum {
   SPECSTEER_FLAG_BONUS = 1u,    /* when all drafts are accepted, also sample one token (STEER) from row draft_len */

@@ -18,7 +18,7 @@ OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_ORDER, ERR_TIMEOUT, ERR_STATIC_LIMIT = 1, 2, 3, 4, 5, 6, 7
 F32, BF16 = 0, 1
 ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
-RECOVER_STEER, RECOVER_RESIDUAL = 0, 1
+RECOVER_STEER, RECOVER_RESIDUAL, RECOVER_ARGMAX = 0, 1, 2
 FLAG_BONUS = 1
 FLAG_TWO_PHASE = 2
 REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1, 2, 4, 8, 16

@@ -73,7 +73,8 @@ specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc
   if (d->dtype != SPECSTEER_F32 && d->dtype != SPECSTEER_BF16) return SPECSTEER_ERR_INVALID_ARG;
   if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z)
     return SPECSTEER_ERR_INVALID_ARG;
-  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL)
+  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL &&
+      d->recover_mode != SPECSTEER_RECOVER_ARGMAX)
     return SPECSTEER_ERR_INVALID_ARG;
   if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
   if (d->B > 0) {
@@ -179,7 +180,14 @@ specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, c
       if (launch_recovery_row_lse(p, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
       ctx->launches += 2;
     }
-    if (launch_recover(p, d->dtype, ctx->li, s, &nl) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    if (d->recover_mode == SPECSTEER_RECOVER_ARGMAX) {
+      if (launch_recover_argmax(p, d->dtype, rows_aligned(d), (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
+                                ctx->topk_count + b0, ctx->li.sm_count, s) != cudaSuccess)
+        return SPECSTEER_ERR_CUDA;
+      nl = 1;
+    } else if (launch_recover(p, d->dtype, ctx->li, s, &nl) != cudaSuccess) {
+      return SPECSTEER_ERR_CUDA;
+    }
     ctx->launches += nl;
   }
   return SPECSTEER_OK;
@@ -552,7 +560,13 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
     RoundParams p = slab_params(ctx, &d, b0, nb);
     int nl = 0;
     CK(launch_verify(p, d.dtype, rows_aligned(&d), ctx->li, s, &nl)); ctx->launches += nl;
-    CK(launch_recover(p, d.dtype, ctx->li, s, &nl)); ctx->launches += nl;
+    if (d.recover_mode == SPECSTEER_RECOVER_ARGMAX) {
+      CK(launch_recover_argmax(p, d.dtype, rows_aligned(&d), (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
+                               ctx->topk_count + b0, ctx->li.sm_count, s));
+      ctx->launches += 1;
+    } else {
+      CK(launch_recover(p, d.dtype, ctx->li, s, &nl)); ctx->launches += nl;
+    }
   }
   auto back = [&](void* hp, const void* dp, size_t bytes) {
     if (hp && dp && bytes) CK(cudaMemcpyAsync(hp, dp, bytes, cudaMemcpyDeviceToHost, s));

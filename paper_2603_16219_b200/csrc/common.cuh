@@ -48,6 +48,19 @@ __device__ __forceinline__ float warp_sum(float v) {
   return v;
 }
 
+// ---- 64-bit selection keys: larger value first, among equal values the lower vocabulary id first ----------
+typedef unsigned long long u64;
+__device__ __forceinline__ uint32_t order_key(float h) {   // unsigned order = float order
+  const uint32_t b = __float_as_uint(h);
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float order_val(uint32_t k) {
+  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+__device__ __forceinline__ u64 entry_key(float h, int idx) {
+  return ((u64)order_key(h) << 32) | (u64)(0xffffffffu - (uint32_t)idx);
+}
+
 // ---- shared-memory barriers and bulk (TMA) copies -------------------------------------------
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 

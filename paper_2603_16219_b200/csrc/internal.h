@@ -107,5 +107,9 @@ cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out
 // the per-request epilogue alone (reads p.shard_parts when p.n_shards > 0)
 cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);
+// Greedy recovery (ARGMAX).  best_ws: [B][kTopkMaxSplit * 32] 64-bit words (the top-k selection's lists), count_ws: [B]
+// counters, zero between launches.  `aligned`: every row of the three tensors starts on a 16-byte boundary.
+cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned, void* best_ws, int* count_ws, int sm_count,
+                                  cudaStream_t s);
 
 }  // namespace specsteer

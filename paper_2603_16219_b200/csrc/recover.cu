@@ -307,6 +307,127 @@ __global__ void __launch_bounds__(kRecThreads) recover_residual_kernel(const Rou
   }
 }
 
+// ARGMAX (greedy decoding): the token of largest h_rec = fl(h_LLM + beta * fl(h_SLM+ - h_SLM-)) (Eq. 8) on row
+// accept_len, the lowest id among equals.  Grid (B, S): S CTAs share a row, each leaves the best key of its part of the
+// vocabulary in the workspace, and the last one to finish (a counter per request, left at zero) writes the outputs.
+template <typename T> struct Vec8;
+template <> struct Vec8<float> {
+  static __device__ __forceinline__ void load(const float* p, long long i, float (&x)[8]) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p + i)), b = __ldg(reinterpret_cast<const float4*>(p + i + 4));
+    x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
+  }
+};
+template <> struct Vec8<uint16_t> {
+  static __device__ __forceinline__ void load(const uint16_t* p, long long i, float (&x)[8]) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4*>(p + i));
+    x[0] = bf16lo(a.x); x[1] = bf16hi(a.x); x[2] = bf16lo(a.y); x[3] = bf16hi(a.y);
+    x[4] = bf16lo(a.z); x[5] = bf16hi(a.z); x[6] = bf16lo(a.w); x[7] = bf16hi(a.w);
+  }
+};
+
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const RoundParams p, u64* best_ws, int* count_ws) {
+  __shared__ u64 wbest[kRecWarps];
+  const int b = blockIdx.x, sp = blockIdx.y, S = gridDim.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = p.K, K1 = K + 1;
+  pdl_wait();
+  const ReqState st = request_state(p, b);
+  if (sp == 0 && p.out_tokens)
+    for (int t = tid; t <= K; t += kRecThreads)
+      p.out_tokens[(long long)b * K1 + t] = (t < st.n) ? p.draft_tokens[(long long)b * K + t] : -1;
+  if (!st.sample) {
+    if (sp == 0 && tid == 0) {
+      if (p.rec_token) p.rec_token[b] = -1;
+      if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+      if (p.n_out) p.n_out[b] = st.n;
+    }
+    return;
+  }
+  const T* hl = reinterpret_cast<const T*>(p.h_llm);
+  const T* hp = reinterpret_cast<const T*>(p.h_plus);
+  const T* hm = reinterpret_cast<const T*>(p.h_minus);
+  const long long off = (long long)b * p.ld_req + (long long)st.n * p.ld_row;
+  const float beta = p.beta[b];
+  const int per = (((p.V + S - 1) / S) + 7) & ~7;
+  const int v0 = sp * per, v1 = min(p.V, v0 + per);
+  u64 best = 0;  // below every key of a real entry
+  for (int v = v0 + tid * 8; v < v1; v += kRecThreads * 8) {
+    if (VEC && v + 8 <= v1) {
+      float l[8], q[8], m[8];
+      Vec8<T>::load(hl, off + v, l); Vec8<T>::load(hp, off + v, q); Vec8<T>::load(hm, off + v, m);
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        const u64 k = entry_key(fmaf(beta, q[i] - m[i], l[i]), v + i);
+        best = k > best ? k : best;
+      }
+    } else {
+      for (int i = 0; i < 8 && v + i < v1; ++i) {
+        const float l = load_logit<T>(hl, off + v + i), q = load_logit<T>(hp, off + v + i), m = load_logit<T>(hm, off + v + i);
+        const u64 k = entry_key(fmaf(beta, q - m, l), v + i);
+        best = k > best ? k : best;
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const u64 other = __shfl_xor_sync(kFullMask, best, o);
+    best = other > best ? other : best;
+  }
+  if (lane == 0) wbest[warp] = best;
+  __syncthreads();
+  if (tid != 0) return;
+  for (int w = 1; w < kRecWarps; ++w) best = wbest[w] > best ? wbest[w] : best;
+  u64* mine = best_ws + (long long)b * kTopkMaxSplit * 32;
+  if (S > 1) {
+    mine[sp] = best;
+    __threadfence();
+    if (atomicAdd(&count_ws[b], 1) != S - 1) return;
+    __threadfence();
+    for (int j = 0; j < S; ++j) {
+      const u64 k = __ldcg(mine + j);
+      best = k > best ? k : best;
+    }
+    count_ws[b] = 0;
+  }
+  if (best == 0) {  // an empty vocabulary range cannot happen (V > 0); kept for safety
+    if (p.rec_token) p.rec_token[b] = -1;
+    if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+    if (p.n_out) p.n_out[b] = st.n;
+    return;
+  }
+  const int tok = (int)(0xffffffffu - (uint32_t)(best & 0xffffffffu));
+  const double r = (double)order_val((uint32_t)(best >> 32));
+  const long long row = (long long)b * K1 + st.n;
+  const double lseR = (double)p.lse2[row * 4 + Q_R];
+  if (p.rec_token) p.rec_token[b] = tok;
+  if (p.rec_logprob) p.rec_logprob[b] = (float)((r * (double)(kLog2e / p.temperature[b]) - lseR) * 0.6931471805599453);
+  if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
+  if (p.n_out) p.n_out[b] = st.n + 1;
+}
+
+cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned, void* best_ws, int* count_ws, int sm_count,
+                                  cudaStream_t s) {
+  if (p.B == 0) return cudaSuccess;
+  int S = (2 * sm_count + p.B - 1) / p.B;   // about two CTAs per SM in total
+  S = S < 1 ? 1 : (S > kTopkMaxSplit ? kTopkMaxSplit : S);
+  while (S > 1 && (p.V + S - 1) / S < 4096) --S;   // a part below 4096 entries is not worth a CTA
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.B, S);
+  cfg.blockDim = dim3(kRecThreads);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  u64* ws = reinterpret_cast<u64*>(best_ws);
+  if (dtype == SPECSTEER_F32)
+    return aligned ? cudaLaunchKernelEx(&cfg, recover_argmax_kernel<float, true>, p, ws, count_ws)
+                   : cudaLaunchKernelEx(&cfg, recover_argmax_kernel<float, false>, p, ws, count_ws);
+  return aligned ? cudaLaunchKernelEx(&cfg, recover_argmax_kernel<uint16_t, true>, p, ws, count_ws)
+                 : cudaLaunchKernelEx(&cfg, recover_argmax_kernel<uint16_t, false>, p, ws, count_ws);
+}
+
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches) {
   (void)li;
   const size_t smem = (size_t)p.n_chunks * sizeof(double);

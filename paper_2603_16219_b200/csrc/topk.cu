@@ -16,18 +16,6 @@ namespace specsteer {
 constexpr int kTopThreads = 512;
 constexpr int kTopWarps = kTopThreads / 32;
 
-typedef unsigned long long u64;
-
-__device__ __forceinline__ uint32_t order_key(float h) {
-  const uint32_t b = __float_as_uint(h);
-  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-}
-__device__ __forceinline__ float order_val(uint32_t k) {
-  return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
-}
-__device__ __forceinline__ u64 entry_key(float h, int idx) {
-  return ((u64)order_key(h) << 32) | (u64)(0xffffffffu - (uint32_t)idx);
-}
 
 // Insert `nk` into the warp's descending list (one key per lane, 0 = empty slot) if it beats the last entry.
 __device__ __forceinline__ void warp_insert(u64& mykey, u64 nk, int lane) {
