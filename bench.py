@@ -196,7 +196,8 @@ def run_cuda(args, rank, world, local_rank):
         # rows, and the recovery call streams its one row per request (Eq. 8)
         for name in ("logp_plus", "logp_star", "log_z"):
             outs.pop(name)
-    desc = binding.make_desc(inputs, outs, flags=flags)
+    rmode = binding.RECOVER_ARGMAX if args.greedy else binding.RECOVER_STEER
+    desc = binding.make_desc(inputs, outs, flags=flags, recover_mode=rmode)
     stream = torch.cuda.current_stream(dev)
 
     # When the batch fits in L2 (126 MB) rotate over enough copies to exceed it; otherwise the batch itself does.
@@ -206,7 +207,7 @@ def run_cuda(args, rank, world, local_rank):
     sets = [(inputs, desc)]
     for i in range(1, n_sets):
         cp = {k: v.clone() for k, v in inputs.items()}
-        sets.append((cp, binding.make_desc(cp, outs, flags=flags)))
+        sets.append((cp, binding.make_desc(cp, outs, flags=flags, recover_mode=rmode)))
 
     def step(i):
         d = sets[i % n_sets][1]
@@ -305,7 +306,8 @@ def run_cuda(args, rank, world, local_rank):
             extra["warm_l2_ms_per_step"] = w0e.elapsed_time(w1e) / args.steps
         sampler.stop()
         if rank == 0:
-            line = {"workload": spec.name, "outputs": ("lean, two-phase" if two_phase else "lean, one pass") if args.lean else "all", "ms_per_step": ms_per_step,
+            line = {"workload": spec.name, "outputs": ("lean, two-phase" if two_phase else "lean, one pass") if args.lean else "all",
+                    "recovery": "greedy (argmax of h_rec)" if args.greedy else "sampled", "ms_per_step": ms_per_step,
                     "verify_kernel_ms": kernel_ms, "verify_gbs": logit_bytes / (kernel_ms * 1e-3) / 1e9,
                     "positions_per_s": value, "clocks": sampler.summary()}
             line.update(extra)
@@ -568,6 +570,8 @@ def main():
                     help="with --kernels-only: also time the top-k split recovery (cloud + edge kernels) with this k")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the device-resident steps and print a short line (profiling aid)")
+    ap.add_argument("--greedy", action="store_true",
+                    help="with --kernels-only: greedy recovery (the token of largest h_rec) instead of sampling")
     ap.add_argument("--lmhead", action="store_true",
                     help="time the round with the LM heads fused in front (hidden states and head weights in, 1 GPU)")
     ap.add_argument("--d-llm", type=int, default=5120, help="with --lmhead: hidden width of the Generalist")
