@@ -267,3 +267,14 @@ def test_one_context_serves_both_paths_and_changing_shapes(env):
     again = _run_gpu(env, lm)
     for k in first:
         assert np.array_equal(first[k], again[k], equal_nan=True), k
+
+
+@pytest.mark.parametrize("V,d_llm,d_slm", [(100, 8, 8), (128, 64, 16), (129, 72, 8), (5, 16, 8)])
+def test_tiny_vocabularies_and_hidden_widths(env, V, d_llm, d_slm):
+    """A vocabulary below one tile, exactly one tile, one entry more; hidden widths below one stage of 64."""
+    _case(env, _spec(env, 0, B=4, K=2, V=V), d_llm, d_slm, seed=20 + V)
+
+
+def test_many_rows_few_vocabulary_tiles(env):
+    """1024 rows = 8 row blocks over 3 vocabulary tiles: fewer tiles than SMs, every CTA at most one tile."""
+    _case(env, _spec(env, 2, B=128, K=7, V=300, ragged=True), 128, 64, seed=30)
