@@ -136,7 +136,8 @@ bool rows_aligned(const specsteer_round_desc* d) {
 // fused target on the drafted rows, the h_SLM+ tensor is left unread there and the recovery call forms the
 // normalisers of its one row itself (Eq. 8 on the row of the first rejection).
 bool two_phase(const specsteer_round_desc* d) {
-  const bool eligible = d->accept_mode == SPECSTEER_ACCEPT_RATIO && d->recover_mode == SPECSTEER_RECOVER_STEER &&
+  const bool eligible = d->accept_mode == SPECSTEER_ACCEPT_RATIO &&
+                        (d->recover_mode == SPECSTEER_RECOVER_STEER || d->recover_mode == SPECSTEER_RECOVER_ARGMAX) &&
                         !d->logp_plus && !d->logp_star && !d->log_z && rows_aligned(d);
   if (!eligible) return false;
   if (d->flags & SPECSTEER_FLAG_TWO_PHASE) return true;
@@ -173,7 +174,7 @@ specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, c
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
     RoundParams p = slab_params(ctx, d, b0, nb);
     int nl = 0;
-    if (lean) {   // the recovery rows have no records yet: one more streaming pass over them alone
+    if (lean && d->recover_mode != SPECSTEER_RECOVER_ARGMAX) {   // the recovery rows have no records yet: one more streaming pass over them alone
       p.sums = SUM_ALL;
       p.row_mode = ROWS_RECOVERY;
       if (launch_verify_stream(p, d->dtype, true, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
@@ -181,7 +182,7 @@ specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, c
       ctx->launches += 2;
     }
     if (d->recover_mode == SPECSTEER_RECOVER_ARGMAX) {
-      if (launch_recover_argmax(p, d->dtype, rows_aligned(d), (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
+      if (launch_recover_argmax(p, d->dtype, rows_aligned(d), lean, (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
                                 ctx->topk_count + b0, ctx->li.sm_count, s) != cudaSuccess)
         return SPECSTEER_ERR_CUDA;
       nl = 1;
@@ -561,7 +562,7 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
     int nl = 0;
     CK(launch_verify(p, d.dtype, rows_aligned(&d), ctx->li, s, &nl)); ctx->launches += nl;
     if (d.recover_mode == SPECSTEER_RECOVER_ARGMAX) {
-      CK(launch_recover_argmax(p, d.dtype, rows_aligned(&d), (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
+      CK(launch_recover_argmax(p, d.dtype, rows_aligned(&d), false, (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
                                ctx->topk_count + b0, ctx->li.sm_count, s));
       ctx->launches += 1;
     } else {

@@ -109,7 +109,8 @@ cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);
 // Greedy recovery (ARGMAX).  best_ws: [B][kTopkMaxSplit * 32] 64-bit words (the top-k selection's lists), count_ws: [B]
 // counters, zero between launches.  `aligned`: every row of the three tensors starts on a 16-byte boundary.
-cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned, void* best_ws, int* count_ws, int sm_count,
-                                  cudaStream_t s);
+// `own_lse`: the row has no normaliser in lse2 (two-phase round): the pass forms it, and the row's finiteness check, itself.
+cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned, bool own_lse, void* best_ws, int* count_ws,
+                                  int sm_count, cudaStream_t s);
 
 }  // namespace specsteer

@@ -325,9 +325,27 @@ template <> struct Vec8<uint16_t> {
   }
 };
 
-template <typename T, bool VEC>
+// An online (maximum, sum of 2^(x - maximum)) pair and its merge; empty = (-inf, 0).
+struct OnlineLse {
+  float m, s;
+};
+__device__ __forceinline__ OnlineLse lse_merge(OnlineLse a, OnlineLse b) {
+  const float m = fmaxf(a.m, b.m);
+  OnlineLse r;
+  r.m = m;
+  r.s = (a.m == kNegInf ? 0.f : a.s * ex2(a.m - m)) + (b.m == kNegInf ? 0.f : b.s * ex2(b.m - m));
+  if (a.s != a.s || b.s != b.s) r.s = a.s + b.s;   // a NaN sum stays NaN whatever the maxima are
+  return r;
+}
+
+// LSE: the row has no normaliser yet (verification read only h_LLM and h_SLM- and not this row's h_SLM+): the pass
+// also forms log2 sum 2^(h_rec c) online for rec_logprob, and checks what the streaming pass would have checked -
+// a NaN or +inf anywhere in the three streams of the row, or a stream that is -inf throughout, raises REQ_NONFINITE.
+template <typename T, bool VEC, bool LSE>
 __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const RoundParams p, u64* best_ws, int* count_ws) {
   __shared__ u64 wbest[kRecWarps];
+  __shared__ OnlineLse wlse[kRecWarps];
+  __shared__ float wmax[kRecWarps][3];
   const int b = blockIdx.x, sp = blockIdx.y, S = gridDim.y, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = p.K, K1 = K + 1;
   pdl_wait();
@@ -348,23 +366,55 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   const T* hm = reinterpret_cast<const T*>(p.h_minus);
   const long long off = (long long)b * p.ld_req + (long long)st.n * p.ld_row;
   const float beta = p.beta[b];
+  const float c = kLog2e / p.temperature[b];
   const int per = (((p.V + S - 1) / S) + 7) & ~7;
   const int v0 = sp * per, v1 = min(p.V, v0 + per);
   u64 best = 0;  // below every key of a real entry
+  OnlineLse acc = {kNegInf, 0.f};
+  float mx[3] = {kNegInf, kNegInf, kNegInf};   // largest entry of each stream
+  bool bad = false;                            // a NaN or +inf entry
   for (int v = v0 + tid * 8; v < v1; v += kRecThreads * 8) {
+    float l[8], q[8], m[8], r[8];
+    int n = 8;
     if (VEC && v + 8 <= v1) {
-      float l[8], q[8], m[8];
       Vec8<T>::load(hl, off + v, l); Vec8<T>::load(hp, off + v, q); Vec8<T>::load(hm, off + v, m);
-#pragma unroll
+    } else {
+      n = min(8, v1 - v);
       for (int i = 0; i < 8; ++i) {
-        const u64 k = entry_key(fmaf(beta, q[i] - m[i], l[i]), v + i);
+        const bool in = i < n;
+        l[i] = in ? load_logit<T>(hl, off + v + i) : kNegInf;
+        q[i] = in ? load_logit<T>(hp, off + v + i) : 0.f;
+        m[i] = in ? load_logit<T>(hm, off + v + i) : 0.f;
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      r[i] = fmaf(beta, q[i] - m[i], l[i]);   // Eq. 8
+      if (i < n) {
+        const u64 k = entry_key(r[i], v + i);
         best = k > best ? k : best;
       }
-    } else {
-      for (int i = 0; i < 8 && v + i < v1; ++i) {
-        const float l = load_logit<T>(hl, off + v + i), q = load_logit<T>(hp, off + v + i), m = load_logit<T>(hm, off + v + i);
-        const u64 k = entry_key(fmaf(beta, q - m, l), v + i);
-        best = k > best ? k : best;
+    }
+    if (LSE) {
+      float x[8];
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        x[i] = r[i] * c;
+        if (i < n) {
+          bad = bad || !(l[i] < -kNegInf) || !(q[i] < -kNegInf) || !(m[i] < -kNegInf);
+          mx[0] = fmaxf(mx[0], l[i]); mx[1] = fmaxf(mx[1], q[i]); mx[2] = fmaxf(mx[2], m[i]);
+        } else {
+          x[i] = kNegInf;
+        }
+      }
+      const float m8 = max8(x);
+      if (m8 > acc.m) {
+        acc.s = (acc.m == kNegInf) ? 0.f : acc.s * ex2(acc.m - m8);
+        acc.m = m8;
+      }
+      if (acc.m > kNegInf) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc.s += ex2(x[i] - acc.m);
       }
     }
   }
@@ -372,24 +422,67 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   for (int o = 16; o > 0; o >>= 1) {
     const u64 other = __shfl_xor_sync(kFullMask, best, o);
     best = other > best ? other : best;
+    if (LSE) {
+      OnlineLse t;
+      t.m = __shfl_xor_sync(kFullMask, acc.m, o);
+      t.s = __shfl_xor_sync(kFullMask, acc.s, o);
+      acc = lse_merge(acc, t);
+#pragma unroll
+      for (int q = 0; q < 3; ++q) mx[q] = fmaxf(mx[q], __shfl_xor_sync(kFullMask, mx[q], o));
+    }
   }
-  if (lane == 0) wbest[warp] = best;
+  if (LSE && __any_sync(kFullMask, bad)) acc.s = __int_as_float(0x7fc00000);
+  if (lane == 0) {
+    wbest[warp] = best;
+    if (LSE) { wlse[warp] = acc; wmax[warp][0] = mx[0]; wmax[warp][1] = mx[1]; wmax[warp][2] = mx[2]; }
+  }
   __syncthreads();
   if (tid != 0) return;
-  for (int w = 1; w < kRecWarps; ++w) best = wbest[w] > best ? wbest[w] : best;
+  for (int w = 1; w < kRecWarps; ++w) {
+    best = wbest[w] > best ? wbest[w] : best;
+    if (LSE) {
+      acc = lse_merge(acc, wlse[w]);
+      for (int q = 0; q < 3; ++q) mx[q] = fmaxf(mx[q], wmax[w][q]);
+    }
+  }
+  // workspace of the request: [0, 16) keys, [16, 32) {maximum, sum}, [32, 48) {max h_LLM, max h_SLM+}, [48, 64) max h_SLM-
   u64* mine = best_ws + (long long)b * kTopkMaxSplit * 32;
+  auto pack = [](float a, float b2) { return ((u64)__float_as_uint(a) << 32) | (u64)__float_as_uint(b2); };
   if (S > 1) {
     mine[sp] = best;
+    if (LSE) { mine[16 + sp] = pack(acc.m, acc.s); mine[32 + sp] = pack(mx[0], mx[1]); mine[48 + sp] = pack(mx[2], 0.f); }
     __threadfence();
     if (atomicAdd(&count_ws[b], 1) != S - 1) return;
     __threadfence();
     for (int j = 0; j < S; ++j) {
+      if (j == sp) continue;
       const u64 k = __ldcg(mine + j);
       best = k > best ? k : best;
+      if (LSE) {
+        const u64 a = __ldcg(mine + 16 + j), b2 = __ldcg(mine + 32 + j), c2 = __ldcg(mine + 48 + j);
+        OnlineLse t = {__uint_as_float((uint32_t)(a >> 32)), __uint_as_float((uint32_t)a)};
+        acc = lse_merge(acc, t);
+        mx[0] = fmaxf(mx[0], __uint_as_float((uint32_t)(b2 >> 32)));
+        mx[1] = fmaxf(mx[1], __uint_as_float((uint32_t)b2));
+        mx[2] = fmaxf(mx[2], __uint_as_float((uint32_t)(c2 >> 32)));
+      }
     }
     count_ws[b] = 0;
   }
-  if (best == 0) {  // an empty vocabulary range cannot happen (V > 0); kept for safety
+  const long long row = (long long)b * K1 + st.n;
+  double lseR;
+  bool fin = best != 0;
+  if (LSE) {
+    lseR = (double)acc.m + log2((double)acc.s);
+    fin = fin && isfinite(lseR) && mx[0] > kNegInf && mx[1] > kNegInf && mx[2] > kNegInf;
+    if (!fin) {
+      p.status_ws[b] = st.status | SPECSTEER_REQ_NONFINITE;
+      if (p.req_status) p.req_status[b] = st.status | SPECSTEER_REQ_NONFINITE;
+    }
+  } else {
+    lseR = (double)p.lse2[row * 4 + Q_R];
+  }
+  if (!fin) {
     if (p.rec_token) p.rec_token[b] = -1;
     if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
     if (p.n_out) p.n_out[b] = st.n;
@@ -397,16 +490,23 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   }
   const int tok = (int)(0xffffffffu - (uint32_t)(best & 0xffffffffu));
   const double r = (double)order_val((uint32_t)(best >> 32));
-  const long long row = (long long)b * K1 + st.n;
-  const double lseR = (double)p.lse2[row * 4 + Q_R];
   if (p.rec_token) p.rec_token[b] = tok;
-  if (p.rec_logprob) p.rec_logprob[b] = (float)((r * (double)(kLog2e / p.temperature[b]) - lseR) * 0.6931471805599453);
+  if (p.rec_logprob) p.rec_logprob[b] = (float)((r * (double)c - lseR) * 0.6931471805599453);
   if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
   if (p.n_out) p.n_out[b] = st.n + 1;
 }
 
-cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned, void* best_ws, int* count_ws, int sm_count,
-                                  cudaStream_t s) {
+template <typename T>
+static cudaError_t launch_argmax_t(const cudaLaunchConfig_t& cfg, bool aligned, bool own_lse, const RoundParams& p, u64* ws,
+                                   int* count_ws) {
+  if (aligned) return own_lse ? cudaLaunchKernelEx(&cfg, recover_argmax_kernel<T, true, true>, p, ws, count_ws)
+                              : cudaLaunchKernelEx(&cfg, recover_argmax_kernel<T, true, false>, p, ws, count_ws);
+  return own_lse ? cudaLaunchKernelEx(&cfg, recover_argmax_kernel<T, false, true>, p, ws, count_ws)
+                 : cudaLaunchKernelEx(&cfg, recover_argmax_kernel<T, false, false>, p, ws, count_ws);
+}
+
+cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned, bool own_lse, void* best_ws, int* count_ws,
+                                  int sm_count, cudaStream_t s) {
   if (p.B == 0) return cudaSuccess;
   int S = (2 * sm_count + p.B - 1) / p.B;   // about two CTAs per SM in total
   S = S < 1 ? 1 : (S > kTopkMaxSplit ? kTopkMaxSplit : S);
@@ -421,11 +521,8 @@ cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned,
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   u64* ws = reinterpret_cast<u64*>(best_ws);
-  if (dtype == SPECSTEER_F32)
-    return aligned ? cudaLaunchKernelEx(&cfg, recover_argmax_kernel<float, true>, p, ws, count_ws)
-                   : cudaLaunchKernelEx(&cfg, recover_argmax_kernel<float, false>, p, ws, count_ws);
-  return aligned ? cudaLaunchKernelEx(&cfg, recover_argmax_kernel<uint16_t, true>, p, ws, count_ws)
-                 : cudaLaunchKernelEx(&cfg, recover_argmax_kernel<uint16_t, false>, p, ws, count_ws);
+  return dtype == SPECSTEER_F32 ? launch_argmax_t<float>(cfg, aligned, own_lse, p, ws, count_ws)
+                                : launch_argmax_t<uint16_t>(cfg, aligned, own_lse, p, ws, count_ws);
 }
 
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches) {

@@ -113,3 +113,73 @@ def test_host_round_in_greedy_mode(env):
     env["ctx"].round_host(b.make_desc(host_in, host_out, recover_mode=ARGMAX, flags=1))
     for k, v in host_out.items():
         assert np.array_equal(v.numpy(), dev[k], equal_nan=True), k
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("flags", [0, 1])
+def test_two_phase_greedy_round(env, dtype, flags):
+    """Only Algorithm 1's outputs, greedy: verification reads h_LLM and h_SLM- over the drafted rows (h_SLM+ is
+    poisoned everywhere else to prove it), and the argmax pass over row accept_len forms that row's normaliser and
+    finiteness check itself.  Three launches."""
+    b = env["binding"]
+    synth = env["synth"]
+    spec = synth.RoundSpec("g", 10, 4, 9004 if dtype == "f32" else 12288, dtype, ragged=True,
+                           beta_choices=(0.5, 1.0, 2.0), temp_choices=(0.7, 1.0))
+    inputs = synth.make_round(spec, device="cuda", seed=41)
+    inputs["draft_len"][0] = 0
+    inputs["u_accept"][1] = 0.0                      # everything accepted
+    inputs["lam"][3] = 1e30                          # rejected at once; row 0 is non-finite only through h_SLM+
+    inputs["h_slm_plus"][3, 0, 5] = float("inf")
+    inputs["lam"][4] = 1e30
+    inputs["h_slm_plus"][4, 0, :] = float("-inf")    # h_SLM+ is -inf throughout the recovery row: only that pass can tell
+    ora = P.run_oracle(env["oracle"], P.to_np_inputs(inputs), 0, ARGMAX, flags)
+    hp = inputs["h_slm_plus"].clone()
+    keep = torch.zeros(hp.shape[:2], dtype=torch.bool, device="cuda")
+    for r in range(spec.B):
+        n, ln = int(ora["accept_len"][r]), int(inputs["draft_len"][r])
+        if n < ln or flags:
+            keep[r, n] = True
+    hp[~keep] = float("nan")
+    poisoned = dict(inputs)
+    poisoned["h_slm_plus"] = hp
+    skip = ("logp_plus", "logp_star", "log_z")
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in skip}
+    d = b.make_desc(poisoned, outs, recover_mode=ARGMAX, flags=flags | b.FLAG_TWO_PHASE)
+    before = env["ctx"].launch_count
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0
+    assert env["ctx"].launch_count - before == 3
+    gpu = {k: v.cpu().numpy() for k, v in outs.items()}
+    safe = (ora["accept_margin"] > P.MARGIN).all(axis=1)
+    assert safe.sum() >= spec.B - 1
+    for k in ("accept_len", "rec_token", "n_out", "req_status", "out_tokens"):
+        assert np.array_equal(gpu[k][safe], ora[k][safe]), k
+    assert gpu["req_status"][3] == b.REQ_NONFINITE and gpu["rec_token"][3] == -1 and gpu["accept_len"][3] == 0
+    assert gpu["req_status"][4] == b.REQ_NONFINITE and gpu["rec_token"][4] == -1 and gpu["accept_len"][4] == 0
+    safe[3] = safe[4] = False   # their per-position diagnostics differ by design: the oracle reads h_SLM+ on drafted rows
+    tol = P.TOL[inputs["h_llm"].dtype]
+    for k in ("alpha", "logp_llm", "logp_minus", "rec_logprob"):
+        fin = np.isfinite(ora[k]) & (safe[:, None] if ora[k].ndim == 2 else safe)
+        assert np.array_equal(np.isnan(gpu[k][safe]), np.isnan(ora[k][safe])), k
+        assert np.abs(gpu[k][fin] - ora[k][fin]).max(initial=0.0) <= tol, k
+
+
+def test_two_phase_greedy_full_size_equals_one_pass(env):
+    """Config 3 at full size: the two-phase greedy round (taken automatically for a batch this large) gives the same
+    accepted lengths and tokens as the one-pass greedy round that was asked for every output."""
+    b, synth = env["binding"], env["synth"]
+    spec = synth.CONFIGS[3]
+    inputs = synth.make_round(spec, device="cuda", seed=0)
+    full = P.run_gpu(env["ctx"], inputs, 0, ARGMAX, 1)
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in ("logp_plus", "logp_star", "log_z")}
+    d = b.make_desc(inputs, outs, recover_mode=ARGMAX, flags=1)
+    before = env["ctx"].launch_count
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 3
+    for k in ("accept_len", "rec_token", "n_out", "out_tokens", "req_status", "accept_flags"):
+        assert np.array_equal(outs[k].cpu().numpy(), full[k]), k
+    assert np.abs(outs["rec_logprob"].cpu().numpy() - full["rec_logprob"]).max() <= 1e-5
