@@ -106,10 +106,10 @@ typedef struct {
   /* ---- outputs (caller-allocated; any may be NULL except accept_len) ----
    * What is requested decides what is read.  Algorithm 1 itself needs the normalisers of h_LLM and h_SLM- on the
    * drafted rows (Eq. 7) and that of h_rec on the one row it recovers from (Eq. 8).
-   *   - RATIO + STEER with logp_plus, logp_star and log_z all NULL (and 16-byte aligned rows): verification reads
-   *     h_LLM and h_SLM- alone, over the drafted rows; specsteer_recover_sample then streams row accept_len of the
-   *     requests that sample, all three tensors: the two-phase round, about a fifth fewer bytes (taken automatically
-   *     for large batches, see SPECSTEER_FLAG_TWO_PHASE).  A non-finite entry of
+   *   - RATIO + STEER (or ARGMAX) with logp_plus, logp_star and log_z all NULL (and 16-byte aligned rows):
+   *     verification reads h_LLM and h_SLM- alone, over the drafted rows; specsteer_recover_sample then streams row
+   *     accept_len of the requests that take a token, all three tensors: the two-phase round, about a fifth fewer
+   *     bytes (taken automatically for large batches, see SPECSTEER_FLAG_TWO_PHASE).  A non-finite entry of
    *     h_SLM+ on a drafted row is then not seen (REQ_NONFINITE is raised for it only on the recovery row).
    *   - logp_star wanted, logp_plus and log_z NULL: one pass over all three tensors and all rows, but the
    *     normaliser of h_SLM+ is not formed (a quarter fewer exponentials; it matters for 16-bit logits).
