@@ -345,6 +345,29 @@ def run_cuda(args, rank, world, local_rank):
         same = torch.equal(lean_outs["accept_len"], outs["accept_len"]) and torch.equal(lean_outs["rec_token"], outs["rec_token"])
         alg1 = {"value": world * positions / (lean_ms * 1e-3), "unit": UNIT, "ms_per_step": lean_ms, "steps": n_lean,
                 "outputs": "no logp_plus, logp_star, log_z", "same_accept_len_and_tokens_as_headline": bool(same)}
+        # the same outputs under greedy decoding (the paper's experimental setting): the token of largest h_rec
+        greedy_sets = [binding.make_desc(si, lean_outs, flags=flags, recover_mode=binding.RECOVER_ARGMAX) for si, _ in sets]
+        for i in range(3):
+            ctx.verify_round(greedy_sets[i % n_sets], stream)
+            ctx.recover_sample(greedy_sets[i % n_sets], stream)
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        w0 = time.perf_counter()
+        g0.record(stream)
+        for i in range(n_lean):
+            ctx.verify_round(greedy_sets[i % n_sets], stream)
+            ctx.recover_sample(greedy_sets[i % n_sets], stream)
+        g1.record(stream)
+        barrier()
+        sampler.window(w0, time.perf_counter())
+        greedy_ms = g0.elapsed_time(g1) / n_lean
+        if dist is not None:
+            t = torch.tensor([greedy_ms], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            greedy_ms = float(t.item())
+        alg1["greedy_recovery"] = {"value": world * positions / (greedy_ms * 1e-3), "unit": UNIT, "ms_per_step": greedy_ms,
+                                   "steps": n_lean,
+                                   "same_accept_len_as_headline": bool(torch.equal(lean_outs["accept_len"], outs["accept_len"]))}
     # ---- end to end: pinned host buffers in, pinned host results out, copies inside the timed region
     host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
     host_out = binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True)

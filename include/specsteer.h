@@ -229,6 +229,27 @@ typedef struct {
 } specsteer_lmhead_desc;
 specsteer_status specsteer_lmhead_round(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc, void *cuda_stream);
 
+/* The fused round with the heads split along the vocabulary over n_shards GPUs (a tensor-parallel LM head): GPU g
+ * holds rows [vocab_offset_g, vocab_offset_g + V_g) of every head (desc->round.V = V_g, w_* point at those rows) and
+ * all the hidden states.  Same four steps and the same two collectives as the vocabulary-sharded round above:
+ *   1. specsteer_lmhead_shard_local: the tensor-core pass over the local rows of the heads, then one 64-byte partial
+ *      per row into row_partials [B][K+1][64 bytes] (the drafted token's logits if the token lies in the shard);
+ *   2. the caller all-gathers the partials into gathered [n_shards][B][K+1][64 bytes];
+ *   3. specsteer_lmhead_shard_combine: every verification output, identical on every GPU;
+ *   4. specsteer_lmhead_shard_recover: the shard that holds the CDF target recomputes its chunk and writes the global
+ *      token id; the others write -1, -inf, the accepted prefix and accept_len, for an element-wise MAX all-reduce
+ *      of rec_token, rec_logprob, out_tokens and n_out.
+ * No logit and no head weight crosses the link.  draft_tokens hold GLOBAL ids.  B <= 1024.
+ * Errors: as specsteer_lmhead_round and the sharded round. */
+specsteer_status specsteer_lmhead_shard_local(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc, int32_t vocab_offset,
+                                              void *row_partials, void *cuda_stream);
+specsteer_status specsteer_lmhead_shard_combine(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc, const void *gathered,
+                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                                int32_t vocab_total, void *cuda_stream);
+specsteer_status specsteer_lmhead_shard_recover(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc, const void *gathered,
+                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                                int32_t vocab_total, void *cuda_stream);
+
 /* Whole round from HOST memory: every pointer in `desc` is a HOST pointer (pinned memory makes the copies
  * asynchronous).  Copies inputs to device staging buffers owned by the context (allocated on the first
  * call, sized for the context's maxima: 3*max_B*(max_K+1)*max_V elements of 4 bytes), runs verification and

@@ -31,6 +31,7 @@ EXPORTS = (
     "specsteer_cloud_topk", "specsteer_edge_resample",
     "specsteer_shard_verify_local", "specsteer_shard_verify_combine", "specsteer_shard_recover_local",
     "specsteer_lmhead_round",
+    "specsteer_lmhead_shard_local", "specsteer_lmhead_shard_combine", "specsteer_lmhead_shard_recover",
 )
 SHARD_PARTIAL_BYTES = 64
 MAX_SHARDS = 32
@@ -106,6 +107,11 @@ def load_library(path: Optional[str] = None):
         fn.restype = C.c_int
     lib.specsteer_lmhead_round.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p]
     lib.specsteer_lmhead_round.restype = C.c_int
+    lib.specsteer_lmhead_shard_local.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_int32, C.c_void_p, C.c_void_p]
+    lib.specsteer_lmhead_shard_local.restype = C.c_int
+    for fn in (lib.specsteer_lmhead_shard_combine, lib.specsteer_lmhead_shard_recover):
+        fn.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
+        fn.restype = C.c_int
     lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.specsteer_ctx_time_streaming.restype = C.c_int
     lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
@@ -280,6 +286,34 @@ class Context:
     def lmhead_round(self, desc: LmheadDesc, stream=None):
         """Verification and recovery with the three LM heads fused in front: no logit tensor is ever stored."""
         _check(self._lib.specsteer_lmhead_round(self._h, C.byref(desc), self._stream(stream)), "specsteer_lmhead_round")
+
+    def lmhead_shard_local(self, desc: LmheadDesc, vocab_offset: int, row_partials: torch.Tensor, stream=None):
+        """Step 1 of the fused round with heads split along the vocabulary: this shard's 64-byte partial per row."""
+        r = desc.round
+        if row_partials.dtype != torch.uint8 or tuple(row_partials.shape) != (r.B, r.K + 1, SHARD_PARTIAL_BYTES) \
+                or not row_partials.is_contiguous():
+            raise ValueError("row_partials must be a contiguous uint8 tensor [B, K+1, 64]")
+        _check(self._lib.specsteer_lmhead_shard_local(self._h, C.byref(desc), int(vocab_offset),
+                                                      C.c_void_p(row_partials.data_ptr()), self._stream(stream)),
+               "specsteer_lmhead_shard_local")
+
+    def _lmhead_shard_call(self, fn, name, desc, gathered, shard_rank, vocab_offset, vocab_total, stream):
+        r = desc.round
+        if gathered.dtype != torch.uint8 or gathered.dim() != 4 or not gathered.is_contiguous() or \
+                tuple(gathered.shape[1:]) != (r.B, r.K + 1, SHARD_PARTIAL_BYTES):
+            raise ValueError("gathered must be a contiguous uint8 tensor [n_shards, B, K+1, 64]")
+        _check(fn(self._h, C.byref(desc), C.c_void_p(gathered.data_ptr()), int(gathered.shape[0]), int(shard_rank),
+                  int(vocab_offset), int(vocab_total), self._stream(stream)), name)
+
+    def lmhead_shard_combine(self, desc, gathered, shard_rank, vocab_offset, vocab_total, stream=None):
+        """Step 3: acceptance from the gathered partials of all shards."""
+        self._lmhead_shard_call(self._lib.specsteer_lmhead_shard_combine, "specsteer_lmhead_shard_combine", desc, gathered,
+                                shard_rank, vocab_offset, vocab_total, stream)
+
+    def lmhead_shard_recover(self, desc, gathered, shard_rank, vocab_offset, vocab_total, stream=None):
+        """Step 4: the shard that holds the CDF target recomputes its chunk and samples."""
+        self._lmhead_shard_call(self._lib.specsteer_lmhead_shard_recover, "specsteer_lmhead_shard_recover", desc, gathered,
+                                shard_rank, vocab_offset, vocab_total, stream)
 
     def cloud_topk(self, desc: RoundDesc, topk_idx: torch.Tensor, topk_val: torch.Tensor, stream=None):
         """Cloud half of the top-k split recovery: fills topk_idx [B, k] int32 and topk_val [B, k] float32."""

@@ -377,7 +377,9 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx* ctx, const specste
   return SPECSTEER_OK;
 }
 
-specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, void* cuda_stream) {
+namespace {
+// Checks an LM-head descriptor, makes sure the second workspace exists and fills the kernels' parameters.
+specsteer_status prep_lmhead(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, RoundParams* p, LmheadOperands* op) {
   if (!ctx || !ld) return SPECSTEER_ERR_INVALID_ARG;
   const specsteer_round_desc* d = &ld->round;
   if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
@@ -399,43 +401,117 @@ specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhe
   if ((size_t)(ld->d_llm + 2 * ld->d_slm) * 2 + (size_t)n_chunks_of(d->V, kLmheadChunk) * 8 + 64 > 200 * 1024)
     return SPECSTEER_ERR_UNSUPPORTED;   // the recovery kernel keeps the row's hidden states and chunk weights in shared memory
   if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
-  ctx->verified = false;
-  ctx->shard_streamed = false;
   if (d->B == 0) return SPECSTEER_OK;
-  DeviceGuard g(ctx->device);
-  if (!g.ok) return SPECSTEER_ERR_CUDA;
-  cudaStream_t s = (cudaStream_t)cuda_stream;
   const int K1 = d->K + 1;
   if (!ctx->lm_ws) {   // sized for the context's maxima, once
     const size_t rows = (size_t)ctx->max_B * (ctx->max_K + 1);
     const size_t part_bytes = align_up(rows * (size_t)n_chunks_of(ctx->max_V, kLmheadChunk) * 32, 256);
     const size_t tok_bytes = align_up(rows * 16, 256);
-    if (cudaMalloc(&ctx->lm_ws, part_bytes + tok_bytes) != cudaSuccess) { ctx->lm_ws = nullptr; return SPECSTEER_ERR_WORKSPACE; }
+    if (cudaMalloc(&ctx->lm_ws, part_bytes + tok_bytes) != cudaSuccess) { ctx->lm_ws = nullptr; (void)cudaGetLastError(); return SPECSTEER_ERR_WORKSPACE; }
     ctx->lm_part = (float*)ctx->lm_ws;
     ctx->lm_tok = (float*)((char*)ctx->lm_ws + part_bytes);
     ctx->ws_bytes += part_bytes + tok_bytes;
   }
   specsteer_round_desc dd = *d;
   dd.dtype = SPECSTEER_F32; dd.ld_row = d->V; dd.ld_req = (int64_t)K1 * d->V;   // no logit tensor exists
-  RoundParams p = slab_params(ctx, &dd, 0, d->B);
-  p.h_llm = p.h_plus = p.h_minus = nullptr;
-  p.sums = SUM_ALL;
-  p.row_mode = ROWS_ALL;
-  p.tile = kLmheadChunk;
-  p.n_chunks = n_chunks_of(d->V, kLmheadChunk);
-  p.part = ctx->lm_part;
-  p.tok_logits = ctx->lm_tok;
+  *p = slab_params(ctx, &dd, 0, d->B);
+  p->h_llm = p->h_plus = p->h_minus = nullptr;
+  p->sums = SUM_ALL;
+  p->row_mode = ROWS_ALL;
+  p->tile = kLmheadChunk;
+  p->n_chunks = n_chunks_of(d->V, kLmheadChunk);
+  p->part = ctx->lm_part;
+  p->tok_logits = ctx->lm_tok;
+  op->x_llm = (const uint16_t*)ld->x_llm; op->w_llm = (const uint16_t*)ld->w_llm;
+  op->x_plus = (const uint16_t*)ld->x_slm_plus; op->w_plus = (const uint16_t*)ld->w_slm_plus;
+  op->x_minus = (const uint16_t*)ld->x_slm_minus; op->w_minus = (const uint16_t*)ld->w_slm_minus;
+  op->d_llm = ld->d_llm; op->d_slm = ld->d_slm;
+  return SPECSTEER_OK;
+}
+}  // namespace
+
+specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, void* cuda_stream) {
+  RoundParams p;
   LmheadOperands op;
-  op.x_llm = (const uint16_t*)ld->x_llm; op.w_llm = (const uint16_t*)ld->w_llm;
-  op.x_plus = (const uint16_t*)ld->x_slm_plus; op.w_plus = (const uint16_t*)ld->w_slm_plus;
-  op.x_minus = (const uint16_t*)ld->x_slm_minus; op.w_minus = (const uint16_t*)ld->w_slm_minus;
-  op.d_llm = ld->d_llm; op.d_slm = ld->d_slm;
+  specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
+  if (st != SPECSTEER_OK) return st;
+  ctx->verified = false;
+  ctx->shard_streamed = false;
+  if (ld->round.B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
   if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (launch_lmhead(p, op, ctx->lm_tok, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (launch_epilogue(p, SPECSTEER_F32, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (launch_lmhead_recover(p, op, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += 3;
+  return SPECSTEER_OK;
+}
+
+// The same round with the heads split along the vocabulary over several GPUs (a tensor-parallel LM head).
+specsteer_status specsteer_lmhead_shard_local(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, int32_t vocab_offset,
+                                              void* row_partials, void* cuda_stream) {
+  RoundParams p;
+  LmheadOperands op;
+  specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
+  if (st != SPECSTEER_OK) return st;
+  if (!row_partials || vocab_offset < 0 || ld->round.B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
+  ctx->verified = false;
+  ctx->shard_streamed = false;
+  if (ld->round.B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  cudaStream_t s = (cudaStream_t)cuda_stream;
+  p.vocab_offset = vocab_offset;
+  p.vocab_total = vocab_offset + ld->round.V;
+  // the "token met" words must start at zero: a token outside this shard leaves its row untouched
+  if (cudaMemsetAsync(ctx->lm_tok, 0, (size_t)ld->round.B * (ld->round.K + 1) * 16, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_lmhead(p, op, ctx->lm_tok, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_shard_rows(p, SPECSTEER_F32, (ShardPartial*)row_partials, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 2;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_lmhead_shard_combine(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, const void* gathered,
+                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                                int32_t vocab_total, void* cuda_stream) {
+  RoundParams p;
+  LmheadOperands op;
+  specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
+  if (st != SPECSTEER_OK) return st;
+  if ((st = check_shard_args(&ld->round, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
+  if (ld->round.B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  p.shard_parts = (const ShardPartial*)gathered;
+  p.n_shards = n_shards; p.shard_rank = shard_rank;
+  p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;
+  p.tok_logits = nullptr;   // the tokens' logits travel inside the partials
+  if (launch_epilogue(p, SPECSTEER_F32, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
+  return SPECSTEER_OK;
+}
+
+specsteer_status specsteer_lmhead_shard_recover(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, const void* gathered,
+                                                int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
+                                                int32_t vocab_total, void* cuda_stream) {
+  RoundParams p;
+  LmheadOperands op;
+  specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
+  if (st != SPECSTEER_OK) return st;
+  if ((st = check_shard_args(&ld->round, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
+  if (ld->round.B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  p.shard_parts = (const ShardPartial*)gathered;
+  p.n_shards = n_shards; p.shard_rank = shard_rank;
+  p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;
+  if (launch_lmhead_recover(p, op, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
   return SPECSTEER_OK;
 }
 

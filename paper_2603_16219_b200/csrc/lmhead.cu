@@ -37,6 +37,7 @@ constexpr int kSmemBytes = kGroups * kGroupBytes + 1024 /* alignment */ + 512 /*
 struct LmKernelParams {
   int R, V, K, d_llm, d_slm, n_chunks;
   int shared_head;    // h_SLM+ and h_SLM- use the same head: its tile is loaded once for both products
+  int vocab_offset;   // the heads passed are rows [vocab_offset, vocab_offset + V) of the full heads (0 if whole)
   const int* draft_tokens;
   const int* draft_len;
   const float* beta;
@@ -313,7 +314,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
         c = kLog2e / p.temperature[b];
         int len = p.draft_len[b];
         if (len < 0 || len > p.K) len = 0;
-        if (t < len) tok = p.draft_tokens[(long long)b * p.K + t];
+        if (t < len) tok = p.draft_tokens[(long long)b * p.K + t] - p.vocab_offset;   // id within the heads passed
       }
       bool ok = !aborted(sh) && mbar_wait(&sh->tmem_full, (uint32_t)(ti & 1));
       ok = __all_sync(kFullMask, ok);
@@ -342,7 +343,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
 #pragma unroll
           for (int j = 0; j < 32; ++j)
             if (j == jj) { tl = L[j]; tp = P[j]; tm = M[j]; }
-          *reinterpret_cast<uint4*>(p.tok_logits + (long long)row * 4) = make_uint4(tl, tp, tm, 0u);
+          *reinterpret_cast<uint4*>(p.tok_logits + (long long)row * 4) = make_uint4(tl, tp, tm, 1u)  /* fourth word: the token lies in these heads */;
         }
       }
       float ref[4], nref[4], s[4] = {0.f, 0.f, 0.f, 0.f};
@@ -387,6 +388,8 @@ struct LmRecShared {
   double warp_tot[kRecT / 32];
   double base, target, W;
   int jstar, jlast, tok_min, tok_last;
+  int plan_owner;               // sharded heads: the shard that holds the CDF target, -1 if nothing can be sampled
+  double plan_target, plan_W;   // the target within that shard, and the weight of the whole row
 };
 
 __device__ __forceinline__ double block_excl_scan_rec(double v, double* warp_tot, int tid) {
@@ -463,7 +466,38 @@ __global__ void __launch_bounds__(kRecT) lmhead_recover_kernel(const RoundParams
     *reinterpret_cast<uint4*>(xm + i) = __ldg(reinterpret_cast<const uint4*>(op.x_minus + row * dS + i));
   }
   if (tid == 0) { sh.jstar = 0x7fffffff; sh.jlast = -1; sh.tok_min = 0x7fffffff; sh.tok_last = -1; }
+  if (p.n_shards > 0 && tid == 0) {
+    // Heads split along the vocabulary: every rank holds every shard's partial of this row, so all of them place
+    // the target identically: shard weights in shard order, the target u*W, the first shard whose cumulative weight
+    // exceeds it (else the last shard of positive weight).
+    double Wg[SPECSTEER_MAX_SHARDS], W = 0.0;
+    for (int g = 0; g < p.n_shards; ++g) {
+      const ShardPartial& sp = p.shard_parts[((long long)g * p.B + b) * K1 + n];
+      Wg[g] = (sp.m[Q_R] == kNegInf) ? 0.0 : sp.s[Q_R] * exp2((double)sp.m[Q_R] - lseR);
+      W += Wg[g];
+    }
+    const double tgt = (double)p.u_recover[b] * W;
+    double cum = 0.0, base = 0.0, base_last = 0.0;
+    int owner = -1, last = -1;
+    for (int g = 0; g < p.n_shards; ++g) {
+      if (Wg[g] > 0.0) { last = g; base_last = cum; }
+      if (cum + Wg[g] > tgt) { owner = g; base = cum; break; }
+      cum += Wg[g];
+    }
+    if (owner < 0) { owner = last; base = base_last; }
+    sh.plan_owner = (W > 0.0 && W == W) ? owner : -1;
+    sh.plan_target = fmax(tgt - base, 0.0);
+    sh.plan_W = W;
+  }
   __syncthreads();
+  if (p.n_shards > 0 && sh.plan_owner != p.shard_rank) {   // another shard (or nobody) samples: values a MAX-reduce ignores
+    if (tid == 0) {
+      if (p.rec_token) p.rec_token[b] = -1;
+      if (p.rec_logprob) p.rec_logprob[b] = sh.plan_owner < 0 ? __int_as_float(0x7fc00000) : kNegInf;
+      if (p.n_out) p.n_out[b] = n;
+    }
+    return;
+  }
 
   // ---- the chunk that holds the CDF target: first chunk whose inclusive cumulative weight exceeds u*W, else the
   // last chunk of positive weight
@@ -472,7 +506,10 @@ __global__ void __launch_bounds__(kRecT) lmhead_recover_kernel(const RoundParams
   double local = 0.0;
   for (int j = j0; j < j1; ++j) local += cw[j];
   const double excl = block_excl_scan_rec(local, sh.warp_tot, tid);
-  if (tid == kRecT - 1) { sh.W = excl + local; sh.target = (double)p.u_recover[b] * (excl + local); }
+  if (tid == kRecT - 1) {
+    sh.W = p.n_shards > 0 ? sh.plan_W : excl + local;
+    sh.target = p.n_shards > 0 ? sh.plan_target : (double)p.u_recover[b] * (excl + local);
+  }
   __syncthreads();
   const double target = sh.target;
   {
@@ -523,9 +560,9 @@ __global__ void __launch_bounds__(kRecT) lmhead_recover_kernel(const RoundParams
   __syncthreads();
   const int tok = sh.tok_min != 0x7fffffff ? sh.tok_min : sh.tok_last;
   if (tid < kBN && tok == v && tok >= 0) {
-    if (p.rec_token) p.rec_token[b] = tok;
+    if (p.rec_token) p.rec_token[b] = tok + p.vocab_offset;
     if (p.rec_logprob) p.rec_logprob[b] = (float)(y2 * 0.6931471805599453 - log(sh.W));
-    if (p.out_tokens) p.out_tokens[(long long)b * K1 + n] = tok;
+    if (p.out_tokens) p.out_tokens[(long long)b * K1 + n] = tok + p.vocab_offset;
     if (p.n_out) p.n_out[b] = n + 1;
   }
   if (tok < 0 && tid == 0) {  // no positive weight anywhere in the chunk: nothing can be sampled
@@ -581,6 +618,7 @@ cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float*
   k.draft_tokens = p.draft_tokens; k.draft_len = p.draft_len; k.beta = p.beta; k.temperature = p.temperature;
   k.part = p.part; k.tok_logits = tok_logits; k.dev_error = p.dev_error;
   k.shared_head = (op.w_plus == op.w_minus) ? 1 : 0;
+  k.vocab_offset = p.vocab_offset;
   static bool attr_set[64] = {};
   if (li.device < 64 && !attr_set[li.device]) {
     cudaError_t e = cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);

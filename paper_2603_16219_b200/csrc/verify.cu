@@ -910,7 +910,13 @@ __global__ void __launch_bounds__(kEpiWarps * 32) shard_rows_kernel(const RoundP
       for (int q = 0; q < 4; ++q) { sp.m[q] = M[q]; sp.s[q] = S[q]; }
       if (t < len) {
         const int y = p.draft_tokens[(long long)b * K + t] - p.vocab_offset;   // id within this shard
-        if (y >= 0 && y < p.V) {
+        if (p.tok_logits) {   // fused LM heads: the tensor-core pass left the token's logits, if it met the token
+          const float4 g = ld_cg_f4(p.tok_logits + row * 4);
+          if (y >= 0 && y < p.V && __float_as_uint(g.w) != 0u) {
+            sp.tok_logit[0] = g.x; sp.tok_logit[1] = g.y; sp.tok_logit[2] = g.z;
+            sp.has_token = 1;
+          }
+        } else if (y >= 0 && y < p.V) {
           const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
           sp.tok_logit[0] = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
           sp.tok_logit[1] = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);

@@ -92,3 +92,20 @@ def sharded_vocab_round(ctx, desc, outputs: Dict[str, torch.Tensor], vocab_offse
     ctx.shard_recover_local(desc, gathered, rank, vocab_offset, vocab_total, stream)
     reduce_recovered(outputs, dist)
     return gathered
+
+
+def sharded_lmhead_round(ctx, desc, outputs: Dict[str, torch.Tensor], vocab_offset: int, vocab_total: int, dist,
+                         stream=None) -> torch.Tensor:
+    """One verify + recover round on hidden states and heads whose rows (the vocabulary) are split across the ranks
+    of `dist`: `desc` (an LM-head descriptor) describes this rank's rows of the heads (round.V = local count;
+    draft_tokens hold global ids) and points at `outputs`.  Same collectives as `sharded_vocab_round`; every rank
+    ends with identical outputs.  Returns the gathered partials."""
+    rank = dist.get_rank()
+    r = desc.round
+    parts = torch.empty((r.B, r.K + 1, 64), dtype=torch.uint8, device=outputs["accept_len"].device)
+    ctx.lmhead_shard_local(desc, vocab_offset, parts, stream)
+    gathered = gather_partials(parts, dist)
+    ctx.lmhead_shard_combine(desc, gathered, rank, vocab_offset, vocab_total, stream)
+    ctx.lmhead_shard_recover(desc, gathered, rank, vocab_offset, vocab_total, stream)
+    reduce_recovered(outputs, dist)
+    return gathered

@@ -115,3 +115,76 @@ def test_vocab_range_covers_every_id_once():
         assert spans[0][0] == 0 and spans[-1][1] == V
         assert all(spans[i][1] == spans[i + 1][0] for i in range(world - 1))
         assert all(lo % align == 0 for lo, hi in spans if hi > lo)
+
+
+class _FakeShardCtx:
+    """Stands in for the CUDA context in the sharded-round helpers: records the order of the calls and plays the
+    kernels' part on CPU tensors (rank r's partial is filled with r + 1; rank 0 owns the targets)."""
+
+    def __init__(self, rank, outputs, prefix):
+        self.rank, self.outputs, self.prefix, self.calls = rank, outputs, prefix, []
+
+    def _local(self, desc, vocab_offset, parts, stream=None):
+        self.calls.append(("local", vocab_offset))
+        parts.fill_(self.rank + 1)
+
+    def _combine(self, desc, gathered, rank, vocab_offset, vocab_total, stream=None):
+        self.calls.append(("combine", rank, vocab_offset, vocab_total, tuple(gathered.shape)))
+        self.outputs["accept_len"].fill_(int(gathered[:, 0, 0, 0].sum()))     # the same on every rank
+
+    def _recover(self, desc, gathered, rank, vocab_offset, vocab_total, stream=None):
+        self.calls.append(("recover", rank))
+        own = rank == 0
+        self.outputs["rec_token"].fill_(11 if own else -1)
+        self.outputs["rec_logprob"].fill_(-1.5 if own else float("-inf"))
+        self.outputs["out_tokens"].fill_(11 if own else -1)
+        self.outputs["n_out"].fill_(1 if own else 0)
+
+    _NAMES = {"shard_verify_local": "_local", "shard_verify_combine": "_combine", "shard_recover_local": "_recover",
+              "lmhead_shard_local": "_local", "lmhead_shard_combine": "_combine", "lmhead_shard_recover": "_recover"}
+
+    def __getattr__(self, name):
+        if name in self._NAMES and name.startswith(self.prefix):
+            return getattr(self, self._NAMES[name])
+        raise AttributeError(name)
+
+
+def _round_worker(rank, world, port, q):
+    import types
+    import torch.distributed as dist
+    from paper_2603_16219_b200 import sharding
+    dist.init_process_group("gloo", init_method="tcp://127.0.0.1:%d" % port, rank=rank, world_size=world)
+    try:
+        ok = True
+        for helper, prefix, desc in (
+                (sharding.sharded_vocab_round, "shard", types.SimpleNamespace(B=2, K=3)),
+                (sharding.sharded_lmhead_round, "lmhead_shard", types.SimpleNamespace(round=types.SimpleNamespace(B=2, K=3)))):
+            outs = {"accept_len": torch.zeros(2, dtype=torch.int32), "rec_token": torch.zeros(2, dtype=torch.int32),
+                    "rec_logprob": torch.zeros(2), "out_tokens": torch.zeros(2, 4, dtype=torch.int32),
+                    "n_out": torch.zeros(2, dtype=torch.int32)}
+            fake = _FakeShardCtx(rank, outs, prefix)
+            gathered = helper(fake, desc, outs, 100 * rank, 200, dist)
+            ok = ok and tuple(gathered.shape) == (world, 2, 4, 64) and [c[0] for c in fake.calls] == ["local", "combine", "recover"]
+            ok = ok and fake.calls[0][1] == 100 * rank and fake.calls[1][1:4] == (rank, 100 * rank, 200)
+            ok = ok and outs["accept_len"].tolist() == [3, 3]            # partials of rank 0 (1) and rank 1 (2)
+            ok = ok and outs["rec_token"].tolist() == [11, 11] and outs["n_out"].tolist() == [1, 1]
+            ok = ok and outs["rec_logprob"].tolist() == [-1.5, -1.5] and bool((outs["out_tokens"] == 11).all())
+        q.put((rank, ok))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_sharded_round_helpers_call_order_and_collectives_on_two_ranks():
+    """Both sharded rounds (logit shards, fused LM-head shards): local pass, all-gather, combine, recover, MAX
+    all-reduce - with the kernels replaced by a stand-in, on two gloo ranks."""
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = _free_port()
+    procs = [ctx.Process(target=_round_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    res = sorted(q.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+    assert res == [(0, True), (1, True)]
