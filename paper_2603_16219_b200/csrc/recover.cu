@@ -369,7 +369,8 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   const float c = kLog2e / p.temperature[b];
   const int per = (((p.V + S - 1) / S) + 7) & ~7;
   const int v0 = sp * per, v1 = min(p.V, v0 + per);
-  u64 best = 0;  // below every key of a real entry
+  float best_r = 0.f;   // the thread walks its entries in ascending id order, so "strictly larger" keeps the lowest id
+  int best_v = -1;
   OnlineLse acc = {kNegInf, 0.f};
   float mx[3] = {kNegInf, kNegInf, kNegInf};   // largest entry of each stream
   bool bad = false;                            // a NaN or +inf entry
@@ -390,10 +391,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       r[i] = fmaf(beta, q[i] - m[i], l[i]);   // Eq. 8
-      if (i < n) {
-        const u64 k = entry_key(r[i], v + i);
-        best = k > best ? k : best;
-      }
+      if (i < n && (best_v < 0 || r[i] > best_r)) { best_r = r[i]; best_v = v + i; }
     }
     if (LSE) {
       float x[8];
@@ -418,6 +416,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
       }
     }
   }
+  u64 best = best_v >= 0 ? entry_key(best_r, best_v) : 0;   // 0 is below every key of a real entry
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
     const u64 other = __shfl_xor_sync(kFullMask, best, o);
