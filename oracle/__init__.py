@@ -8,6 +8,12 @@ does, and this package imports nothing from the product.
 
 Inputs are numpy arrays (bf16 logits as ``uint16`` bit patterns); outputs come
 back as a dict of numpy arrays, floating point in float64.
+
+Also here: the top-k split recovery of the deployment appendix (``cloud_topk_row``,
+``edge_resample_row``, ``topk_recover_round``) and the LM-head step in front of the
+round (``lmhead_logits``: h = x W^T in float64 from bf16 operands;
+``lmhead_verify_recover_round``).  Every function is pinned
+(tests/test_oracle_pins.py, test_oracle_topk_pins.py, test_oracle_lmhead_pins.py).
 """
 from __future__ import annotations
 

@@ -15,13 +15,20 @@
  *   - Eq. 6 (exact rule):   alpha = min(1, P*(y) / P_SLM+(y)) with the true Z_t.
  *   - Eq. 2-4 (fused target): P* = P_LLM * exp(r) / Z_t, r = log P+ - log P-.
  *   - Eq. 8 (recovery logits): h_rec = h_LLM + beta * (h_SLM+ - h_SLM-).
+ *   - Greedy decoding (the experimental settings): ORACLE_RECOVER_ARGMAX takes the
+ *     token of largest h_rec instead of sampling; the order is decided on h_rec as
+ *     single precision forms it (see one_request).
  * Every distribution is a softmax of logits divided by a per-request
- * temperature (the paper runs at temperature 1).
+ * temperature (the paper runs at temperature 1).  Logits may also be given in
+ * double (ORACLE_DTYPE_F64): the LM-head oracle in __init__.py forms them as
+ * x W^T in float64 and hands them to the same round.
  *
  * Pins (tests/test_oracle_pins.py, tests/golden/): special cases that reduce
  * to library log-softmax, hand-derived rational examples, the output-token law
  * by enumeration and Monte-Carlo, and the speculative-sampling theorem for the
- * EXACT_Z + RESIDUAL pair.  Parts with no pin: none of the functions below.
+ * EXACT_Z + RESIDUAL pair; greedy recovery by exact rationals, numpy argmax and
+ * a float32 tie; the float64 logit decode and the LM-head step in
+ * tests/test_oracle_lmhead_pins.py.  Parts with no pin: none of the functions below.
  *
  * No blocking, fusion or reordering: each log-sum-exp is "max, then sum of
  * exp(x - max)" over the row in vocabulary order; the sampler walks the CDF in
