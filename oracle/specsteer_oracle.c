@@ -246,20 +246,34 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
       /* Greedy decoding (the paper's experimental setting): y_new is the token of largest h_rec (Eq. 8), the lowest
        * id among equals, on the rejection row and on the bonus row alike.  The comparison is made on h_rec as single
        * precision forms it, fl(h_LLM + beta * fl(h_SLM+ - h_SLM-)) with one fused multiply-add, so that ties are the
-       * same everywhere; the temperature does not change the order.  Its log-probability is the one under
+       * same everywhere (float32 and bf16 logits); the temperature does not change the order.  Its log-probability is the one under
        * Softmax(h_rec / T). */
-      const float beta32 = a->beta[b];
-      float best = -INFINITY;
-      for (int v = 0; v < V; ++v) {
-        float l = (float)logit_at(a->h_llm, a->dtype, off + v), pp = (float)logit_at(a->h_slm_plus, a->dtype, off + v),
-              mm = (float)logit_at(a->h_slm_minus, a->dtype, off + v);
-        float r = fmaf(beta32, pp - mm, l);
-        if (rec_token < 0 || r > best) { best = r; rec_token = v; }
+      double gap = INFINITY;   /* reported in cdf_margin: distance to the runner-up where the order is not exact */
+      if (a->dtype == ORACLE_DTYPE_F64) {
+        /* logits that were themselves computed (the LM-head path): nobody can reproduce their last bits, so the
+         * order is taken in double and the gap between the two largest values is reported for the comparison */
+        double best = -INFINITY, second = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+          double r = logit_at(a->h_llm, a->dtype, off + v) +
+                     beta * (logit_at(a->h_slm_plus, a->dtype, off + v) - logit_at(a->h_slm_minus, a->dtype, off + v));
+          if (rec_token < 0 || r > best) { second = best; best = r; rec_token = v; }
+          else if (r > second) second = r;
+        }
+        gap = best - second;
+      } else {
+        const float beta32 = a->beta[b];
+        float best = -INFINITY;
+        for (int v = 0; v < V; ++v) {
+          float l = (float)logit_at(a->h_llm, a->dtype, off + v), pp = (float)logit_at(a->h_slm_plus, a->dtype, off + v),
+                mm = (float)logit_at(a->h_slm_minus, a->dtype, off + v);
+          float r = fmaf(beta32, pp - mm, l);
+          if (rec_token < 0 || r > best) { best = r; rec_token = v; }
+        }
       }
       rec_logprob = w->r[rec_token] - w->lseR;
       if (a->out_tokens) a->out_tokens[(int64_t)b * (K + 1) + n] = rec_token;
       n_out = n + 1;
-      if (a->cdf_margin) a->cdf_margin[b] = INFINITY;   /* no uniform is involved */
+      if (a->cdf_margin) a->cdf_margin[b] = gap;   /* no uniform is involved */
       if (a->rec_token_lo) a->rec_token_lo[b] = rec_token;
       if (a->rec_token_hi) a->rec_token_hi[b] = rec_token;
       goto done;
@@ -299,7 +313,6 @@ done:
 int specsteer_oracle_round(const oracle_round_args *a) {
   if (!a || a->B < 0 || a->K < 0 || a->V <= 0 || a->ld_row < a->V || !a->accept_len) return -1;
   if (a->ld_req < (int64_t)(a->K + 1) * a->ld_row) return -1;
-  if (a->recover_mode == ORACLE_RECOVER_ARGMAX && a->dtype == ORACLE_DTYPE_F64) return -3;  /* defined on float32 values */
   int nthreads = a->nthreads > 0 ? a->nthreads : 1;
   int failed = 0;
 #ifdef _OPENMP

@@ -423,10 +423,28 @@ def test_argmax_recovery_decides_on_single_precision_values(oracle_mod):
     assert _round(o, L, P, M, **kw)["rec_token"][0] == 1
 
 
-def test_argmax_recovery_is_not_defined_for_float64_logits(oracle_mod):
+def test_argmax_recovery_on_float64_logits_orders_in_double_and_reports_the_gap(oracle_mod):
+    """Logits that were themselves computed (float64): numpy's argmax of h_rec in double, lowest id among equals, and
+    the distance to the runner-up in cdf_margin (float32 logits report +inf there: their order is exact)."""
     o = oracle_mod
-    L = np.zeros((1, 1, 4))
-    with pytest.raises(RuntimeError):
-        o.verify_recover_round(L, L, L, np.zeros((1, 0), np.int32), np.zeros(1, np.int32), np.ones(1, np.float32),
-                               np.ones(1, np.float32), np.ones(1, np.float32), np.zeros((1, 0), np.float32),
-                               np.zeros(1, np.float32), recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
+    rng = np.random.default_rng(43)
+    B, V = 4, 3001
+    L, P, M = (rng.standard_normal((B, 1, V)) * 2 for _ in range(3))
+    L[1, 0, 77] = L[1, 0, 2000] = 50.0                  # an exact tie between two ids: the lower one, gap 0
+    P[1, 0, 77] = P[1, 0, 2000] = M[1, 0, 77] = M[1, 0, 2000] = 0.0
+    beta = np.array([1.0, 0.5, 2.0, 0.0], np.float32)
+    g = o.verify_recover_round(L, P, M, np.zeros((B, 0), np.int32), np.zeros(B, np.int32), np.ones(B, np.float32), beta,
+                               np.ones(B, np.float32), np.zeros((B, 0), np.float32), np.zeros(B, np.float32),
+                               recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
+    for b in range(B):
+        r = L[b, 0] + float(beta[b]) * (P[b, 0] - M[b, 0])
+        assert g["rec_token"][b] == int(np.argmax(r))
+        top2 = np.sort(r)[-2:]
+        assert g["cdf_margin"][b] == pytest.approx(top2[1] - top2[0], abs=1e-15)
+        assert g["rec_logprob"][b] == pytest.approx(sps.log_softmax(r)[g["rec_token"][b]], abs=1e-12)
+    assert g["rec_token"][1] == 77 and g["cdf_margin"][1] == 0.0
+    f = o.verify_recover_round(L.astype(np.float32), P.astype(np.float32), M.astype(np.float32), np.zeros((B, 0), np.int32),
+                               np.zeros(B, np.int32), np.ones(B, np.float32), beta, np.ones(B, np.float32),
+                               np.zeros((B, 0), np.float32), np.zeros(B, np.float32), recover_mode=o.RECOVER_ARGMAX,
+                               flags=o.FLAG_BONUS)
+    assert np.isinf(f["cdf_margin"]).all()
