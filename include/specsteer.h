@@ -66,7 +66,9 @@ typedef enum {
                                      h_rec is compared as float32 forms it, fl(h_LLM + beta * fl(h_SLM+ - h_SLM-)) with
                                      one fused multiply-add; u_recover is not used; rec_logprob is its log-probability
                                      under Softmax(h_rec / T).  One more pass over row accept_len of every request
-                                     that takes a token.  Not available in the sharded and LM-head rounds. */
+                                     that takes a token (in the LM-head round: none, the tensor-core pass leaves the
+                                     largest h_rec of every tile; the order is then that of its float32 accumulators).
+                                     Not available in the sharded rounds. */
 } specsteer_recover_mode;
 
 enum {
@@ -213,9 +215,9 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx *ctx, const specste
  *     ld_row, ld_req and dtype are ignored.  Every output may be requested; every row of every request is computed.
  *   - x_*: DEVICE, bf16, [B][K+1][d] dense; w_*: DEVICE, bf16, [V][d] dense (row v = the head's weights of token v);
  *     all 16-byte aligned, d_llm and d_slm multiples of 8.  w_slm_plus and w_slm_minus may be the same pointer.
- *   - RATIO or EXACT_Z acceptance, STEER recovery (RESIDUAL: UNSUPPORTED).
+ *   - RATIO or EXACT_Z acceptance, STEER or ARGMAX recovery (RESIDUAL: UNSUPPORTED).
  *   - The first call allocates a second workspace for the context's maxima
- *     (max_B*(max_K+1)*(16 + 32*ceil(max_V/128)) bytes); later calls allocate nothing.
+ *     (max_B*(max_K+1)*(16 + 40*ceil(max_V/128)) bytes); later calls allocate nothing.
  *   - Accuracy: the logits carry the rounding of a float32 accumulation over d bf16 products, so decisions may
  *     differ from exact arithmetic where their margin is below about 1e-4.
  * Three launches; stream-ordered; specsteer_ctx_time_streaming brackets the tensor-core kernel.

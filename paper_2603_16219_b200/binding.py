@@ -199,7 +199,7 @@ def make_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor],
 
 
 def make_lmhead_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor], *, accept_mode=ACCEPT_RATIO,
-                     flags=0) -> LmheadDesc:
+                     recover_mode=RECOVER_STEER, flags=0) -> LmheadDesc:
     """Descriptor of a round on hidden states and head weights: inputs hold x_llm [B, K+1, d_llm], w_llm [V, d_llm],
     x_slm_plus / x_slm_minus [B, K+1, d_slm], w_slm_plus / w_slm_minus [V, d_slm] (bf16, contiguous) and the
     per-request tensors of ``make_desc``."""
@@ -217,7 +217,7 @@ def make_lmhead_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.T
     d = ld.round
     d.B, d.K, d.V = B, K, V
     d.ld_row, d.ld_req, d.dtype = V, K1 * V, F32
-    d.accept_mode, d.recover_mode, d.flags = int(accept_mode), RECOVER_STEER, int(flags)
+    d.accept_mode, d.recover_mode, d.flags = int(accept_mode), int(recover_mode), int(flags)
 
     def ptr(t, dt, n):
         if t.dtype != dt or not t.is_contiguous() or t.numel() != n:

@@ -42,6 +42,7 @@ struct specsteer_ctx {
   void* lm_ws;
   float* lm_part;
   float* lm_tok;
+  void* lm_keys;      // [rows][chunks of 128] per-tile keys of the largest h_rec, for greedy recovery
 };
 
 static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
@@ -384,7 +385,7 @@ specsteer_status prep_lmhead(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld
   const specsteer_round_desc* d = &ld->round;
   if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
   if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
+  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_ARGMAX) return SPECSTEER_ERR_UNSUPPORTED;
   if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
   if (ld->d_llm <= 0 || ld->d_slm <= 0) return SPECSTEER_ERR_INVALID_ARG;
   if (ld->d_llm % 8 || ld->d_slm % 8) return SPECSTEER_ERR_UNSUPPORTED;   // rows of the operands must be 16-byte multiples
@@ -407,10 +408,12 @@ specsteer_status prep_lmhead(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld
     const size_t rows = (size_t)ctx->max_B * (ctx->max_K + 1);
     const size_t part_bytes = align_up(rows * (size_t)n_chunks_of(ctx->max_V, kLmheadChunk) * 32, 256);
     const size_t tok_bytes = align_up(rows * 16, 256);
-    if (cudaMalloc(&ctx->lm_ws, part_bytes + tok_bytes) != cudaSuccess) { ctx->lm_ws = nullptr; (void)cudaGetLastError(); return SPECSTEER_ERR_WORKSPACE; }
+    const size_t key_bytes = align_up(rows * (size_t)n_chunks_of(ctx->max_V, kLmheadChunk) * 8, 256);
+    if (cudaMalloc(&ctx->lm_ws, part_bytes + tok_bytes + key_bytes) != cudaSuccess) { ctx->lm_ws = nullptr; (void)cudaGetLastError(); return SPECSTEER_ERR_WORKSPACE; }
     ctx->lm_part = (float*)ctx->lm_ws;
     ctx->lm_tok = (float*)((char*)ctx->lm_ws + part_bytes);
-    ctx->ws_bytes += part_bytes + tok_bytes;
+    ctx->lm_keys = (char*)ctx->lm_ws + part_bytes + tok_bytes;
+    ctx->ws_bytes += part_bytes + tok_bytes + key_bytes;
   }
   specsteer_round_desc dd = *d;
   dd.dtype = SPECSTEER_F32; dd.ld_row = d->V; dd.ld_req = (int64_t)K1 * d->V;   // no logit tensor exists
@@ -442,10 +445,11 @@ specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhe
   if (!g.ok) return SPECSTEER_ERR_CUDA;
   cudaStream_t s = (cudaStream_t)cuda_stream;
   if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-  if (launch_lmhead(p, op, ctx->lm_tok, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  const bool greedy = ld->round.recover_mode == SPECSTEER_RECOVER_ARGMAX;
+  if (launch_lmhead(p, op, ctx->lm_tok, greedy ? ctx->lm_keys : nullptr, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (launch_epilogue(p, SPECSTEER_F32, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-  if (launch_lmhead_recover(p, op, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if ((greedy ? launch_lmhead_argmax(p, ctx->lm_keys, s) : launch_lmhead_recover(p, op, s)) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += 3;
   return SPECSTEER_OK;
 }
@@ -458,6 +462,7 @@ specsteer_status specsteer_lmhead_shard_local(specsteer_ctx* ctx, const specstee
   specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
   if (st != SPECSTEER_OK) return st;
   if (!row_partials || vocab_offset < 0 || ld->round.B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
+  if (ld->round.recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
   ctx->verified = false;
   ctx->shard_streamed = false;
   if (ld->round.B == 0) return SPECSTEER_OK;
@@ -469,7 +474,7 @@ specsteer_status specsteer_lmhead_shard_local(specsteer_ctx* ctx, const specstee
   // the "token met" words must start at zero: a token outside this shard leaves its row untouched
   if (cudaMemsetAsync(ctx->lm_tok, 0, (size_t)ld->round.B * (ld->round.K + 1) * 16, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-  if (launch_lmhead(p, op, ctx->lm_tok, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_lmhead(p, op, ctx->lm_tok, nullptr, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (launch_shard_rows(p, SPECSTEER_F32, (ShardPartial*)row_partials, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += 2;
@@ -484,6 +489,7 @@ specsteer_status specsteer_lmhead_shard_combine(specsteer_ctx* ctx, const specst
   specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
   if (st != SPECSTEER_OK) return st;
   if ((st = check_shard_args(&ld->round, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
+  if (ld->round.recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
   if (ld->round.B == 0) return SPECSTEER_OK;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
@@ -504,6 +510,7 @@ specsteer_status specsteer_lmhead_shard_recover(specsteer_ctx* ctx, const specst
   specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
   if (st != SPECSTEER_OK) return st;
   if ((st = check_shard_args(&ld->round, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
+  if (ld->round.recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
   if (ld->round.B == 0) return SPECSTEER_OK;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;

@@ -88,8 +88,12 @@ struct LaunchInfo {
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
                           int* n_launches, cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
 // The tensor-core pass: partial records of every row at kLmheadChunk entries per chunk, and tok_logits.
-cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, const LaunchInfo& li,
-                          cudaStream_t s);
+// argmax_keys: [B*(K+1)][n_chunks] 64-bit words that receive, per tile, the key of the largest h_rec (greedy recovery),
+// or null when nobody needs them.
+cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, void* argmax_keys,
+                          const LaunchInfo& li, cudaStream_t s);
+// Greedy recovery from those keys.
+cudaError_t launch_lmhead_argmax(const RoundParams& p, const void* argmax_keys, cudaStream_t s);
 // Recovery (Eq. 8) from those records; the logits of the one chunk that holds the CDF target are recomputed.
 cudaError_t launch_lmhead_recover(const RoundParams& p, const LmheadOperands& op, cudaStream_t s);
 constexpr int kTopkMaxSplit = 16;  // CTAs that may share one row in specsteer_cloud_topk

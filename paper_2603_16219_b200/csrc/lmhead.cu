@@ -43,7 +43,8 @@ struct LmKernelParams {
   const float* beta;
   const float* temperature;
   float* part;        // [R][n_chunks][8]
-  float* tok_logits;  // [R][4]: the drafted token's h_LLM, h_SLM+, h_SLM- (and one unused word)
+  float* tok_logits;  // [R][4]: the drafted token's h_LLM, h_SLM+, h_SLM- and a "token met" word
+  u64* argmax_keys;   // [R][n_chunks]: per tile the key of the largest h_rec (greedy recovery), or null
   int* dev_error;
 };
 
@@ -120,13 +121,14 @@ __device__ __forceinline__ void set_abort(LmShared* sh, int* dev_error) {
 // One slice of 32 columns of the three accumulators: running maxima of the four scaled quantities.
 template <bool MASKED>
 __device__ __forceinline__ void slice_max(const uint32_t (&L)[32], const uint32_t (&P)[32], const uint32_t (&M)[32], float beta,
-                                          int nv, float (&mx)[4]) {
+                                          int nv, float (&mx)[4], int jbase, int& arg_r) {
 #pragma unroll
   for (int j = 0; j < 32; ++j) {
     if (MASKED && j >= nv) break;
     const float l = __uint_as_float(L[j]), p = __uint_as_float(P[j]), m = __uint_as_float(M[j]);
     const float r = fmaf(beta, p - m, l);  // Eq. 8
-    mx[Q_L] = fmaxf(mx[Q_L], l); mx[Q_P] = fmaxf(mx[Q_P], p); mx[Q_M] = fmaxf(mx[Q_M], m); mx[Q_R] = fmaxf(mx[Q_R], r);
+    mx[Q_L] = fmaxf(mx[Q_L], l); mx[Q_P] = fmaxf(mx[Q_P], p); mx[Q_M] = fmaxf(mx[Q_M], m);
+    if (r > mx[Q_R]) { mx[Q_R] = r; arg_r = jbase + j; }   // ascending columns: the first maximiser stays
   }
 }
 template <bool MASKED>
@@ -329,14 +331,15 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
       const int n_valid = min(kBN, p.V - n0);
       // pass 1: maxima of the four quantities, and the drafted token's logits if they are in this tile
       float mx[4] = {kNegInf, kNegInf, kNegInf, kNegInf};
+      int arg_r = -1;   // column of the tile's largest h_rec (greedy recovery)
 #pragma unroll 1
       for (int j0 = 0; j0 < kBN; j0 += 32) {
         uint32_t L[32], P[32], M[32];
         tmem_ld32(t_l + j0, L); tmem_ld32(t_p + j0, P); tmem_ld32(t_m + j0, M);
         tmem_ld_wait();
         const int nv = n_valid - j0;
-        if (nv >= 32) slice_max<false>(L, P, M, beta, 32, mx);
-        else if (nv > 0) slice_max<true>(L, P, M, beta, nv, mx);
+        if (nv >= 32) slice_max<false>(L, P, M, beta, 32, mx, j0, arg_r);
+        else if (nv > 0) slice_max<true>(L, P, M, beta, nv, mx, j0, arg_r);
         const int jj = tok - n0 - j0;
         if (jj >= 0 && jj < 32 && jj < nv) {
           uint32_t tl = 0, tp = 0, tm = 0;
@@ -365,6 +368,8 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->tmem_empty);  // the accumulators may be overwritten
+      if (valid && p.argmax_keys)
+        p.argmax_keys[(long long)row * p.n_chunks + nb] = arg_r >= 0 ? entry_key(mx[Q_R], n0 + arg_r) : 0ull;
       if (valid) {
         const float2 rl = make_record(ref[Q_L], s[Q_L]), rp = make_record(ref[Q_P], s[Q_P]),
                      rm = make_record(ref[Q_M], s[Q_M]), rr = make_record(ref[Q_R], s[Q_R]);
@@ -604,8 +609,8 @@ bool encode_operand(CUtensorMap* tm, const void* base, int rows, int d) {
 
 }  // namespace
 
-cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, const LaunchInfo& li,
-                          cudaStream_t s) {
+cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, void* argmax_keys,
+                          const LaunchInfo& li, cudaStream_t s) {
   const int R = p.B * (p.K + 1);
   if (R == 0) return cudaSuccess;
   CUtensorMap tm[6];
@@ -617,6 +622,7 @@ cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float*
   k.R = R; k.V = p.V; k.K = p.K; k.d_llm = op.d_llm; k.d_slm = op.d_slm; k.n_chunks = p.n_chunks;
   k.draft_tokens = p.draft_tokens; k.draft_len = p.draft_len; k.beta = p.beta; k.temperature = p.temperature;
   k.part = p.part; k.tok_logits = tok_logits; k.dev_error = p.dev_error;
+  k.argmax_keys = reinterpret_cast<u64*>(argmax_keys);
   k.shared_head = (op.w_plus == op.w_minus) ? 1 : 0;
   k.vocab_offset = p.vocab_offset;
   static bool attr_set[64] = {};
@@ -629,6 +635,59 @@ cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float*
   const long long tiles = (long long)mb * nb;
   const int grid = (int)(tiles < li.sm_count ? tiles : li.sm_count);
   lmhead_kernel<<<grid, kThreads, kSmemBytes, s>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], k);
+  return cudaGetLastError();
+}
+
+// Greedy recovery on the fused path: the largest of the per-tile keys of row accept_len (value first, lower id among
+// equal values), its log-probability from the row's normaliser.
+__global__ void __launch_bounds__(256) lmhead_argmax_kernel(const RoundParams p, const u64* keys) {
+  __shared__ u64 wbest[8];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int K = p.K, K1 = K + 1;
+  pdl_wait();
+  const int n = p.accept_len[b];
+  const int status = p.status_ws[b];
+  int len = p.draft_len[b];
+  if (len < 0 || len > K) len = 0;
+  const bool bad = (status & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+  const bool sample = !bad && (n < len || (p.flags & SPECSTEER_FLAG_BONUS));
+  if (p.out_tokens)
+    for (int t = tid; t <= K; t += 256)
+      p.out_tokens[(long long)b * K1 + t] = (t < n) ? p.draft_tokens[(long long)b * K + t] : -1;
+  const long long row = (long long)b * K1 + n;
+  u64 best = 0;
+  if (sample)
+    for (int j = tid; j < p.n_chunks; j += 256) {
+      const u64 k = __ldcg(keys + row * p.n_chunks + j);
+      best = k > best ? k : best;
+    }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const u64 other = __shfl_xor_sync(kFullMask, best, o);
+    best = other > best ? other : best;
+  }
+  if (lane == 0) wbest[warp] = best;
+  __syncthreads();
+  if (tid != 0) return;
+  for (int w = 1; w < 8; ++w) best = wbest[w] > best ? wbest[w] : best;
+  if (!sample || best == 0) {
+    if (p.rec_token) p.rec_token[b] = -1;
+    if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+    if (p.n_out) p.n_out[b] = n;
+    return;
+  }
+  const int tok = (int)(0xffffffffu - (uint32_t)(best & 0xffffffffu));
+  const double r = (double)order_val((uint32_t)(best >> 32));
+  const double lseR = (double)p.lse2[row * 4 + Q_R];
+  if (p.rec_token) p.rec_token[b] = tok;
+  if (p.rec_logprob) p.rec_logprob[b] = (float)((r * (double)(kLog2e / p.temperature[b]) - lseR) * 0.6931471805599453);
+  if (p.out_tokens) p.out_tokens[(long long)b * K1 + n] = tok;
+  if (p.n_out) p.n_out[b] = n + 1;
+}
+
+cudaError_t launch_lmhead_argmax(const RoundParams& p, const void* argmax_keys, cudaStream_t s) {
+  if (p.B == 0) return cudaSuccess;
+  lmhead_argmax_kernel<<<p.B, 256, 0, s>>>(p, reinterpret_cast<const u64*>(argmax_keys));
   return cudaGetLastError();
 }
 

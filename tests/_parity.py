@@ -81,7 +81,17 @@ def compare(oracle, gpu, npin, accept_mode, recover_mode, flags, tol, V=None, se
             if g["accept_flags"][b][t] != ob["accept_flags"][t]:
                 assert ob["accept_margin"][t] < MARGIN or (force is not None and force[0, t] >= 0), (b, t)
         # ---- recovered token
-        if g["rec_token"][b] != ob["rec_token"]:
+        if g["rec_token"][b] != ob["rec_token"] and recover_mode == 2:
+            # greedy recovery on logits nobody can reproduce to the last bit (the oracle reports the gap between the
+            # two largest h_rec): another token is admissible only if it is itself within the margin of the largest
+            assert ob["rec_token"] >= 0 and g["rec_token"][b] >= 0, (b, g["rec_token"][b], ob["rec_token"])
+            assert ob["cdf_margin"] < MARGIN, (b, g["rec_token"][b], ob["rec_token"], ob["cdf_margin"])
+            n = int(ob["accept_len"])
+            r = npin["h_llm"][b, n, :V].astype(np.float64) + float(npin["beta"][b]) * (
+                npin["h_slm_plus"][b, n, :V].astype(np.float64) - npin["h_slm_minus"][b, n, :V].astype(np.float64))
+            assert r[g["rec_token"][b]] >= r.max() - MARGIN, (b, g["rec_token"][b], ob["rec_token"])
+            stats["excused_token"] += 1
+        elif g["rec_token"][b] != ob["rec_token"]:
             lo, hi = int(ob["rec_token_lo"]), int(ob["rec_token_hi"])
             assert ob["rec_token"] >= 0 and g["rec_token"][b] >= 0, (b, g["rec_token"][b], ob["rec_token"])
             assert ob["cdf_margin"] < MARGIN and lo <= g["rec_token"][b] <= hi, (

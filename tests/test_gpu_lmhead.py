@@ -278,3 +278,53 @@ def test_tiny_vocabularies_and_hidden_widths(env, V, d_llm, d_slm):
 def test_many_rows_few_vocabulary_tiles(env):
     """1024 rows = 8 row blocks over 3 vocabulary tiles: fewer tiles than SMs, every CTA at most one tile."""
     _case(env, _spec(env, 2, B=128, K=7, V=300, ragged=True), 128, 64, seed=30)
+
+
+# ------------------------------------------------------------------ greedy recovery on the fused path
+def _greedy_case(env, spec, d_llm, d_slm, seed, flags=1, accept_mode=0, mutate=None):
+    inputs = env["synth"].make_lmhead_round(spec, d_llm, d_slm, device="cuda", seed=seed)
+    if mutate:
+        mutate(inputs)
+    b = env["binding"]
+    B, K1 = inputs["x_llm"].shape[:2]
+    outs = b.alloc_outputs(B, K1 - 1, "cuda")
+    before = env["ctx"].launch_count
+    env["ctx"].lmhead_round(b.make_lmhead_desc(inputs, outs, accept_mode=accept_mode, recover_mode=b.RECOVER_ARGMAX, flags=flags))
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 3
+    gpu = {k: v.cpu().numpy() for k, v in outs.items()}
+    stats = P.compare(env["oracle"], gpu, _np_inputs(env["oracle"], inputs), accept_mode, 2, flags, TOL, margin=MARGIN)
+    return inputs, gpu, stats
+
+
+@pytest.mark.parametrize("V,d_llm,d_slm", [(3001, 320, 128), (48000, 256, 64), (100, 64, 32)])
+def test_greedy_recovery_on_the_fused_path(env, V, d_llm, d_slm):
+    """The token of largest h_rec, taken from the per-tile maxima the tensor-core pass leaves.  The order is that of
+    float32 accumulators, so a token other than the oracle's is admissible only where the two largest values are
+    within the margin (compare() checks that the token is then itself within the margin of the largest)."""
+    _, gpu, stats = _greedy_case(env, _spec(env, 1, B=12, K=4, V=V), d_llm, d_slm, seed=50 + V % 7)
+    assert (gpu["rec_token"] >= 0).all() and stats["excused_token"] <= 1
+
+
+def test_greedy_recovery_fused_ragged_no_bonus_exact_rule(env):
+    spec = _spec(env, 4, B=30, K=6, V=7000, ragged=True)
+
+    def mutate(inputs):
+        inputs["temperature"][2] = -1.0
+        inputs["draft_len"][3] = 0
+    inputs, gpu, _ = _greedy_case(env, spec, 256, 128, seed=57, flags=0, accept_mode=1, mutate=mutate)
+    assert gpu["rec_token"][2] == -1 and gpu["rec_token"][3] == -1
+    dl = inputs["draft_len"].cpu().numpy()
+    ok = np.ones(30, bool); ok[2] = False
+    assert ((gpu["rec_token"] >= 0) == (gpu["accept_len"] < dl))[ok].all()
+
+
+def test_greedy_and_sampled_fused_rounds_share_the_verification(env):
+    b = env["binding"]
+    inputs = env["synth"].make_lmhead_round(_spec(env, 0, B=16, K=3, V=9000), 192, 64, device="cuda", seed=58)
+    sampled = _run_gpu(env, inputs)
+    outs = b.alloc_outputs(16, 3, "cuda")
+    env["ctx"].lmhead_round(b.make_lmhead_desc(inputs, outs, recover_mode=b.RECOVER_ARGMAX, flags=1))
+    torch.cuda.synchronize()
+    for k in ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "logp_plus", "logp_star", "log_z", "req_status"):
+        assert np.array_equal(outs[k].cpu().numpy(), sampled[k], equal_nan=True), k
