@@ -498,7 +498,8 @@ def run_lmhead(args, local_rank):
     positions = int(inputs["draft_len"].sum().item())
     ctx = binding.Context(B, K, V, device=local_rank)
     outs = binding.alloc_outputs(B, K, dev)
-    desc = binding.make_lmhead_desc(inputs, outs, flags=binding.FLAG_BONUS)
+    desc = binding.make_lmhead_desc(inputs, outs, flags=binding.FLAG_BONUS,
+                                    recover_mode=binding.RECOVER_ARGMAX if args.greedy else binding.RECOVER_STEER)
     stream = torch.cuda.current_stream(dev)
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -539,7 +540,8 @@ def run_lmhead(args, local_rank):
     h = {n: torch.empty(B, K + 1, V, dtype=torch.float32, device=dev) for n in ("h_llm", "h_slm_plus", "h_slm_minus")}
     li = {k: inputs[k] for k in ("draft_tokens", "draft_len", "lam", "beta", "temperature", "u_accept", "u_recover")}
     li.update(h)
-    d2 = binding.make_desc(li, outs, flags=binding.FLAG_BONUS)
+    d2 = binding.make_desc(li, outs, flags=binding.FLAG_BONUS,
+                           recover_mode=binding.RECOVER_ARGMAX if args.greedy else binding.RECOVER_STEER)
     pairs = (("h_llm", "x_llm", "w_llm"), ("h_slm_plus", "x_slm_plus", "w_slm_plus"), ("h_slm_minus", "x_slm_minus", "w_slm_minus"))
 
     def unfused():
@@ -566,6 +568,7 @@ def run_lmhead(args, local_rank):
     achieved = flops / (kernel_ms * 1e-3) / 1e12
     line = {
         "workload": "%s_lmhead_dllm%d_dslm%d" % (spec.name, dL, dS), "metric": METRIC,
+        "recovery": "greedy (argmax of h_rec)" if args.greedy else "sampled",
         "value": positions / (fused_ms * 1e-3), "unit": UNIT, "ms_per_step": fused_ms, "steps": steps, "dtype": "bf16",
         "roofline": {"bound": "tensor", "kernel": "lmhead_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": None,
