@@ -179,15 +179,14 @@ specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, c
       p.sums = SUM_ALL;
       p.row_mode = ROWS_RECOVERY;
       if (launch_verify_stream(p, d->dtype, true, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-      if (launch_recovery_row_lse(p, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-      ctx->launches += 2;
+      ctx->launches += 1;
     }
     if (d->recover_mode == SPECSTEER_RECOVER_ARGMAX) {
       if (launch_recover_argmax(p, d->dtype, rows_aligned(d), lean, (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
                                 ctx->topk_count + b0, ctx->li.sm_count, s) != cudaSuccess)
         return SPECSTEER_ERR_CUDA;
       nl = 1;
-    } else if (launch_recover(p, d->dtype, ctx->li, s, &nl) != cudaSuccess) {
+    } else if (launch_recover(p, d->dtype, ctx->li, s, &nl, lean) != cudaSuccess) {
       return SPECSTEER_ERR_CUDA;
     }
     ctx->launches += nl;

@@ -104,13 +104,13 @@ cudaError_t launch_edge_resample(const RoundParams& p, int dtype, int k, const i
                                  cudaStream_t s);
 // the streaming kernel alone (partial records into the workspace), no epilogue
 cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s);
-// log-normalisers of row accept_len of every sampling request from its records (after a ROWS_RECOVERY pass)
-cudaError_t launch_recovery_row_lse(const RoundParams& p, cudaStream_t s);
 // per-row ShardPartial of this shard from its partial records: out[B][K+1]
 cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out, cudaStream_t s);
 // the per-request epilogue alone (reads p.shard_parts when p.n_shards > 0)
 cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s);
-cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches);
+// own_lse: row accept_len has records but no normalisers yet (two-phase round); the STEER kernel forms them first.
+cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches,
+                           bool own_lse = false);
 // Greedy recovery (ARGMAX).  best_ws: [B][kTopkMaxSplit * 32] 64-bit words (the top-k selection's lists), count_ws: [B]
 // counters, zero between launches.  `aligned`: every row of the three tensors starts on a 16-byte boundary.
 // `own_lse`: the row has no normaliser in lse2 (two-phase round): the pass forms it, and the row's finiteness check, itself.

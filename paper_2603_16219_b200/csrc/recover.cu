@@ -4,6 +4,7 @@
 // The RESIDUAL kernel makes two extra passes over the row in double precision.
 #include "common.cuh"
 #include "internal.h"
+#include "records.cuh"
 #include "specsteer.h"
 
 namespace specsteer {
@@ -119,7 +120,10 @@ __device__ __forceinline__ ReqState request_state(const RoundParams& p, int b) {
   return s;
 }
 
-template <typename T, int TILE>
+// OWN_LSE: the two-phase round.  Row accept_len has just been streamed on its own and has records but no
+// normalisers yet: warp 0 combines them first (all four, as the epilogue would have), stores them, and flags a
+// non-finite row, after which nothing is sampled.
+template <typename T, int TILE, bool OWN_LSE>
 __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundParams p) {
   constexpr int kPerThread = TILE / kRecThreads;  // consecutive vocabulary entries per thread
   constexpr int kTile = TILE;
@@ -142,8 +146,40 @@ __global__ void __launch_bounds__(kRecThreads) recover_steer_kernel(const RoundP
     return;
   }
   const long long row = (long long)b * K1 + st.n;
-  const double lseR = (double)p.lse2[row * 4 + Q_R];
   const float* rec = p.part + row * p.n_chunks * 8;
+  if (OWN_LSE) {
+    __shared__ double s_lse;
+    __shared__ int s_fin;
+    if (tid < 32) {
+      float M[4];
+      double S[4];
+      row_sums_from_records(p, rec, tid, M, S);
+      const double lg = log2_pos(tid == 0 ? S[0] : (tid == 1 ? S[1] : (tid == 2 ? S[2] : S[3])));
+      bool fin = true;
+      float lse[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const double v = (double)M[q] + __shfl_sync(kFullMask, lg, q);
+        fin = fin && isfinite(v);
+        lse[q] = (float)v;
+      }
+      if (tid == 0) {
+        *reinterpret_cast<float4*>(p.lse2 + row * 4) = make_float4(lse[0], lse[1], lse[2], lse[3]);
+        s_lse = (double)lse[Q_R];
+        s_fin = fin ? 1 : 0;
+        if (!fin) {
+          p.status_ws[b] = st.status | SPECSTEER_REQ_NONFINITE;
+          if (p.req_status) p.req_status[b] = st.status | SPECSTEER_REQ_NONFINITE;
+          if (p.rec_token) p.rec_token[b] = -1;
+          if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+          if (p.n_out) p.n_out[b] = st.n;
+        }
+      }
+    }
+    __syncthreads();
+    if (!s_fin) return;
+  }
+  const double lseR = OWN_LSE ? (double)__ldcg(p.lse2 + row * 4 + Q_R) : (double)p.lse2[row * 4 + Q_R];
   for (int j = tid; j < p.n_chunks; j += kRecThreads) {
     const float m = rec[j * 8 + 6], s = rec[j * 8 + 7];
     cw[j] = (m == kNegInf) ? 0.0 : (double)s * exp2((double)m - lseR);
@@ -524,7 +560,8 @@ cudaError_t launch_recover_argmax(const RoundParams& p, int dtype, bool aligned,
                                 : launch_argmax_t<uint16_t>(cfg, aligned, own_lse, p, ws, count_ws);
 }
 
-cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches) {
+cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches,
+                           bool own_lse) {
   (void)li;
   const size_t smem = (size_t)p.n_chunks * sizeof(double);
   *n_launches = 1;
@@ -538,8 +575,13 @@ cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  cudaError_t e = dtype == SPECSTEER_F32 ? cudaLaunchKernelEx(&cfg, recover_steer_kernel<float, kChunkF32>, p)
-                                         : cudaLaunchKernelEx(&cfg, recover_steer_kernel<uint16_t, kChunkBF16>, p);
+  cudaError_t e;
+  if (own_lse)
+    e = dtype == SPECSTEER_F32 ? cudaLaunchKernelEx(&cfg, recover_steer_kernel<float, kChunkF32, true>, p)
+                               : cudaLaunchKernelEx(&cfg, recover_steer_kernel<uint16_t, kChunkBF16, true>, p);
+  else
+    e = dtype == SPECSTEER_F32 ? cudaLaunchKernelEx(&cfg, recover_steer_kernel<float, kChunkF32, false>, p)
+                               : cudaLaunchKernelEx(&cfg, recover_steer_kernel<uint16_t, kChunkBF16, false>, p);
   if (e != cudaSuccess || p.recover_mode != SPECSTEER_RECOVER_RESIDUAL) return e;
   *n_launches = 2;
   if (dtype == SPECSTEER_F32) recover_residual_kernel<float, kChunkF32><<<p.B, kRecThreads, smem, s>>>(p);

@@ -13,6 +13,7 @@
 // partials instead of the records.
 #include "common.cuh"
 #include "internal.h"
+#include "records.cuh"
 #include "specsteer.h"
 
 namespace specsteer {
@@ -66,28 +67,6 @@ __device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b) {
   return d;
 }
 
-// Reduce four per-lane values over the warp at once (22 instructions instead of 40): after the first
-// two exchange steps each lane carries one of the four quantities.  On return lanes [8q, 8q+8) hold the
-// reduction of v[q] in the return value.
-template <bool IS_MAX>
-__device__ __forceinline__ float warp_reduce4(const float (&v)[4], int lane) {
-  const bool hi16 = (lane & 16) != 0, hi8 = (lane & 8) != 0;
-  const float keep_a = hi16 ? v[2] : v[0], keep_b = hi16 ? v[3] : v[1];
-  const float send_a = hi16 ? v[0] : v[2], send_b = hi16 ? v[1] : v[3];
-  const float xa = __shfl_xor_sync(kFullMask, send_a, 16), xb = __shfl_xor_sync(kFullMask, send_b, 16);
-  const float ra = IS_MAX ? fmaxf(keep_a, xa) : keep_a + xa;
-  const float rb = IS_MAX ? fmaxf(keep_b, xb) : keep_b + xb;
-  const float keep = hi8 ? rb : ra, send = hi8 ? ra : rb;
-  const float x = __shfl_xor_sync(kFullMask, send, 8);
-  float r = IS_MAX ? fmaxf(keep, x) : keep + x;
-#pragma unroll
-  for (int o = 4; o > 0; o >>= 1) {
-    const float y = __shfl_xor_sync(kFullMask, r, o);
-    r = IS_MAX ? fmaxf(r, y) : r + y;
-  }
-  return r;
-}
-
 // A warp's running state for the four normalisers of a chunk (L, P, M and r of Eq. 8).  The reference
 // exponents are the same in every lane; the sums are per lane.
 struct Acc {
@@ -96,11 +75,6 @@ struct Acc {
   f32x2 nref2[4];  // (-ref, -ref), or (0, 0) while ref is -inf: the addend of the exponent FMA
   f32x2 s2[4];     // two partial sums of 2^(x*c - ref)
 };
-
-// 2^d for an integer-valued d <= 0 (exact); 0 below the normal range.
-__device__ __forceinline__ float pow2_nonpos_int(float d) {
-  return (d < -126.f) ? 0.f : __int_as_float(((int)d + 127) << 23);
-}
 
 __device__ __forceinline__ void acc_set_ref(Acc& a, int q, float nr, float inv_c) {
   a.ref[q] = nr;
@@ -352,28 +326,6 @@ struct RowResult {
   int8_t tok_ok;
 };
 
-// log2(x) in double for x > 0 (about 1e-12 absolute): exponent plus the atanh series of the mantissa
-// folded into [sqrt(1/2), sqrt(2)).  Short on purpose: the library routine costs several times the
-// instructions and every warp of the epilogue is latency-bound.  x = 0 gives -inf, x = +inf gives +inf,
-// negative or NaN gives NaN; subnormal inputs do not occur here (sums of float32 values >= 1, or 0).
-__device__ __forceinline__ double log2_pos(double x) {
-  if (!(x > 0.0)) return (x == 0.0) ? -__longlong_as_double(0x7ff0000000000000ll) : __longlong_as_double(0x7ff8000000000000ll);
-  const int hi = __double2hiint(x), lo = __double2loint(x);
-  if (hi >= 0x7ff00000) return x;  // +inf
-  int e = (hi >> 20) - 1023;
-  double m = __hiloint2double((hi & 0x000fffff) | 0x3ff00000, lo);  // [1, 2)
-  if (m > 1.4142135623730951) { m *= 0.5; e += 1; }
-  const double z = (m - 1.0) / (m + 1.0), w = z * z;
-  double q = 1.0 / 13.0;
-  q = fma(q, w, 1.0 / 11.0);
-  q = fma(q, w, 1.0 / 9.0);
-  q = fma(q, w, 1.0 / 7.0);
-  q = fma(q, w, 1.0 / 5.0);
-  q = fma(q, w, 1.0 / 3.0);
-  q = fma(q, w, 1.0);
-  return fma(z * q, 2.8853900817779268 /* 2/ln 2 */, (double)e);
-}
-
 // exp(x) in double for x <= 0 (about 1e-14 relative); 0 below the normal range.
 __device__ __forceinline__ double exp_nonpos(double x) {
   const double y = x * 1.4426950408889634;
@@ -397,39 +349,6 @@ __device__ __forceinline__ double exp_nonpos(double x) {
 // 2^d in double for an integer-valued d <= 0; 0 below 2^-1000.
 __device__ __forceinline__ double pow2_nonpos_int_d(float d) {
   return (d < -1000.f) ? 0.0 : __hiloint2double(((int)d + 1023) << 20, 0);
-}
-
-// One warp: the largest exponent per normaliser over the row's records and the float64 sums relative to it
-// (pass 2 finds the lines of pass 1 in L1); every lane gets the results.
-__device__ __forceinline__ void row_sums_from_records(const RoundParams& p, const float* rec, int lane, float (&M)[4],
-                                                      double (&S)[4]) {
-  float Ml[4] = {kNegInf, kNegInf, kNegInf, kNegInf};
-#pragma unroll 4
-  for (int ch = lane; ch < p.n_chunks; ch += 32) {
-    const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
-    const float4 z = __ldg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
-    Ml[0] = fmaxf(Ml[0], x.x); Ml[1] = fmaxf(Ml[1], x.z); Ml[2] = fmaxf(Ml[2], z.x); Ml[3] = fmaxf(Ml[3], z.z);
-  }
-  const float mine = warp_reduce4<true>(Ml, lane);
-#pragma unroll
-  for (int q = 0; q < 4; ++q) { M[q] = __shfl_sync(kFullMask, mine, 8 * q); S[q] = 0.0; }
-#pragma unroll 4
-  for (int ch = lane; ch < p.n_chunks; ch += 32) {
-    const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
-    const float4 z = __ldg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
-    const float mm[4] = {x.x, x.z, z.x, z.z}, ss[4] = {x.y, x.w, z.y, z.w};
-#pragma unroll
-    for (int q = 0; q < 4; ++q) {
-      float w = ss[q];
-      if (mm[q] != M[q]) w = (mm[q] == kNegInf || M[q] == -kNegInf) ? 0.f : w * pow2_nonpos_int(mm[q] - M[q]);
-      S[q] += (double)w;
-    }
-  }
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) S[q] += __shfl_xor_sync(kFullMask, S[q], o);
-  }
 }
 
 // One warp: combine the partial records of `row` (exact power-of-two rescale, sums in double) and, for a
@@ -842,47 +761,6 @@ static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cud
     attr_set = true;
   }
   kern<<<li.sm_count, (NCW + NPW) * 32, smem, s>>>(p);
-  return cudaGetLastError();
-}
-
-// ---- normalisers of the recovery rows alone ------------------------------------------------------------
-// When verification read only h_LLM and h_SLM- (the two tensors Eq. 7 needs), the streaming kernel is run once
-// more over row accept_len of the requests that sample, all four normalisers; this kernel turns that row's
-// records into its log-normalisers for the recovery kernel and flags a non-finite row.
-__global__ void __launch_bounds__(32) recovery_row_lse_kernel(const RoundParams p) {
-  const int b = blockIdx.x, lane = threadIdx.x;
-  const int K1 = p.K + 1;
-  pdl_launch_dependents();
-  pdl_wait();
-  int len = p.draft_len[b];
-  if (len < 0 || len > p.K) len = 0;
-  const int n = p.accept_len[b], status = p.status_ws[b];
-  const bool bad = (status & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
-  if (bad || !(n < len || (p.flags & SPECSTEER_FLAG_BONUS))) return;
-  const long long row = (long long)b * K1 + n;
-  float M[4];
-  double S[4];
-  row_sums_from_records(p, p.part + row * p.n_chunks * 8, lane, M, S);
-  const double lg = log2_pos(lane == 0 ? S[0] : (lane == 1 ? S[1] : (lane == 2 ? S[2] : S[3])));
-  bool fin = true;
-  float lse[4];
-#pragma unroll
-  for (int q = 0; q < 4; ++q) {
-    const double v = (double)M[q] + __shfl_sync(kFullMask, lg, q);
-    fin = fin && isfinite(v);
-    lse[q] = (float)v;
-  }
-  if (lane == 0) {
-    *reinterpret_cast<float4*>(p.lse2 + row * 4) = make_float4(lse[0], lse[1], lse[2], lse[3]);
-    if (!fin) {
-      p.status_ws[b] = status | SPECSTEER_REQ_NONFINITE;
-      if (p.req_status) p.req_status[b] = status | SPECSTEER_REQ_NONFINITE;
-    }
-  }
-}
-
-cudaError_t launch_recovery_row_lse(const RoundParams& p, cudaStream_t s) {
-  recovery_row_lse_kernel<<<p.B, 32, 0, s>>>(p);
   return cudaGetLastError();
 }
 
