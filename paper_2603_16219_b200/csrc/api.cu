@@ -142,7 +142,7 @@ bool two_phase(const specsteer_round_desc* d) {
                         !d->logp_plus && !d->logp_star && !d->log_z && rows_aligned(d);
   if (!eligible) return false;
   if (d->flags & SPECSTEER_FLAG_TWO_PHASE) return true;
-  // two more launches (about 10 us) against a fifth of the bytes: worth it from roughly 128 MB of logits upwards
+  // one more launch and a short second pass (about 10 us) against a fifth of the bytes: worth it from roughly 128 MB of logits upwards
   const double bytes = 3.0 * d->B * (d->K + 1) * (double)d->V * (d->dtype == SPECSTEER_F32 ? 4 : 2);
   return bytes >= 128.0 * 1024 * 1024;
 }
