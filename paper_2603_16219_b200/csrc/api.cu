@@ -147,24 +147,53 @@ bool two_phase(const specsteer_round_desc* d) {
   return bytes >= 128.0 * 1024 * 1024;
 }
 
+// Verification of the requests [b0, b0 + nb).  lean: two tensors over the drafted rows, in the larger chunks of that
+// launch shape (the two-phase round).
+specsteer_status verify_slab(specsteer_ctx* ctx, const specsteer_round_desc* d, int b0, int nb, bool lean, cudaStream_t s,
+                             cudaEvent_t ev_begin, cudaEvent_t ev_end) {
+  RoundParams p = slab_params(ctx, d, b0, nb);
+  if (lean) {
+    p.sums = SUM_L | SUM_M;
+    p.row_mode = ROWS_DRAFTED;
+    p.tile = d->dtype == SPECSTEER_F32 ? kChunkRatioF32 : kChunkRatioBF16;
+    p.n_chunks = n_chunks_of(d->V, p.tile);
+  }
+  int nl = 0;
+  if (launch_verify(p, d->dtype, rows_aligned(d), ctx->li, s, &nl, ev_begin, ev_end) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += nl;
+  return SPECSTEER_OK;
+}
+
+// Recovery of the requests [b0, b0 + nb).  lean: the verification left row accept_len unread.
+specsteer_status recover_slab(specsteer_ctx* ctx, const specsteer_round_desc* d, int b0, int nb, bool lean, cudaStream_t s) {
+  RoundParams p = slab_params(ctx, d, b0, nb);
+  int nl = 0;
+  if (lean && d->recover_mode != SPECSTEER_RECOVER_ARGMAX) {   // the recovery rows have no records yet: one more streaming pass over them alone
+    p.sums = SUM_ALL;
+    p.row_mode = ROWS_RECOVERY;
+    if (launch_verify_stream(p, d->dtype, true, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    ctx->launches += 1;
+  }
+  if (d->recover_mode == SPECSTEER_RECOVER_ARGMAX) {
+    if (launch_recover_argmax(p, d->dtype, rows_aligned(d), lean, (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
+                              ctx->topk_count + b0, ctx->li.sm_count, s) != cudaSuccess)
+      return SPECSTEER_ERR_CUDA;
+    nl = 1;
+  } else if (launch_recover(p, d->dtype, ctx->li, s, &nl, lean) != cudaSuccess) {
+    return SPECSTEER_ERR_CUDA;
+  }
+  ctx->launches += nl;
+  return SPECSTEER_OK;
+}
+
 specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
-  const bool aligned = rows_aligned(d);
   const bool lean = two_phase(d);
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
-    RoundParams p = slab_params(ctx, d, b0, nb);
-    if (lean) {   // two tensors over the drafted rows, in the larger chunks of that launch shape
-      p.sums = SUM_L | SUM_M;
-      p.row_mode = ROWS_DRAFTED;
-      p.tile = d->dtype == SPECSTEER_F32 ? kChunkRatioF32 : kChunkRatioBF16;
-      p.n_chunks = n_chunks_of(d->V, p.tile);
-    }
-    int nl = 0;
     const bool first = b0 == 0, last = b0 + nb >= d->B;
-    if (launch_verify(p, d->dtype, aligned, ctx->li, s, &nl, first ? ctx->ev_stream_begin : nullptr,
-                      last ? ctx->ev_stream_end : nullptr) != cudaSuccess)
-      return SPECSTEER_ERR_CUDA;
-    ctx->launches += nl;
+    specsteer_status st = verify_slab(ctx, d, b0, nb, lean, s, first ? ctx->ev_stream_begin : nullptr,
+                                      last ? ctx->ev_stream_end : nullptr);
+    if (st != SPECSTEER_OK) return st;
   }
   return SPECSTEER_OK;
 }
@@ -173,23 +202,8 @@ specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, c
   const bool lean = ctx->v_two_phase;   // what the verification of this round did, not what this descriptor says
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
-    RoundParams p = slab_params(ctx, d, b0, nb);
-    int nl = 0;
-    if (lean && d->recover_mode != SPECSTEER_RECOVER_ARGMAX) {   // the recovery rows have no records yet: one more streaming pass over them alone
-      p.sums = SUM_ALL;
-      p.row_mode = ROWS_RECOVERY;
-      if (launch_verify_stream(p, d->dtype, true, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-      ctx->launches += 1;
-    }
-    if (d->recover_mode == SPECSTEER_RECOVER_ARGMAX) {
-      if (launch_recover_argmax(p, d->dtype, rows_aligned(d), lean, (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
-                                ctx->topk_count + b0, ctx->li.sm_count, s) != cudaSuccess)
-        return SPECSTEER_ERR_CUDA;
-      nl = 1;
-    } else if (launch_recover(p, d->dtype, ctx->li, s, &nl, lean) != cudaSuccess) {
-      return SPECSTEER_ERR_CUDA;
-    }
-    ctx->launches += nl;
+    specsteer_status st = recover_slab(ctx, d, b0, nb, lean, s);
+    if (st != SPECSTEER_OK) return st;
   }
   return SPECSTEER_OK;
 }
@@ -627,8 +641,60 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
   CK(cudaEventRecord(ctx->ev_done[0], s));
   CK(cudaStreamWaitEvent(ctx->copy_stream, ctx->ev_done[0], 0));
 
-  // slabs of requests: copy slab i+1 on the copy stream while slab i computes on `s`
   const size_t req_bytes = (size_t)h->ld_req * es;
+  const size_t row_bytes = (size_t)h->ld_row * es;
+  specsteer_round_desc forced = d;
+  forced.flags |= SPECSTEER_FLAG_TWO_PHASE;
+  if (two_phase(&forced)) {
+    // Only Algorithm 1's outputs are wanted: the link, not the GPU, bounds this call, so copy only what the two-phase
+    // round reads.  First h_LLM and h_SLM- of the drafted rows, slab by slab, each slab verified while the next one is
+    // copied; then, with the accepted lengths on the host, row accept_len of h_SLM+ for every request that takes a token
+    // (and of the other two tensors when that row is the bonus row, which verification did not need); then recovery.
+    size_t per2 = (size_t)(96u << 20) / (2 * req_bytes);
+    const int slab2 = (int)(per2 < 1 ? 1 : (per2 > (size_t)kMaxSlabB ? (size_t)kMaxSlabB : per2));
+    int idx2 = 0;
+    for (int b0 = 0; b0 < B && !fail; b0 += slab2, idx2 ^= 1) {
+      const int nb = B - b0 < slab2 ? B - b0 : slab2;
+      for (int b = b0; b < b0 + nb; ++b) {
+        int ln = h->draft_len[b];
+        if (ln < 0 || ln > K) ln = 0;
+        if (ln == 0) continue;
+        const size_t o = (size_t)b * req_bytes, nbytes = (size_t)ln * row_bytes;
+        CK(cudaMemcpyAsync((char*)d.h_llm + o, (const char*)h->h_llm + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+        CK(cudaMemcpyAsync((char*)d.h_slm_minus + o, (const char*)h->h_slm_minus + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+      }
+      CK(cudaEventRecord(ctx->ev_copied[idx2], ctx->copy_stream));
+      CK(cudaStreamWaitEvent(s, ctx->ev_copied[idx2], 0));
+      if (verify_slab(ctx, &forced, b0, nb, true, s, nullptr, nullptr) != SPECSTEER_OK) fail = true;
+    }
+    int32_t* n_host = (int32_t*)malloc((size_t)B * 8);
+    if (!n_host) fail = true;
+    if (!fail) {
+      int32_t* st_host = n_host + B;
+      CK(cudaMemcpyAsync(n_host, d.accept_len, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+      CK(cudaMemcpyAsync(st_host, ctx->status_ws, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
+      CK(cudaStreamSynchronize(s));
+      for (int b = 0; b < B && !fail; ++b) {
+        int ln = h->draft_len[b];
+        if (ln < 0 || ln > K) ln = 0;
+        const int n = n_host[b];
+        const bool bad = (st_host[b] & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+        if (bad || n < 0 || n > ln || !(n < ln || (h->flags & SPECSTEER_FLAG_BONUS))) continue;
+        const size_t o = (size_t)b * req_bytes + (size_t)n * row_bytes;
+        CK(cudaMemcpyAsync((char*)d.h_slm_plus + o, (const char*)h->h_slm_plus + o, row_bytes, cudaMemcpyHostToDevice, s));
+        if (n >= ln) {
+          CK(cudaMemcpyAsync((char*)d.h_llm + o, (const char*)h->h_llm + o, row_bytes, cudaMemcpyHostToDevice, s));
+          CK(cudaMemcpyAsync((char*)d.h_slm_minus + o, (const char*)h->h_slm_minus + o, row_bytes, cudaMemcpyHostToDevice, s));
+        }
+      }
+      for (int b0 = 0; b0 < B && !fail; b0 += kMaxSlabB) {
+        const int nb = B - b0 < kMaxSlabB ? B - b0 : kMaxSlabB;
+        if (recover_slab(ctx, &forced, b0, nb, true, s) != SPECSTEER_OK) fail = true;
+      }
+    }
+    free(n_host);
+  } else {
+  // slabs of requests: copy slab i+1 on the copy stream while slab i computes on `s`
   size_t per = (size_t)(96u << 20) / (3 * req_bytes);
   int slab = (int)(per < 1 ? 1 : (per > (size_t)kMaxSlabB ? (size_t)kMaxSlabB : per));
   int idx = 0;
@@ -650,6 +716,7 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
     } else {
       CK(launch_recover(p, d.dtype, ctx->li, s, &nl)); ctx->launches += nl;
     }
+  }
   }
   auto back = [&](void* hp, const void* dp, size_t bytes) {
     if (hp && dp && bytes) CK(cudaMemcpyAsync(hp, dp, bytes, cudaMemcpyDeviceToHost, s));

@@ -489,8 +489,11 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
     __threadfence();
     if (atomicAdd(&count_ws[b], 1) != S - 1) return;
     __threadfence();
+    // merge all parts in index order, this CTA's own included, so that the sums do not depend on who finished last
+    best = 0;
+    acc.m = kNegInf; acc.s = 0.f;
+    mx[0] = mx[1] = mx[2] = kNegInf;
     for (int j = 0; j < S; ++j) {
-      if (j == sp) continue;
       const u64 k = __ldcg(mine + j);
       best = k > best ? k : best;
       if (LSE) {

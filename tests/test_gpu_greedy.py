@@ -183,3 +183,21 @@ def test_two_phase_greedy_full_size_equals_one_pass(env):
     for k in ("accept_len", "rec_token", "n_out", "out_tokens", "req_status", "accept_flags"):
         assert np.array_equal(outs[k].cpu().numpy(), full[k]), k
     assert np.abs(outs["rec_logprob"].cpu().numpy() - full["rec_logprob"]).max() <= 1e-5
+
+
+def test_two_phase_greedy_is_deterministic(env):
+    """The row's parts are merged in index order by whichever CTA finishes last: repeated rounds give the same bits."""
+    b, synth = env["binding"], env["synth"]
+    spec = synth.RoundSpec("g", 5, 3, 70000, "bf16", beta_choices=(0.5, 1.0, 2.0), temp_choices=(0.7, 1.3))
+    inputs = synth.make_round(spec, device="cuda", seed=77)
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in ("logp_plus", "logp_star", "log_z")}
+    d = b.make_desc(inputs, outs, recover_mode=ARGMAX, flags=1 | b.FLAG_TWO_PHASE)
+    seen = None
+    for _ in range(12):
+        env["ctx"].verify_round(d)
+        env["ctx"].recover_sample(d)
+        torch.cuda.synchronize()
+        got = (outs["rec_token"].cpu().numpy().copy(), outs["rec_logprob"].cpu().numpy().copy())
+        if seen is None:
+            seen = got
+        assert np.array_equal(seen[0], got[0]) and np.array_equal(seen[1], got[1])

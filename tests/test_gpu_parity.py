@@ -464,3 +464,47 @@ def test_host_round_matches_device_round(env):
     env["ctx"].round_host(desc)
     for k, v in host_out.items():
         assert np.array_equal(dev[k], v.numpy(), equal_nan=True), k
+
+
+@pytest.mark.parametrize("recover_mode", [0, 2], ids=["sampled", "greedy"])
+@pytest.mark.parametrize("dtype,flags", [("f32", 1), ("bf16", 0), ("bf16", 1)])
+def test_host_round_with_algorithm1_outputs_copies_only_what_it_reads(env, dtype, flags, recover_mode):
+    """Only Algorithm 1's outputs requested from host buffers: h_LLM and h_SLM- of the drafted rows go over first,
+    then row accept_len of h_SLM+ (and of the other two when it is the bonus row).  Everything else on the host is
+    poisoned with NaN to prove it is never used; results equal the device-resident two-phase round."""
+    b = env["binding"]
+    V = 9004 if dtype == "f32" else 12288
+    spec, inputs = _small(env["synth"], 21, 4, V, dtype, seed=70 + flags, ragged=True,
+                          beta_choices=(0.5, 1.0, 2.0), temp_choices=(0.7, 1.0))
+    inputs["draft_len"][0] = 0
+    inputs["u_accept"][1] = 0.0                  # everything accepted: the bonus row (or nothing) is recovered
+    inputs["temperature"][2] = 0.0               # BAD_PARAM
+    inputs["h_llm"][3, 0, 11] = float("nan")     # non-finite already in verification
+    inputs["lam"][4] = 1e30
+    inputs["h_slm_plus"][4, 0, 5] = float("inf")  # non-finite only on the recovery row
+    skip = ("logp_plus", "logp_star", "log_z")
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in skip}
+    d = b.make_desc(inputs, outs, recover_mode=recover_mode, flags=flags | b.FLAG_TWO_PHASE)
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    dev = {k: v.cpu().numpy() for k, v in outs.items()}
+    # host copies with everything the round does not need turned into NaN
+    n, dl = dev["accept_len"], inputs["draft_len"].cpu().numpy()
+    host_in = {k: v.cpu().clone() for k, v in inputs.items()}
+    rows = torch.arange(spec.K + 1)[None, :]
+    drafted = rows < torch.as_tensor(dl)[:, None]
+    rec_row = (rows == torch.as_tensor(n)[:, None]) & torch.as_tensor(
+        ((n < dl) | bool(flags)) & ((dev["req_status"] & 16) == 0))[:, None]
+    nan = float("nan")
+    host_in["h_llm"][~(drafted | rec_row)] = nan
+    host_in["h_slm_minus"][~(drafted | rec_row)] = nan
+    host_in["h_slm_plus"][~rec_row] = nan
+    host_in["h_llm"][3, 0, 11] = nan             # (kept: part of the case)
+    host_in = {k: v.pin_memory() for k, v in host_in.items()}
+    host_out = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cpu", pin=True).items() if k not in skip}
+    env["ctx"].round_host(b.make_desc(host_in, host_out, recover_mode=recover_mode, flags=flags))
+    assert env["ctx"].device_error() == 0
+    for k, v in host_out.items():
+        assert np.array_equal(dev[k], v.numpy(), equal_nan=True), k
+    assert dev["req_status"][2] == 16 and dev["req_status"][3] & 4 and dev["req_status"][4] & 4
