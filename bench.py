@@ -394,6 +394,33 @@ def run_cuda(args, rank, world, local_rank):
         e2e_s = float(t.item())
     e2e_value = world * positions / e2e_s
     assert torch.equal(host_out["accept_len"], outs["accept_len"].cpu())
+    # the same call asked for Algorithm 1's outputs only: it then copies just what the two-phase round reads
+    e2e_alg1 = None
+    if not args.lean:
+        lean_host_out = {k: v for k, v in binding.alloc_outputs(spec.B, spec.K, "cpu", pin=True).items()
+                         if k not in ("logp_plus", "logp_star", "log_z")}
+        lean_hdesc = binding.make_desc(host_in, lean_host_out, flags=flags)
+        for _ in range(2):
+            ctx.round_host(lean_hdesc, stream)
+        barrier()
+        w0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            ctx.round_host(lean_hdesc, stream)
+        torch.cuda.synchronize(dev)
+        w1 = time.perf_counter()
+        sampler.window(w0, w1)
+        lean_s = (w1 - w0) / e2e_steps
+        if dist is not None:
+            t = torch.tensor([lean_s], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            lean_s = float(t.item())
+        n_acc = lean_host_out["accept_len"].to(torch.int64)
+        dl = host_in["draft_len"].to(torch.int64)
+        rows_copied = int(2 * spec.B * spec.K + (lean_host_out["rec_token"] >= 0).sum() + 2 * ((n_acc >= dl) & (lean_host_out["rec_token"] >= 0)).sum())
+        e2e_alg1 = {"value": world * positions / lean_s, "unit": UNIT, "ms_per_step": 1e3 * lean_s, "steps": e2e_steps,
+                    "h2d_bytes_per_step": rows_copied * spec.V * spec.elem_bytes + h2d - 3 * spec.rows * spec.V * spec.elem_bytes,
+                    "same_accept_len_and_tokens": bool(torch.equal(lean_host_out["accept_len"], host_out["accept_len"]) and
+                                                       torch.equal(lean_host_out["rec_token"], host_out["rec_token"]))}
     sampler.stop()
 
     if rank != 0:
@@ -455,7 +482,8 @@ def run_cuda(args, rank, world, local_rank):
         "roofline": roofline,
         "cpu_baseline": cpu,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "api": "specsteer_round_host (pinned host buffers)"},
+                "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "api": "specsteer_round_host (pinned host buffers)",
+                "algorithm1_outputs_only": e2e_alg1},
         "algorithm1_outputs_only": alg1,
         "gpu_launches": int(gpu_launches),
         "clocks": sampler.summary(),

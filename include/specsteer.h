@@ -257,6 +257,11 @@ specsteer_status specsteer_lmhead_shard_recover(specsteer_ctx *ctx, const specst
  * call, sized for the context's maxima: 3*max_B*(max_K+1)*max_V elements of 4 bytes), runs verification and
  * recovery, copies every non-NULL output back, and returns after the stream has drained.  Requests are
  * processed in slabs so that the copy of one slab overlaps the kernels of the previous one.
+ * The host-to-device link bounds this call, so when only Algorithm 1's outputs are wanted (the conditions of the
+ * two-phase round: RATIO, STEER or ARGMAX, logp_plus / logp_star / log_z NULL, 16-byte aligned rows) it copies only
+ * what that round reads: rows [0, K) of h_LLM and h_SLM-, then - once the accepted lengths are back on the host -
+ * row accept_len of h_SLM+ for every request that takes a token (and of the other two tensors when that row is the
+ * bonus row).  Nothing else of the three host tensors is touched.
  * Errors: as the two calls above, plus WORKSPACE. */
 specsteer_status specsteer_round_host(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
 

@@ -647,7 +647,7 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
   forced.flags |= SPECSTEER_FLAG_TWO_PHASE;
   if (two_phase(&forced)) {
     // Only Algorithm 1's outputs are wanted: the link, not the GPU, bounds this call, so copy only what the two-phase
-    // round reads.  First h_LLM and h_SLM- of the drafted rows, slab by slab, each slab verified while the next one is
+    // round reads.  First rows [0, K) of h_LLM and h_SLM-, slab by slab, each slab verified while the next one is
     // copied; then, with the accepted lengths on the host, row accept_len of h_SLM+ for every request that takes a token
     // (and of the other two tensors when that row is the bonus row, which verification did not need); then recovery.
     size_t per2 = (size_t)(96u << 20) / (2 * req_bytes);
@@ -655,13 +655,12 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
     int idx2 = 0;
     for (int b0 = 0; b0 < B && !fail; b0 += slab2, idx2 ^= 1) {
       const int nb = B - b0 < slab2 ? B - b0 : slab2;
-      for (int b = b0; b < b0 + nb; ++b) {
-        int ln = h->draft_len[b];
-        if (ln < 0 || ln > K) ln = 0;
-        if (ln == 0) continue;
-        const size_t o = (size_t)b * req_bytes, nbytes = (size_t)ln * row_bytes;
-        CK(cudaMemcpyAsync((char*)d.h_llm + o, (const char*)h->h_llm + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
-        CK(cudaMemcpyAsync((char*)d.h_slm_minus + o, (const char*)h->h_slm_minus + o, nbytes, cudaMemcpyHostToDevice, ctx->copy_stream));
+      if (K > 0) {   // rows [0, K) of every request of the slab: one strided copy per tensor (rows beyond draft_len ride along)
+        const size_t o = (size_t)b0 * req_bytes;
+        CK(cudaMemcpy2DAsync((char*)d.h_llm + o, req_bytes, (const char*)h->h_llm + o, req_bytes, (size_t)K * row_bytes, nb,
+                             cudaMemcpyHostToDevice, ctx->copy_stream));
+        CK(cudaMemcpy2DAsync((char*)d.h_slm_minus + o, req_bytes, (const char*)h->h_slm_minus + o, req_bytes,
+                             (size_t)K * row_bytes, nb, cudaMemcpyHostToDevice, ctx->copy_stream));
       }
       CK(cudaEventRecord(ctx->ev_copied[idx2], ctx->copy_stream));
       CK(cudaStreamWaitEvent(s, ctx->ev_copied[idx2], 0));
@@ -674,6 +673,11 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
       CK(cudaMemcpyAsync(n_host, d.accept_len, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
       CK(cudaMemcpyAsync(st_host, ctx->status_ws, (size_t)B * 4, cudaMemcpyDeviceToHost, s));
       CK(cudaStreamSynchronize(s));
+      // single rows, many of them: spread over both streams so that one copy's set-up hides behind another's transfer
+      int turn = 0;
+      auto row_copy = [&](void* dst, const void* src) {
+        CK(cudaMemcpyAsync(dst, src, row_bytes, cudaMemcpyHostToDevice, (turn++ & 1) ? ctx->copy_stream : s));
+      };
       for (int b = 0; b < B && !fail; ++b) {
         int ln = h->draft_len[b];
         if (ln < 0 || ln > K) ln = 0;
@@ -681,12 +685,14 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
         const bool bad = (st_host[b] & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
         if (bad || n < 0 || n > ln || !(n < ln || (h->flags & SPECSTEER_FLAG_BONUS))) continue;
         const size_t o = (size_t)b * req_bytes + (size_t)n * row_bytes;
-        CK(cudaMemcpyAsync((char*)d.h_slm_plus + o, (const char*)h->h_slm_plus + o, row_bytes, cudaMemcpyHostToDevice, s));
-        if (n >= ln) {
-          CK(cudaMemcpyAsync((char*)d.h_llm + o, (const char*)h->h_llm + o, row_bytes, cudaMemcpyHostToDevice, s));
-          CK(cudaMemcpyAsync((char*)d.h_slm_minus + o, (const char*)h->h_slm_minus + o, row_bytes, cudaMemcpyHostToDevice, s));
+        row_copy((char*)d.h_slm_plus + o, (const char*)h->h_slm_plus + o);
+        if (n >= K) {   // the bonus row of a request with K drafts: the first copies stopped before it
+          row_copy((char*)d.h_llm + o, (const char*)h->h_llm + o);
+          row_copy((char*)d.h_slm_minus + o, (const char*)h->h_slm_minus + o);
         }
       }
+      CK(cudaEventRecord(ctx->ev_copied[0], ctx->copy_stream));
+      CK(cudaStreamWaitEvent(s, ctx->ev_copied[0], 0));
       for (int b0 = 0; b0 < B && !fail; b0 += kMaxSlabB) {
         const int nb = B - b0 < kMaxSlabB ? B - b0 : kMaxSlabB;
         if (recover_slab(ctx, &forced, b0, nb, true, s) != SPECSTEER_OK) fail = true;

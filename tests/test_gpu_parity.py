@@ -469,7 +469,7 @@ def test_host_round_matches_device_round(env):
 @pytest.mark.parametrize("recover_mode", [0, 2], ids=["sampled", "greedy"])
 @pytest.mark.parametrize("dtype,flags", [("f32", 1), ("bf16", 0), ("bf16", 1)])
 def test_host_round_with_algorithm1_outputs_copies_only_what_it_reads(env, dtype, flags, recover_mode):
-    """Only Algorithm 1's outputs requested from host buffers: h_LLM and h_SLM- of the drafted rows go over first,
+    """Only Algorithm 1's outputs requested from host buffers: rows [0, K) of h_LLM and h_SLM- go over first,
     then row accept_len of h_SLM+ (and of the other two when it is the bonus row).  Everything else on the host is
     poisoned with NaN to prove it is never used; results equal the device-resident two-phase round."""
     b = env["binding"]
@@ -493,7 +493,7 @@ def test_host_round_with_algorithm1_outputs_copies_only_what_it_reads(env, dtype
     n, dl = dev["accept_len"], inputs["draft_len"].cpu().numpy()
     host_in = {k: v.cpu().clone() for k, v in inputs.items()}
     rows = torch.arange(spec.K + 1)[None, :]
-    drafted = rows < torch.as_tensor(dl)[:, None]
+    drafted = (rows < spec.K).expand(spec.B, -1)      # rows [0, K) of the two tensors travel whatever draft_len is
     rec_row = (rows == torch.as_tensor(n)[:, None]) & torch.as_tensor(
         ((n < dl) | bool(flags)) & ((dev["req_status"] & 16) == 0))[:, None]
     nan = float("nan")
