@@ -152,7 +152,8 @@ specsteer_status specsteer_verify_round(specsteer_ctx *ctx, const specsteer_roun
  * FLAG_BONUS) samples one token from row accept_len by inverse CDF in vocabulary order:
  * the smallest v with sum_{j<=v} w(j) > u_recover * sum_j w(j).  Must follow specsteer_verify_round with
  * the same descriptor on the same stream (ERR_ORDER otherwise).  Writes rec_token, rec_logprob,
- * out_tokens, n_out.  Errors: INVALID_ARG, ORDER, CUDA. */
+ * out_tokens, n_out.  With SPECSTEER_RECOVER_ARGMAX (greedy decoding) the token is the maximiser of h_rec on that
+ * row instead and u_recover is not used.  Errors: INVALID_ARG, ORDER, CUDA. */
 specsteer_status specsteer_recover_sample(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
 
 /* Top-k split recovery (the paper's deployment appendix, "Minimal Downlink (Steering Recovery)", case "If
