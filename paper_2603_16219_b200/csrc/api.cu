@@ -46,6 +46,7 @@ struct specsteer_ctx {
 };
 
 static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
+static_assert(sizeof(specsteer_lmhead_desc) == 288, "the Python mirror of the LM-head descriptor assumes this layout");
 
 namespace {
 

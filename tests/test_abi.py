@@ -120,3 +120,19 @@ def test_lmhead_descriptor_marshalling_rejects_bad_operands():
     broken["beta"] = torch.ones(B + 1)
     with pytest.raises(ValueError):
         b.make_lmhead_desc(broken, outs)
+
+
+def test_lmhead_descriptor_layout_matches_header(lib):
+    from paper_2603_16219_b200 import binding
+    hdr = open(os.path.join(ROOT, "include", "specsteer.h")).read()
+    end = hdr.index("} specsteer_lmhead_desc;")
+    body = re.sub(r"/\*.*?\*/", "", hdr[hdr.rindex("typedef struct {", 0, end):end], flags=re.S)
+    fields = []
+    for decl in body.split(";"):
+        decl = decl.replace("typedef struct {", "").strip()
+        if not decl:
+            continue
+        for part in decl.split(","):
+            fields.append(re.findall(r"([A-Za-z_0-9]+)\s*$", part.strip())[0])
+    assert fields == [n for n, _ in binding.LmheadDesc._fields_]
+    assert C.sizeof(binding.LmheadDesc) == C.sizeof(binding.RoundDesc) + 6 * 8 + 2 * 4 == 288
