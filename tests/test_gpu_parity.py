@@ -508,3 +508,24 @@ def test_host_round_with_algorithm1_outputs_copies_only_what_it_reads(env, dtype
     for k, v in host_out.items():
         assert np.array_equal(dev[k], v.numpy(), equal_nan=True), k
     assert dev["req_status"][2] == 16 and dev["req_status"][3] & 4 and dev["req_status"][4] & 4
+
+
+@pytest.mark.parametrize("B,K,V", [(3, 0, 4100), (1100, 1, 520)])
+def test_host_round_with_algorithm1_outputs_edge_shapes(env, B, K, V):
+    """No drafts at all (only bonus rows travel), and more requests than one slab holds."""
+    b = env["binding"]
+    spec, inputs = _small(env["synth"], B, K, V, "f32", seed=90 + K)
+    skip = ("logp_plus", "logp_star", "log_z")
+    for recover_mode in (0, 2):
+        outs = {k: v for k, v in b.alloc_outputs(B, K, "cuda").items() if k not in skip}
+        d = b.make_desc(inputs, outs, recover_mode=recover_mode, flags=1 | b.FLAG_TWO_PHASE)
+        env["ctx"].verify_round(d)
+        env["ctx"].recover_sample(d)
+        torch.cuda.synchronize()
+        host_in = {k: v.cpu().pin_memory() for k, v in inputs.items()}
+        host_out = {k: v for k, v in b.alloc_outputs(B, K, "cpu", pin=True).items() if k not in skip}
+        env["ctx"].round_host(b.make_desc(host_in, host_out, recover_mode=recover_mode, flags=1))
+        assert env["ctx"].device_error() == 0
+        for k, v in host_out.items():
+            assert np.array_equal(outs[k].cpu().numpy(), v.numpy(), equal_nan=True), (k, recover_mode)
+        assert (host_out["rec_token"].numpy() >= 0).all()
