@@ -68,7 +68,7 @@ typedef enum {
                                      under Softmax(h_rec / T).  One more pass over row accept_len of every request
                                      that takes a token (in the LM-head round: none, the tensor-core pass leaves the
                                      largest h_rec of every tile; the order is then that of its float32 accumulators).
-                                     Not available in the sharded rounds. */
+                                     In the sharded rounds: specsteer_shard_greedy_local / _finish. */
 } specsteer_recover_mode;
 
 enum {
@@ -252,6 +252,24 @@ specsteer_status specsteer_lmhead_shard_combine(specsteer_ctx *ctx, const specst
 specsteer_status specsteer_lmhead_shard_recover(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc, const void *gathered,
                                                 int32_t n_shards, int32_t shard_rank, int32_t vocab_offset,
                                                 int32_t vocab_total, void *cuda_stream);
+
+/* Greedy recovery (SPECSTEER_RECOVER_ARGMAX) in the two vocabulary-sharded rounds.  Steps 1-3 are as above; in place
+ * of step 4:
+ *   4a. specsteer_shard_greedy_local (logit shards; after specsteer_shard_verify_combine) or
+ *       specsteer_lmhead_shard_greedy_local (head shards; after specsteer_lmhead_shard_combine): best_keys[B]
+ *       (device, int64) receives this shard's best entry of row accept_len as a key that orders by h_rec first and
+ *       by the lower GLOBAL token id among equal values ((order-preserving float bits << 31) | (0x7fffffff - id));
+ *       -1 for a request that takes no token;
+ *   4b. the caller takes the element-wise MAX of best_keys over the shards (one all-reduce of B int64);
+ *   4c. specsteer_shard_greedy_finish on every GPU: rec_token, rec_logprob, out_tokens and n_out from the reduced
+ *       keys, identical everywhere (desc: the round descriptor, or &lmhead_desc->round).
+ * Errors: INVALID_ARG, UNSUPPORTED (another recovery mode), ORDER, TIMEOUT, CUDA. */
+specsteer_status specsteer_shard_greedy_local(specsteer_ctx *ctx, const specsteer_round_desc *desc, int32_t vocab_offset,
+                                              int64_t *best_keys, void *cuda_stream);
+specsteer_status specsteer_lmhead_shard_greedy_local(specsteer_ctx *ctx, const specsteer_lmhead_desc *desc,
+                                                     int64_t *best_keys, void *cuda_stream);
+specsteer_status specsteer_shard_greedy_finish(specsteer_ctx *ctx, const specsteer_round_desc *desc,
+                                               const int64_t *best_keys, void *cuda_stream);
 
 /* Whole round from HOST memory: every pointer in `desc` is a HOST pointer (pinned memory makes the copies
  * asynchronous).  Copies inputs to device staging buffers owned by the context (allocated on the first

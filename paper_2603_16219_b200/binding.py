@@ -32,6 +32,7 @@ EXPORTS = (
     "specsteer_shard_verify_local", "specsteer_shard_verify_combine", "specsteer_shard_recover_local",
     "specsteer_lmhead_round",
     "specsteer_lmhead_shard_local", "specsteer_lmhead_shard_combine", "specsteer_lmhead_shard_recover",
+    "specsteer_shard_greedy_local", "specsteer_lmhead_shard_greedy_local", "specsteer_shard_greedy_finish",
 )
 SHARD_PARTIAL_BYTES = 64
 MAX_SHARDS = 32
@@ -107,6 +108,12 @@ def load_library(path: Optional[str] = None):
         fn.restype = C.c_int
     lib.specsteer_lmhead_round.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p]
     lib.specsteer_lmhead_round.restype = C.c_int
+    lib.specsteer_shard_greedy_local.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_int32, C.c_void_p, C.c_void_p]
+    lib.specsteer_shard_greedy_local.restype = C.c_int
+    lib.specsteer_lmhead_shard_greedy_local.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p, C.c_void_p]
+    lib.specsteer_lmhead_shard_greedy_local.restype = C.c_int
+    lib.specsteer_shard_greedy_finish.argtypes = [C.c_void_p, C.POINTER(RoundDesc), C.c_void_p, C.c_void_p]
+    lib.specsteer_shard_greedy_finish.restype = C.c_int
     lib.specsteer_lmhead_shard_local.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_int32, C.c_void_p, C.c_void_p]
     lib.specsteer_lmhead_shard_local.restype = C.c_int
     for fn in (lib.specsteer_lmhead_shard_combine, lib.specsteer_lmhead_shard_recover):
@@ -314,6 +321,28 @@ class Context:
         """Step 4: the shard that holds the CDF target recomputes its chunk and samples."""
         self._lmhead_shard_call(self._lib.specsteer_lmhead_shard_recover, "specsteer_lmhead_shard_recover", desc, gathered,
                                 shard_rank, vocab_offset, vocab_total, stream)
+
+    @staticmethod
+    def _keys(best_keys: torch.Tensor, B: int):
+        if best_keys.dtype != torch.int64 or tuple(best_keys.shape) != (B,) or not best_keys.is_contiguous():
+            raise ValueError("best_keys must be a contiguous int64 tensor [B]")
+        return C.c_void_p(best_keys.data_ptr())
+
+    def shard_greedy_local(self, desc: RoundDesc, vocab_offset: int, best_keys: torch.Tensor, stream=None):
+        """Greedy recovery in the vocabulary-sharded round: this shard's best key per request."""
+        _check(self._lib.specsteer_shard_greedy_local(self._h, C.byref(desc), int(vocab_offset), self._keys(best_keys, desc.B),
+                                                      self._stream(stream)), "specsteer_shard_greedy_local")
+
+    def lmhead_shard_greedy_local(self, desc: LmheadDesc, best_keys: torch.Tensor, stream=None):
+        """The same with the heads split along the vocabulary."""
+        _check(self._lib.specsteer_lmhead_shard_greedy_local(self._h, C.byref(desc), self._keys(best_keys, desc.round.B),
+                                                             self._stream(stream)), "specsteer_lmhead_shard_greedy_local")
+
+    def shard_greedy_finish(self, desc, best_keys: torch.Tensor, stream=None):
+        """Outputs from the keys reduced (MAX) over the shards; desc: a RoundDesc or an LmheadDesc."""
+        r = desc.round if isinstance(desc, LmheadDesc) else desc
+        _check(self._lib.specsteer_shard_greedy_finish(self._h, C.byref(r), self._keys(best_keys, r.B), self._stream(stream)),
+               "specsteer_shard_greedy_finish")
 
     def cloud_topk(self, desc: RoundDesc, topk_idx: torch.Tensor, topk_val: torch.Tensor, stream=None):
         """Cloud half of the top-k split recovery: fills topk_idx [B, k] int32 and topk_val [B, k] float32."""

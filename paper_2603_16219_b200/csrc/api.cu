@@ -392,6 +392,48 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx* ctx, const specste
   return SPECSTEER_OK;
 }
 
+// Greedy recovery in the vocabulary-sharded round: this shard's best key per request (see the header).
+specsteer_status specsteer_shard_greedy_local(specsteer_ctx* ctx, const specsteer_round_desc* d, int32_t vocab_offset,
+                                              int64_t* best_keys, void* cuda_stream) {
+  specsteer_status st = check_desc(ctx, d);
+  if (st != SPECSTEER_OK) return st;
+  if (!best_keys || vocab_offset < 0 || d->B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->recover_mode != SPECSTEER_RECOVER_ARGMAX) return SPECSTEER_ERR_UNSUPPORTED;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (!ctx->verified || !ctx->shard_streamed || !same_round(ctx, d)) return SPECSTEER_ERR_ORDER;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  RoundParams p = slab_params(ctx, d, 0, d->B);
+  p.vocab_offset = vocab_offset;
+  p.greedy_keys = (long long*)best_keys;
+  if (launch_recover_argmax(p, d->dtype, rows_aligned(d), false, ctx->topk_lists, ctx->topk_count, ctx->li.sm_count,
+                            (cudaStream_t)cuda_stream) != cudaSuccess)
+    return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
+  return SPECSTEER_OK;
+}
+
+// Last step of a sharded greedy round, the same on every GPU.  Only the per-request arrays of the descriptor are used
+// (the LM-head rounds pass their embedded round descriptor, whose logit pointers are NULL).
+specsteer_status specsteer_shard_greedy_finish(specsteer_ctx* ctx, const specsteer_round_desc* d, const int64_t* best_keys,
+                                               void* cuda_stream) {
+  if (!ctx || !d || !best_keys) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->B < 0 || d->K < 0 || d->B > ctx->max_B || d->K > ctx->max_K || d->B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->recover_mode != SPECSTEER_RECOVER_ARGMAX) return SPECSTEER_ERR_UNSUPPORTED;
+  if (d->B > 0 && (!d->draft_len || !d->temperature || !d->accept_len || (d->K > 0 && !d->draft_tokens))) return SPECSTEER_ERR_INVALID_ARG;
+  if (ctx->poisoned) return SPECSTEER_ERR_TIMEOUT;
+  if (d->B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  specsteer_round_desc dd = *d;
+  dd.dtype = SPECSTEER_F32; dd.ld_row = d->V > 0 ? d->V : 1; dd.ld_req = (int64_t)(d->K + 1) * dd.ld_row;
+  RoundParams p = slab_params(ctx, &dd, 0, d->B);
+  if (launch_greedy_finish(p, (const long long*)best_keys, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
+  return SPECSTEER_OK;
+}
+
 namespace {
 // Checks an LM-head descriptor, makes sure the second workspace exists and fills the kernels' parameters.
 specsteer_status prep_lmhead(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, RoundParams* p, LmheadOperands* op) {
@@ -476,7 +518,6 @@ specsteer_status specsteer_lmhead_shard_local(specsteer_ctx* ctx, const specstee
   specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
   if (st != SPECSTEER_OK) return st;
   if (!row_partials || vocab_offset < 0 || ld->round.B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
-  if (ld->round.recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
   ctx->verified = false;
   ctx->shard_streamed = false;
   if (ld->round.B == 0) return SPECSTEER_OK;
@@ -488,7 +529,8 @@ specsteer_status specsteer_lmhead_shard_local(specsteer_ctx* ctx, const specstee
   // the "token met" words must start at zero: a token outside this shard leaves its row untouched
   if (cudaMemsetAsync(ctx->lm_tok, 0, (size_t)ld->round.B * (ld->round.K + 1) * 16, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
-  if (launch_lmhead(p, op, ctx->lm_tok, nullptr, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  const bool greedy = ld->round.recover_mode == SPECSTEER_RECOVER_ARGMAX;   // the per-tile keys carry global ids
+  if (launch_lmhead(p, op, ctx->lm_tok, greedy ? ctx->lm_keys : nullptr, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (launch_shard_rows(p, SPECSTEER_F32, (ShardPartial*)row_partials, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += 2;
@@ -503,7 +545,6 @@ specsteer_status specsteer_lmhead_shard_combine(specsteer_ctx* ctx, const specst
   specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
   if (st != SPECSTEER_OK) return st;
   if ((st = check_shard_args(&ld->round, gathered, n_shards, shard_rank, vocab_offset, vocab_total)) != SPECSTEER_OK) return st;
-  if (ld->round.recover_mode != SPECSTEER_RECOVER_STEER) return SPECSTEER_ERR_UNSUPPORTED;
   if (ld->round.B == 0) return SPECSTEER_OK;
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
@@ -532,6 +573,25 @@ specsteer_status specsteer_lmhead_shard_recover(specsteer_ctx* ctx, const specst
   p.n_shards = n_shards; p.shard_rank = shard_rank;
   p.vocab_offset = vocab_offset; p.vocab_total = vocab_total;
   if (launch_lmhead_recover(p, op, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 1;
+  return SPECSTEER_OK;
+}
+
+// Greedy recovery with the heads split along the vocabulary: this shard's best key per request, from the per-tile
+// keys the tensor-core pass of specsteer_lmhead_shard_local left (after specsteer_lmhead_shard_combine).
+specsteer_status specsteer_lmhead_shard_greedy_local(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, int64_t* best_keys,
+                                                     void* cuda_stream) {
+  RoundParams p;
+  LmheadOperands op;
+  specsteer_status st = prep_lmhead(ctx, ld, &p, &op);
+  if (st != SPECSTEER_OK) return st;
+  if (!best_keys || ld->round.B > kMaxSlabB) return SPECSTEER_ERR_INVALID_ARG;
+  if (ld->round.recover_mode != SPECSTEER_RECOVER_ARGMAX) return SPECSTEER_ERR_UNSUPPORTED;
+  if (ld->round.B == 0) return SPECSTEER_OK;
+  DeviceGuard g(ctx->device);
+  if (!g.ok) return SPECSTEER_ERR_CUDA;
+  p.greedy_keys = (long long*)best_keys;
+  if (launch_lmhead_argmax(p, ctx->lm_keys, (cudaStream_t)cuda_stream) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += 1;
   return SPECSTEER_OK;
 }

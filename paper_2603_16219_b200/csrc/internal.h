@@ -67,6 +67,9 @@ struct RoundParams {
   int vocab_offset, vocab_total;    // this shard covers global ids [vocab_offset, vocab_offset + V)
   // fused LM-head path: the logit tensors do not exist; the drafted tokens' logits were left here instead
   const float* tok_logits;          // [B*(K+1)][4] {h_LLM, h_SLM+, h_SLM-, unused} of the row's drafted token, or null
+  // greedy recovery in a sharded round: the argmax kernels leave this shard's best key per request here instead of
+  // writing the outputs ((order-preserving value bits << 31) | (0x7fffffff - global id); -1: no token), or null
+  long long* greedy_keys;
 };
 
 // The LM heads in front of the round: h = x W^T, all operands bf16, row-major, dense.
@@ -92,6 +95,8 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
 // or null when nobody needs them.
 cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, void* argmax_keys,
                           const LaunchInfo& li, cudaStream_t s);
+// Sharded greedy rounds, last step: the outputs from the keys every shard agreed on (MAX over shards).
+cudaError_t launch_greedy_finish(const RoundParams& p, const long long* keys, cudaStream_t s);
 // Greedy recovery from those keys.
 cudaError_t launch_lmhead_argmax(const RoundParams& p, const void* argmax_keys, cudaStream_t s);
 // Recovery (Eq. 8) from those records; the logits of the one chunk that holds the CDF target are recomputed.

@@ -369,7 +369,7 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->tmem_empty);  // the accumulators may be overwritten
       if (valid && p.argmax_keys)
-        p.argmax_keys[(long long)row * p.n_chunks + nb] = arg_r >= 0 ? entry_key(mx[Q_R], n0 + arg_r) : 0ull;
+        p.argmax_keys[(long long)row * p.n_chunks + nb] = arg_r >= 0 ? entry_key(mx[Q_R], n0 + arg_r + p.vocab_offset) : 0ull;
       if (valid) {
         const float2 rl = make_record(ref[Q_L], s[Q_L]), rp = make_record(ref[Q_P], s[Q_P]),
                      rm = make_record(ref[Q_M], s[Q_M]), rr = make_record(ref[Q_R], s[Q_R]);
@@ -651,7 +651,7 @@ __global__ void __launch_bounds__(256) lmhead_argmax_kernel(const RoundParams p,
   if (len < 0 || len > K) len = 0;
   const bool bad = (status & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
   const bool sample = !bad && (n < len || (p.flags & SPECSTEER_FLAG_BONUS));
-  if (p.out_tokens)
+  if (p.out_tokens && !p.greedy_keys)
     for (int t = tid; t <= K; t += 256)
       p.out_tokens[(long long)b * K1 + t] = (t < n) ? p.draft_tokens[(long long)b * K + t] : -1;
   const long long row = (long long)b * K1 + n;
@@ -670,6 +670,11 @@ __global__ void __launch_bounds__(256) lmhead_argmax_kernel(const RoundParams p,
   __syncthreads();
   if (tid != 0) return;
   for (int w = 1; w < 8; ++w) best = wbest[w] > best ? wbest[w] : best;
+  if (p.greedy_keys) {   // heads split along the vocabulary: the key (its id is already global) goes to the reduction over shards
+    const long long id = (long long)(0xffffffffu - (uint32_t)(best & 0xffffffffu));
+    p.greedy_keys[b] = (sample && best) ? (long long)(((best >> 32) << 31) | (u64)(0x7fffffffll - id)) : -1;
+    return;
+  }
   if (!sample || best == 0) {
     if (p.rec_token) p.rec_token[b] = -1;
     if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);

@@ -386,14 +386,18 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   const int K = p.K, K1 = K + 1;
   pdl_wait();
   const ReqState st = request_state(p, b);
-  if (sp == 0 && p.out_tokens)
+  if (sp == 0 && p.out_tokens && !p.greedy_keys)
     for (int t = tid; t <= K; t += kRecThreads)
       p.out_tokens[(long long)b * K1 + t] = (t < st.n) ? p.draft_tokens[(long long)b * K + t] : -1;
   if (!st.sample) {
     if (sp == 0 && tid == 0) {
-      if (p.rec_token) p.rec_token[b] = -1;
-      if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
-      if (p.n_out) p.n_out[b] = st.n;
+      if (p.greedy_keys) {
+        p.greedy_keys[b] = -1;
+      } else {
+        if (p.rec_token) p.rec_token[b] = -1;
+        if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+        if (p.n_out) p.n_out[b] = st.n;
+      }
     }
     return;
   }
@@ -507,6 +511,11 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
     }
     count_ws[b] = 0;
   }
+  if (p.greedy_keys) {   // sharded round: leave the key (with the global id) for the reduction over shards
+    const long long id = (long long)(0xffffffffu - (uint32_t)(best & 0xffffffffu)) + p.vocab_offset;
+    p.greedy_keys[b] = best ? (long long)(((best >> 32) << 31) | (u64)(0x7fffffffll - id)) : -1;
+    return;
+  }
   const long long row = (long long)b * K1 + st.n;
   double lseR;
   bool fin = best != 0;
@@ -532,6 +541,38 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   if (p.rec_logprob) p.rec_logprob[b] = (float)((r * (double)c - lseR) * 0.6931471805599453);
   if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
   if (p.n_out) p.n_out[b] = st.n + 1;
+}
+
+// Sharded greedy rounds, last step (identical on every GPU): outputs from the keys reduced over the shards.
+__global__ void __launch_bounds__(128) greedy_finish_kernel(const RoundParams p, const long long* keys) {
+  const int b = blockIdx.x * 128 + threadIdx.x;
+  if (b >= p.B) return;
+  const int K = p.K, K1 = K + 1;
+  const ReqState st = request_state(p, b);
+  if (p.out_tokens)
+    for (int t = 0; t <= K; ++t)
+      p.out_tokens[(long long)b * K1 + t] = (t < st.n) ? p.draft_tokens[(long long)b * K + t] : -1;
+  const long long key = keys[b];
+  if (!st.sample || key < 0) {
+    if (p.rec_token) p.rec_token[b] = -1;
+    if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+    if (p.n_out) p.n_out[b] = st.n;
+    return;
+  }
+  const int tok = (int)(0x7fffffffll - (key & 0x7fffffffll));
+  const double r = (double)order_val((uint32_t)((unsigned long long)key >> 31));
+  const long long row = (long long)b * K1 + st.n;
+  const double lseR = (double)p.lse2[row * 4 + Q_R];
+  if (p.rec_token) p.rec_token[b] = tok;
+  if (p.rec_logprob) p.rec_logprob[b] = (float)((r * (double)(kLog2e / p.temperature[b]) - lseR) * 0.6931471805599453);
+  if (p.out_tokens) p.out_tokens[(long long)b * K1 + st.n] = tok;
+  if (p.n_out) p.n_out[b] = st.n + 1;
+}
+
+cudaError_t launch_greedy_finish(const RoundParams& p, const long long* keys, cudaStream_t s) {
+  if (p.B == 0) return cudaSuccess;
+  greedy_finish_kernel<<<(p.B + 127) / 128, 128, 0, s>>>(p, keys);
+  return cudaGetLastError();
 }
 
 template <typename T>

@@ -77,6 +77,11 @@ def reduce_recovered(outputs: Dict[str, torch.Tensor], dist) -> None:
             dist.all_reduce(t, op=dist.ReduceOp.MAX)
 
 
+def reduce_keys(best_keys: torch.Tensor, dist) -> None:
+    """Element-wise MAX over ranks of the shards' best keys of a greedy round (int64 [B], in place)."""
+    dist.all_reduce(best_keys, op=dist.ReduceOp.MAX)
+
+
 def sharded_vocab_round(ctx, desc, outputs: Dict[str, torch.Tensor], vocab_offset: int, vocab_total: int, dist,
                         stream=None) -> torch.Tensor:
     """One verify + recover round over a vocabulary split across the ranks of `dist`.
@@ -89,6 +94,12 @@ def sharded_vocab_round(ctx, desc, outputs: Dict[str, torch.Tensor], vocab_offse
     ctx.shard_verify_local(desc, vocab_offset, parts, stream)
     gathered = gather_partials(parts, dist)
     ctx.shard_verify_combine(desc, gathered, rank, vocab_offset, vocab_total, stream)
+    if getattr(desc, "recover_mode", 0) == 2:     # greedy: every shard's best key, MAX over shards, then the outputs
+        keys = torch.empty(desc.B, dtype=torch.int64, device=outputs["accept_len"].device)
+        ctx.shard_greedy_local(desc, vocab_offset, keys, stream)
+        reduce_keys(keys, dist)
+        ctx.shard_greedy_finish(desc, keys, stream)
+        return gathered
     ctx.shard_recover_local(desc, gathered, rank, vocab_offset, vocab_total, stream)
     reduce_recovered(outputs, dist)
     return gathered
@@ -106,6 +117,12 @@ def sharded_lmhead_round(ctx, desc, outputs: Dict[str, torch.Tensor], vocab_offs
     ctx.lmhead_shard_local(desc, vocab_offset, parts, stream)
     gathered = gather_partials(parts, dist)
     ctx.lmhead_shard_combine(desc, gathered, rank, vocab_offset, vocab_total, stream)
+    if getattr(r, "recover_mode", 0) == 2:
+        keys = torch.empty(r.B, dtype=torch.int64, device=outputs["accept_len"].device)
+        ctx.lmhead_shard_greedy_local(desc, keys, stream)
+        reduce_keys(keys, dist)
+        ctx.shard_greedy_finish(desc, keys, stream)
+        return gathered
     ctx.lmhead_shard_recover(desc, gathered, rank, vocab_offset, vocab_total, stream)
     reduce_recovered(outputs, dist)
     return gathered

@@ -143,6 +143,16 @@ class _FakeShardCtx:
     _NAMES = {"shard_verify_local": "_local", "shard_verify_combine": "_combine", "shard_recover_local": "_recover",
               "lmhead_shard_local": "_local", "lmhead_shard_combine": "_combine", "lmhead_shard_recover": "_recover"}
 
+    def shard_greedy_local(self, desc, vocab_offset, keys, stream=None):
+        self.calls.append(("greedy_local", vocab_offset))
+        keys.copy_(torch.tensor([100 + self.rank, 7 - self.rank], dtype=torch.int64))   # rank 1 wins request 0, rank 0 request 1
+
+    def lmhead_shard_greedy_local(self, desc, keys, stream=None):
+        self.shard_greedy_local(desc, None, keys)
+
+    def shard_greedy_finish(self, desc, keys, stream=None):
+        self.calls.append(("greedy_finish", keys.tolist()))
+
     def __getattr__(self, name):
         if name in self._NAMES and name.startswith(self.prefix):
             return getattr(self, self._NAMES[name])
@@ -169,6 +179,16 @@ def _round_worker(rank, world, port, q):
             ok = ok and outs["accept_len"].tolist() == [3, 3]            # partials of rank 0 (1) and rank 1 (2)
             ok = ok and outs["rec_token"].tolist() == [11, 11] and outs["n_out"].tolist() == [1, 1]
             ok = ok and outs["rec_logprob"].tolist() == [-1.5, -1.5] and bool((outs["out_tokens"] == 11).all())
+        # greedy rounds: local keys, their MAX over the ranks, the common last step
+        for helper, prefix, desc in (
+                (sharding.sharded_vocab_round, "shard", types.SimpleNamespace(B=2, K=3, recover_mode=2)),
+                (sharding.sharded_lmhead_round, "lmhead_shard",
+                 types.SimpleNamespace(round=types.SimpleNamespace(B=2, K=3, recover_mode=2)))):
+            outs = {"accept_len": torch.zeros(2, dtype=torch.int32)}
+            fake = _FakeShardCtx(rank, outs, prefix)
+            helper(fake, desc, outs, 100 * rank, 200, dist)
+            ok = ok and [c[0] for c in fake.calls] == ["local", "combine", "greedy_local", "greedy_finish"]
+            ok = ok and fake.calls[-1][1] == [101, 7]
         q.put((rank, ok))
     finally:
         dist.destroy_process_group()

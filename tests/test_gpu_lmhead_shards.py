@@ -16,7 +16,7 @@ from test_gpu_lmhead import MARGIN, TOL, _np_inputs
 pytestmark = pytest.mark.gpu
 
 
-def _sharded(binding, sharding, inputs, G, accept_mode, flags, align=8):
+def _sharded(binding, sharding, inputs, G, accept_mode, flags, align=8, recover_mode=0):
     B, K1 = inputs["x_llm"].shape[:2]
     K = K1 - 1
     V = inputs["w_llm"].shape[0]
@@ -34,7 +34,7 @@ def _sharded(binding, sharding, inputs, G, accept_mode, flags, align=8):
             loc["w_slm_minus"] = loc["w_slm_plus"]           # keep the shared head shared
         ctx = binding.Context(B, K, hi - lo, device=0)
         o = binding.alloc_outputs(B, K, "cuda")
-        d = binding.make_lmhead_desc(loc, o, accept_mode=accept_mode, flags=flags)
+        d = binding.make_lmhead_desc(loc, o, accept_mode=accept_mode, recover_mode=recover_mode, flags=flags)
         keep.append(loc)
         ctxs.append(ctx); descs.append(d); outs.append(o)
         parts.append(torch.empty((B, K1, 64), dtype=torch.uint8, device="cuda"))
@@ -42,9 +42,18 @@ def _sharded(binding, sharding, inputs, G, accept_mode, flags, align=8):
     for g in live:
         ctxs[g].lmhead_shard_local(descs[g], ranges[g][0], parts[g])
     gathered = torch.stack([parts[g] for g in live], 0).contiguous()
+    keys = []
     for r, g in enumerate(live):
         ctxs[g].lmhead_shard_combine(descs[g], gathered, r, ranges[g][0], V)
-        ctxs[g].lmhead_shard_recover(descs[g], gathered, r, ranges[g][0], V)
+        if recover_mode == 2:
+            keys.append(torch.empty(B, dtype=torch.int64, device="cuda"))
+            ctxs[g].lmhead_shard_greedy_local(descs[g], keys[-1])
+        else:
+            ctxs[g].lmhead_shard_recover(descs[g], gathered, r, ranges[g][0], V)
+    if recover_mode == 2:
+        best = torch.stack(keys, 0).max(dim=0).values.contiguous()
+        for g in live:
+            ctxs[g].shard_greedy_finish(descs[g], best)
     torch.cuda.synchronize()
     for g in live:
         assert ctxs[g].device_error() == 0
@@ -110,4 +119,26 @@ def test_one_shard_equals_the_unsharded_entry_point(oracle_mod):
         assert np.array_equal(outs[k].cpu().numpy(), one[k]), k
     for k in ("logp_llm", "logp_minus", "logp_plus", "logp_star", "log_z", "rec_logprob"):
         assert np.allclose(outs[k].cpu().numpy(), one[k], atol=1e-5, equal_nan=True), k
+    ctx.close()
+
+
+
+@pytest.mark.parametrize("V,G,d_llm,d_slm", [(5000, 2, 192, 64), (20011, 3, 256, 128), (40000, 8, 320, 64)])
+def test_sharded_fused_greedy_round(oracle_mod, V, G, d_llm, d_slm):
+    """Greedy recovery with the heads split along the vocabulary: per-tile keys with global ids, each shard's best, the
+    maximum over shards, the common last step.  Token as for the unsharded fused round (margin on the runner-up gap)."""
+    from paper_2603_16219_b200 import binding, build, sharding, synth
+    build.build()
+    spec = synth.RoundSpec("lm_shards_greedy", 6, 3, V, "bf16", ragged=True, beta_choices=(0.5, 1.0, 2.0), temp_choices=(0.7, 1.0))
+    inputs = synth.make_lmhead_round(spec, d_llm, d_slm, device="cuda", seed=V + G + 1)
+    npin = _np_inputs(oracle_mod, inputs)
+    for flags in (1, 0):
+        gpu = _sharded(binding, sharding, inputs, G, 0, flags, recover_mode=2)
+        P.compare(oracle_mod, gpu, npin, 0, 2, flags, TOL, margin=MARGIN)
+    # and the sharded result is the unsharded fused greedy round's, token for token
+    ctx = binding.Context(spec.B, spec.K, V, device=0)
+    outs = binding.alloc_outputs(spec.B, spec.K, "cuda")
+    ctx.lmhead_round(binding.make_lmhead_desc(inputs, outs, recover_mode=2, flags=0))
+    torch.cuda.synchronize()
+    assert np.array_equal(outs["rec_token"].cpu().numpy(), gpu["rec_token"])
     ctx.close()
