@@ -32,7 +32,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per used row of the streaming kernel, from the ncu captures summarised under
 # profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows), keyed by
 # configuration.  Absent = not captured for the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_ROW = {3: 1856744, 4: 1559398}
+NCU_TRAFFIC_BYTES_PER_ROW = {3: 1858819, 4: 1558613}
 
 
 def _peaks():
