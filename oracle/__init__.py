@@ -33,6 +33,7 @@ DTYPE_F32, DTYPE_BF16, DTYPE_F64 = 0, 1, 2
 ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
 RECOVER_STEER, RECOVER_RESIDUAL, RECOVER_ARGMAX = 0, 1, 2
 FLAG_BONUS = 1
+FLAG_ALG1_READS = 2   # the round reading only what Algorithm 1 reads (see specsteer_oracle.h)
 REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1, 2, 4, 8, 16
 
 

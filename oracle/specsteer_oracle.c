@@ -16,8 +16,12 @@
  *   - Eq. 2-4 (fused target): P* = P_LLM * exp(r) / Z_t, r = log P+ - log P-.
  *   - Eq. 8 (recovery logits): h_rec = h_LLM + beta * (h_SLM+ - h_SLM-).
  *   - Greedy decoding (the experimental settings): ORACLE_RECOVER_ARGMAX takes the
- *     token of largest h_rec instead of sampling; the order is decided on h_rec as
- *     single precision forms it (see one_request).
+ *     token of largest h_rec (Eq. 8, over the reals: ordered in double) instead of
+ *     sampling, and reports the gap to the runner-up; the single-precision ordering
+ *     the CUDA library documents as its tie-break is reported beside it, not used.
+ *   - ORACLE_FLAG_ALG1_READS: the round reading exactly what Algorithm 1 reads:
+ *     h_LLM and h_SLM- on the drafted rows (Eq. 7), all three tensors only on the
+ *     row the new token comes from (Eq. 8).  h_SLM+ on a drafted row is never touched.
  * Every distribution is a softmax of logits divided by a per-request
  * temperature (the paper runs at temperature 1).  Logits may also be given in
  * double (ORACLE_DTYPE_F64): the LM-head oracle in __init__.py forms them as
@@ -27,7 +31,9 @@
  * to library log-softmax, hand-derived rational examples, the output-token law
  * by enumeration and Monte-Carlo, and the speculative-sampling theorem for the
  * EXACT_Z + RESIDUAL pair; greedy recovery by exact rationals, numpy argmax and
- * a float32 tie; the float64 logit decode and the LM-head step in
+ * a pair that only double precision separates; the Algorithm-1-reads round by
+ * equality with the full round on finite inputs and by poisoning what it must not
+ * read; the float64 logit decode and the LM-head step in
  * tests/test_oracle_lmhead_pins.py.  Parts with no pin: none of the functions below.
  *
  * No blocking, fusion or reordering: each log-sum-exp is "max, then sum of
@@ -94,6 +100,20 @@ static void row_load(row_t *w, int V, int dtype, const void *hl, const void *hp,
   w->lseP = specsteer_oracle_logsumexp(w->p, V);
   w->lseM = specsteer_oracle_logsumexp(w->m, V);
   w->lseR = specsteer_oracle_logsumexp(w->r, V);
+}
+
+/* What Eq. 7 reads of a drafted row: h_LLM and h_SLM- alone.  Everything that involves h_SLM+ is left NaN. */
+static void row_load_ratio(row_t *w, int V, int dtype, const void *hl, const void *hm, int64_t off, double T) {
+  for (int v = 0; v < V; ++v) {
+    w->ell[v] = logit_at(hl, dtype, off + v) / T;
+    w->m[v] = logit_at(hm, dtype, off + v) / T;
+    w->p[v] = NAN;
+    w->r[v] = NAN;
+  }
+  w->lseL = specsteer_oracle_logsumexp(w->ell, V);
+  w->lseM = specsteer_oracle_logsumexp(w->m, V);
+  w->lseP = NAN;
+  w->lseR = NAN;
 }
 
 static int row_finite(const row_t *w) {
@@ -177,12 +197,14 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
   int decided = 0, stop_nonfinite = 0;
   double rec_logprob = NAN;
 
+  /* every problem the request shows is reported: a bad length and a bad parameter give both bits */
+  const int alg1 = (a->flags & ORACLE_FLAG_ALG1_READS) != 0;
+  if (len < 0 || len > K) { status |= ORACLE_REQ_BAD_LEN; len = 0; }
   int params_ok = isfinite(T) && T > 0.0 && isfinite(lam) && lam > 0.0 && isfinite(beta);
   if (!params_ok) {
     status |= ORACLE_REQ_BAD_PARAM;
     goto done;
   }
-  if (len < 0 || len > K) { status |= ORACLE_REQ_BAD_LEN; len = 0; }
 
   /* Algorithm 1, the for-loop over draft positions.  The decision (n) is fixed at the first
    * rejection; later drafted rows are still evaluated so that their per-position diagnostics
@@ -191,13 +213,20 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
   for (int t = 0; t < len; ++t) {
     int64_t off = (int64_t)b * a->ld_req + (int64_t)t * a->ld_row;
     int64_t i = (int64_t)b * K + t;
-    row_load(w, V, a->dtype, a->h_llm, a->h_slm_plus, a->h_slm_minus, off, beta, T);
-    if (!row_finite(w)) {
+    int fin;
+    if (alg1) {   /* Algorithm 1's verification: the cloud holds h_LLM and h_SLM- only (Eq. 7) */
+      row_load_ratio(w, V, a->dtype, a->h_llm, a->h_slm_minus, off, T);
+      fin = isfinite(w->lseL) && isfinite(w->lseM);
+    } else {
+      row_load(w, V, a->dtype, a->h_llm, a->h_slm_plus, a->h_slm_minus, off, beta, T);
+      fin = row_finite(w);
+    }
+    if (!fin) {
       if (!decided) { status |= ORACLE_REQ_NONFINITE; n = t; decided = 1; stop_nonfinite = 1; }
       continue;
     }
     double logZ = w->lseR - w->lseL - beta * (w->lseP - w->lseM);  /* log sum_v P_LLM (P+/P-)^beta; Eq. 2 at beta=1 */
-    if (a->log_z) a->log_z[(int64_t)b * (K + 1) + t] = logZ;
+    if (a->log_z && !alg1) a->log_z[(int64_t)b * (K + 1) + t] = logZ;
     int y = yhat[t];
     double al = 0.0, rho = 0.0;
     int accept, testable = 1;   /* a bad token or an undefined ratio is a rejection whatever the uniform */
@@ -209,8 +238,8 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
       double logpP = w->p[y] - w->lseP, logpS = w->r[y] - w->lseR;
       if (a->logp_llm) a->logp_llm[i] = logpL;
       if (a->logp_minus) a->logp_minus[i] = logpM;
-      if (a->logp_plus) a->logp_plus[i] = logpP;
-      if (a->logp_star) a->logp_star[i] = logpS;
+      if (a->logp_plus && !alg1) a->logp_plus[i] = logpP;
+      if (a->logp_star && !alg1) a->logp_star[i] = logpS;
       double logrho = (a->accept_mode == ORACLE_ACCEPT_RATIO)
                           ? (logpL - logpM - log(lam))   /* Eq. 7 */
                           : (logpS - logpP);             /* Eq. 6 */
@@ -230,7 +259,7 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
   for (int t = 0; t < n; ++t) if (a->out_tokens) a->out_tokens[(int64_t)b * (K + 1) + t] = yhat[t];
   n_out = n;
   /* diagnostic: with FLAG_BONUS row `len` belongs to the round, so its log Z_t is reported whatever n is */
-  if ((a->flags & ORACLE_FLAG_BONUS) && a->log_z) {
+  if ((a->flags & ORACLE_FLAG_BONUS) && a->log_z && !alg1) {
     row_load(w, V, a->dtype, a->h_llm, a->h_slm_plus, a->h_slm_minus,
              (int64_t)b * a->ld_req + (int64_t)len * a->ld_row, beta, T);
     if (row_finite(w)) a->log_z[(int64_t)b * (K + 1) + len] = w->lseR - w->lseL - beta * (w->lseP - w->lseM);
@@ -244,37 +273,39 @@ static void one_request(const oracle_round_args *a, int b, row_t *w, double *wgt
     if (!row_finite(w)) { status |= ORACLE_REQ_NONFINITE; goto done; }
     if (a->recover_mode == ORACLE_RECOVER_ARGMAX) {
       /* Greedy decoding (the paper's experimental setting): y_new is the token of largest h_rec (Eq. 8), the lowest
-       * id among equals, on the rejection row and on the bonus row alike.  The comparison is made on h_rec as single
-       * precision forms it, fl(h_LLM + beta * fl(h_SLM+ - h_SLM-)) with one fused multiply-add, so that ties are the
-       * same everywhere (float32 and bf16 logits); the temperature does not change the order.  Its log-probability is the one under
-       * Softmax(h_rec / T). */
-      double gap = INFINITY;   /* reported in cdf_margin: distance to the runner-up where the order is not exact */
-      if (a->dtype == ORACLE_DTYPE_F64) {
-        /* logits that were themselves computed (the LM-head path): nobody can reproduce their last bits, so the
-         * order is taken in double and the gap between the two largest values is reported for the comparison */
-        double best = -INFINITY, second = -INFINITY;
-        for (int v = 0; v < V; ++v) {
-          double r = logit_at(a->h_llm, a->dtype, off + v) +
-                     beta * (logit_at(a->h_slm_plus, a->dtype, off + v) - logit_at(a->h_slm_minus, a->dtype, off + v));
-          if (rec_token < 0 || r > best) { second = best; best = r; rec_token = v; }
-          else if (r > second) second = r;
-        }
-        gap = best - second;
-      } else {
+       * id among equals, on the rejection row and on the bonus row alike; the temperature does not change the order.
+       * Its log-probability is the one under Softmax(h_rec / T). */
+      /* The order of Eq. 8 over the reals: h_rec is formed and compared in double from the exactly upcast logits.
+       * cdf_margin reports the gap between the largest and the second largest value (0 for an exact tie), so that a
+       * comparison can tell a decided order from one that rounding in a narrower type may turn around. */
+      double best = -INFINITY, second = -INFINITY;
+      for (int v = 0; v < V; ++v) {
+        double r = logit_at(a->h_llm, a->dtype, off + v) +
+                   beta * (logit_at(a->h_slm_plus, a->dtype, off + v) - logit_at(a->h_slm_minus, a->dtype, off + v));
+        if (rec_token < 0 || r > best) { second = best; best = r; rec_token = v; }
+        else if (r > second) second = r;
+      }
+      double gap = best - second;
+      /* Beside it, not used for anything above: the token the single-precision form of Eq. 8 would order first,
+       * fl(h_LLM + beta * fl(h_SLM+ - h_SLM-)) with one fused multiply-add, lowest id among equals - the rule the CUDA
+       * library documents for breaking what double precision calls a near-tie.  Reported in rec_token_lo. */
+      int tie_token = rec_token;
+      if (a->dtype != ORACLE_DTYPE_F64) {
         const float beta32 = a->beta[b];
-        float best = -INFINITY;
+        float best32 = -INFINITY;
+        tie_token = -1;
         for (int v = 0; v < V; ++v) {
           float l = (float)logit_at(a->h_llm, a->dtype, off + v), pp = (float)logit_at(a->h_slm_plus, a->dtype, off + v),
                 mm = (float)logit_at(a->h_slm_minus, a->dtype, off + v);
           float r = fmaf(beta32, pp - mm, l);
-          if (rec_token < 0 || r > best) { best = r; rec_token = v; }
+          if (tie_token < 0 || r > best32) { best32 = r; tie_token = v; }
         }
       }
       rec_logprob = w->r[rec_token] - w->lseR;
       if (a->out_tokens) a->out_tokens[(int64_t)b * (K + 1) + n] = rec_token;
       n_out = n + 1;
       if (a->cdf_margin) a->cdf_margin[b] = gap;   /* no uniform is involved */
-      if (a->rec_token_lo) a->rec_token_lo[b] = rec_token;
+      if (a->rec_token_lo) a->rec_token_lo[b] = tie_token;
       if (a->rec_token_hi) a->rec_token_hi[b] = rec_token;
       goto done;
     }
@@ -313,6 +344,8 @@ done:
 int specsteer_oracle_round(const oracle_round_args *a) {
   if (!a || a->B < 0 || a->K < 0 || a->V <= 0 || a->ld_row < a->V || !a->accept_len) return -1;
   if (a->ld_req < (int64_t)(a->K + 1) * a->ld_row) return -1;
+  /* Eq. 6 needs P_SLM+ and Z_t on every drafted row: it cannot be evaluated from what Algorithm 1's verification reads */
+  if ((a->flags & ORACLE_FLAG_ALG1_READS) && a->accept_mode != ORACLE_ACCEPT_RATIO) return -3;
   int nthreads = a->nthreads > 0 ? a->nthreads : 1;
   int failed = 0;
 #ifdef _OPENMP

@@ -15,7 +15,10 @@ enum { ORACLE_DTYPE_F32 = 0, ORACLE_DTYPE_BF16 = 1, ORACLE_DTYPE_F64 = 2 };
 enum { ORACLE_ACCEPT_RATIO = 0 /* Eq. 7 */, ORACLE_ACCEPT_EXACT_Z = 1 /* Eq. 6 */ };
 enum { ORACLE_RECOVER_STEER = 0 /* Eq. 8 softmax */, ORACLE_RECOVER_RESIDUAL = 1,
        ORACLE_RECOVER_ARGMAX = 2 /* greedy decoding: the token of largest h_rec (Eq. 8) */ };
-enum { ORACLE_FLAG_BONUS = 1u };
+enum { ORACLE_FLAG_BONUS = 1u,
+       /* read what Algorithm 1 reads: h_LLM and h_SLM- on drafted rows (Eq. 7; RATIO only), all three tensors on the row
+        * the new token comes from (Eq. 8).  logp_plus, logp_star and log_z are then not defined (NaN). */
+       ORACLE_FLAG_ALG1_READS = 2u };
 enum {
   ORACLE_REQ_BAD_TOKEN = 1, ORACLE_REQ_BAD_LEN = 2, ORACLE_REQ_NONFINITE = 4,
   ORACLE_REQ_RESIDUAL_EMPTY = 8, ORACLE_REQ_BAD_PARAM = 16
@@ -44,8 +47,10 @@ typedef struct {
   int32_t *out_tokens;                 /* [B][K+1] */
   int32_t *n_out, *req_status;         /* [B] */
   double *accept_margin;               /* [B][K]: distance of u from the decision boundary */
-  double *cdf_margin;                  /* [B]: distance of the CDF target from the chosen interval's ends, / W */
-  int32_t *rec_token_lo, *rec_token_hi;/* [B]: tokens picked at target -/+ margin_tol*W */
+  double *cdf_margin;                  /* [B]: distance of the CDF target from the chosen interval's ends, / W;
+                                          ARGMAX: the gap between the two largest h_rec, in double */
+  int32_t *rec_token_lo, *rec_token_hi;/* [B]: tokens picked at target -/+ margin_tol*W; ARGMAX: lo = the token the
+                                          single-precision form of Eq. 8 orders first (a tie-break rule, reported only) */
 } oracle_round_args;
 
 /* One whole round for B requests (Algorithm 1 phases 2 and 3).  Returns 0, or <0 on bad arguments / no memory. */

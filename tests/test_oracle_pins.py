@@ -70,15 +70,20 @@ def test_log_z_is_partition_function_of_eq2(oracle_mod):
     tok = rng.integers(0, V, (B, K)).astype(np.int32)
     beta = np.array([1.0, 0.5, 2.0], np.float32)
     T = np.array([1.0, 0.7, 1.3], np.float32)
-    out = _round(oracle_mod, L, P, M, tok, rng.random((B, K), np.float32), rng.random(B, np.float32),
-                 beta=beta, T=T, flags=oracle_mod.FLAG_BONUS)
+    length = np.array([2, 1, 2], np.int32)
+    u_acc = np.array([[0.0, 1.0], [0.0, 0.0], [0.0, 0.0]], np.float32)     # request 0 is rejected at position 1
+    out = _round(oracle_mod, L, P, M, tok, u_acc, rng.random(B, np.float32),
+                 lam=np.array([1e6, 0.5, 0.5], np.float32), beta=beta, T=T, length=length, flags=oracle_mod.FLAG_BONUS)
+    assert out["accept_len"].tolist() == [1, 1, 2]
     for b in range(B):
         pl, pp, pm = (sps.softmax(a[b].astype(np.float64) / float(T[b]), axis=-1) for a in (L, P, M))
         z = (pl * (pp / pm) ** float(beta[b])).sum(-1)
-        n = out["accept_len"][b]
-        rows = list(range(K)) + ([K] if n == K else [])
-        np.testing.assert_allclose(out["log_z"][b, rows], np.log(z[rows]), atol=1e-10)
-        for t in range(K):
+        # rows 0 .. draft_len: with the bonus row part of the round, its log Z_t is reported whatever accept_len is
+        # (request 0 stops at position 1 and still reports row 2); rows beyond draft_len are not read
+        ln = int(length[b])
+        np.testing.assert_allclose(out["log_z"][b, :ln + 1], np.log(z[:ln + 1]), atol=1e-10)
+        assert np.isnan(out["log_z"][b, ln + 1:]).all()
+        for t in range(ln):
             y = tok[b, t]
             assert out["logp_llm"][b, t] == pytest.approx(np.log(pl[t, y]), abs=1e-10)
             assert out["logp_plus"][b, t] == pytest.approx(np.log(pp[t, y]), abs=1e-10)
@@ -330,6 +335,75 @@ def test_status_words_and_degenerate_inputs(oracle_mod):
     assert out["req_status"][3] == o.REQ_BAD_PARAM and out["n_out"][3] == 0 and out["rec_token"][3] == -1
     assert out["req_status"][4] == 0 and out["accept_len"][4] == 0 and out["n_out"][4] == 1
     assert out["req_status"][5] == o.REQ_NONFINITE and out["accept_len"][5] == 0 and out["n_out"][5] == 0
+    # every problem a request shows is reported: a bad length together with a bad parameter gives both bits
+    length[3] = -1
+    out = _round(o, L, P, M, tok, u, np.full(B, 0.5, np.float32), T=T, length=length, flags=o.FLAG_BONUS)
+    assert out["req_status"][3] == (o.REQ_BAD_PARAM | o.REQ_BAD_LEN) and out["n_out"][3] == 0 and out["accept_len"][3] == 0
+
+
+# ---------------------------------------------------------------- the round reading what Algorithm 1 reads
+def test_alg1_reads_equals_the_full_round_on_finite_inputs(oracle_mod):
+    """Algorithm 1 Phase 2 uses P_LLM and P_SLM- only (Eq. 7) and Phase 3 the three logit rows of one position
+    (Eq. 8).  On finite inputs the round that reads nothing else decides, samples and reports exactly what the full
+    round does; what it never forms (logp_plus, logp_star, log_z) stays NaN.  Acceptance against scipy's softmax."""
+    o = oracle_mod
+    rng = np.random.default_rng(50)
+    B, K, V = 12, 3, 97
+    L, P, M = _rand_rows(rng, B, K, V)
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    ua, ur = rng.random((B, K)).astype(np.float32), rng.random(B).astype(np.float32)
+    length = rng.integers(0, K + 1, B).astype(np.int32)
+    beta = rng.choice([0.5, 1.0, 2.0], B).astype(np.float32)
+    T = rng.choice([0.7, 1.0], B).astype(np.float32)
+    lam = rng.choice([0.5, 2.0, 8.0], B).astype(np.float32)
+    for rmode in (o.RECOVER_STEER, o.RECOVER_ARGMAX):
+        for fl in (0, o.FLAG_BONUS):
+            full = _round(o, L, P, M, tok, ua, ur, lam=lam, beta=beta, T=T, length=length, recover_mode=rmode, flags=fl)
+            alg1 = _round(o, L, P, M, tok, ua, ur, lam=lam, beta=beta, T=T, length=length, recover_mode=rmode,
+                          flags=fl | o.FLAG_ALG1_READS)
+            for k in ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "rec_token", "rec_logprob",
+                      "out_tokens", "n_out", "req_status", "accept_margin", "cdf_margin"):
+                assert np.array_equal(full[k], alg1[k], equal_nan=True), k
+            for k in ("logp_plus", "logp_star", "log_z"):
+                assert np.isnan(alg1[k]).all(), k
+    assert (full["accept_len"] < length).any() and (full["accept_len"] == length).any()
+    for b in range(B):
+        pl = sps.softmax(L[b].astype(np.float64) / float(T[b]), -1)
+        pm = sps.softmax(M[b].astype(np.float64) / float(T[b]), -1)
+        for t in range(int(length[b])):
+            y = tok[b, t]
+            assert alg1["alpha"][b, t] == pytest.approx(min(1.0, pl[t, y] / (float(lam[b]) * pm[t, y])), abs=1e-12)   # Eq. 7
+
+
+def test_alg1_reads_never_touches_h_slm_plus_on_drafted_rows(oracle_mod):
+    """NaN in h_SLM+ everywhere except the row the new token comes from changes nothing; NaN or +inf on that row
+    is a non-finite recovery row; Eq. 6 cannot be asked of this round."""
+    o = oracle_mod
+    rng = np.random.default_rng(51)
+    B, K, V = 10, 3, 61
+    L, P, M = _rand_rows(rng, B, K, V)
+    tok = rng.integers(0, V, (B, K)).astype(np.int32)
+    ua, ur = rng.random((B, K)).astype(np.float32), rng.random(B).astype(np.float32)
+    for fl in (0, o.FLAG_BONUS):
+        clean = _round(o, L, P, M, tok, ua, ur, lam=2.0, flags=fl | o.FLAG_ALG1_READS)
+        Pn = np.full_like(P, np.nan)
+        for b in range(B):
+            Pn[b, clean["accept_len"][b]] = P[b, clean["accept_len"][b]]
+        got = _round(o, L, Pn, M, tok, ua, ur, lam=2.0, flags=fl | o.FLAG_ALG1_READS)
+        for k in clean:
+            assert np.array_equal(clean[k], got[k], equal_nan=True), k
+        assert (got["req_status"] == 0).all()
+        # the full round sees the poison on the first drafted row
+        assert (_round(o, L, Pn, M, tok, ua, ur, lam=2.0, flags=fl)["req_status"][clean["accept_len"] > 0] == o.REQ_NONFINITE).all()
+        assert (clean["accept_len"] > 0).any() and (clean["accept_len"] < K).any()
+    b = int(np.argmax(clean["rec_token"] >= 0))
+    Pbad = P.copy()
+    Pbad[b, clean["accept_len"][b], 7] = np.inf
+    got = _round(o, L, Pbad, M, tok, ua, ur, lam=2.0, flags=o.FLAG_BONUS | o.FLAG_ALG1_READS)
+    assert got["req_status"][b] == o.REQ_NONFINITE and got["rec_token"][b] == -1
+    assert got["accept_len"][b] == clean["accept_len"][b] and got["n_out"][b] == clean["accept_len"][b]
+    with pytest.raises(RuntimeError):
+        _round(o, L, P, M, tok, ua, ur, accept_mode=o.ACCEPT_EXACT_Z, flags=o.FLAG_ALG1_READS)
 
 
 def test_forced_decisions_and_margins(oracle_mod):
@@ -376,7 +450,9 @@ def test_argmax_recovery_is_the_first_maximiser_of_h_rec(oracle_mod, beta):
         assert g["out_tokens"][b][n] == want and (g["out_tokens"][b][:n] == tok[b][:n]).all()
         hr = np.array([float(x) for x in h])
         assert g["rec_logprob"][b] == pytest.approx(sps.log_softmax(hr)[want], abs=1e-12)
-        assert np.isinf(g["cdf_margin"][b])
+        runner_up = max(h[v] for v in range(V) if v != want)
+        assert g["cdf_margin"][b] == float(h[want] - runner_up)       # the gap to the runner-up, exact on this grid
+        assert g["rec_token_lo"][b] == want                           # float32 forms these values exactly too
 
 
 def test_argmax_recovery_with_beta_zero_is_numpy_argmax_of_the_generalist(oracle_mod):
@@ -409,23 +485,50 @@ def test_argmax_recovery_ignores_the_temperature_but_reports_the_tempered_probab
     assert np.array_equal(toks[0], toks[1]) and np.array_equal(toks[1], toks[2])
 
 
-def test_argmax_recovery_decides_on_single_precision_values(oracle_mod):
-    """Two entries whose exact h_rec differ by 2^-30: equal once formed in float32, so the lower id wins (exact
-    arithmetic would pick the other).  A difference float32 does resolve is honoured."""
+def test_argmax_recovery_orders_h_rec_over_the_reals_and_reports_what_single_precision_would_do(oracle_mod):
+    """Two entries whose exact h_rec differ by 2^-30 (Eq. 8 is a statement about real numbers): the larger one is
+    the token, the gap is 2^-30, and the token single precision would order first - there the two are equal, so the
+    lower id - is reported beside it without deciding anything.  A difference float32 resolves moves both."""
     o = oracle_mod
     L = np.array([[[1.0, 1.0, 0.0]]], np.float32)
     P = np.array([[[0.0, 2.0 ** -30, 0.0]]], np.float32)
     M = np.zeros((1, 1, 3), np.float32)
     kw = dict(tok=np.zeros((1, 0), np.int32), u_acc=np.zeros((1, 0), np.float32), u_rec=np.zeros(1, np.float32),
               recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
-    assert _round(o, L, P, M, **kw)["rec_token"][0] == 0
+    g = _round(o, L, P, M, **kw)
+    assert g["rec_token"][0] == 1 and g["cdf_margin"][0] == 2.0 ** -30 and g["rec_token_lo"][0] == 0
+    assert g["out_tokens"][0][0] == 1 and g["rec_token_hi"][0] == 1
+    assert g["rec_logprob"][0] == pytest.approx(sps.log_softmax(np.array([1.0, 1.0 + 2.0 ** -30, 0.0]))[1], abs=1e-15)
     P[0, 0, 1] = 2.0 ** -20
-    assert _round(o, L, P, M, **kw)["rec_token"][0] == 1
+    g = _round(o, L, P, M, **kw)
+    assert g["rec_token"][0] == 1 and g["rec_token_lo"][0] == 1 and g["cdf_margin"][0] == 2.0 ** -20
+    # bf16 logits go the same way (their values are exact in both precisions)
+    bits = lambda a: (a.view(np.uint32) >> 16).astype(np.uint16)
+    P[0, 0, 1] = 2.0 ** -30
+    g = _round(o, bits(L), bits(P), bits(M), **kw)
+    assert g["rec_token"][0] == 1 and g["rec_token_lo"][0] == 0 and g["cdf_margin"][0] == 2.0 ** -30
+
+
+def test_argmax_recovery_on_float32_logits_is_numpy_argmax_in_double(oracle_mod):
+    """Random float32 rows, several beta: the token is numpy's argmax of h_rec formed in double, the gap the
+    difference of its two largest values."""
+    o = oracle_mod
+    rng = np.random.default_rng(44)
+    B, V = 5, 2003
+    L, P, M = _rand_rows(rng, B, 0, V)
+    beta = np.array([1.0, 0.5, 2.0, 0.3, 2.7], np.float32)
+    g = _round(o, L, P, M, np.zeros((B, 0), np.int32), np.zeros((B, 0), np.float32), np.zeros(B, np.float32), beta=beta,
+               recover_mode=o.RECOVER_ARGMAX, flags=o.FLAG_BONUS)
+    for b in range(B):
+        r = L[b, 0].astype(np.float64) + float(beta[b]) * (P[b, 0].astype(np.float64) - M[b, 0].astype(np.float64))
+        assert g["rec_token"][b] == int(np.argmax(r))
+        top2 = np.sort(r)[-2:]
+        assert g["cdf_margin"][b] == pytest.approx(top2[1] - top2[0], abs=1e-15)
 
 
 def test_argmax_recovery_on_float64_logits_orders_in_double_and_reports_the_gap(oracle_mod):
     """Logits that were themselves computed (float64): numpy's argmax of h_rec in double, lowest id among equals, and
-    the distance to the runner-up in cdf_margin (float32 logits report +inf there: their order is exact)."""
+    the distance to the runner-up in cdf_margin."""
     o = oracle_mod
     rng = np.random.default_rng(43)
     B, V = 4, 3001
@@ -447,4 +550,4 @@ def test_argmax_recovery_on_float64_logits_orders_in_double_and_reports_the_gap(
                                np.zeros(B, np.int32), np.ones(B, np.float32), beta, np.ones(B, np.float32),
                                np.zeros((B, 0), np.float32), np.zeros(B, np.float32), recover_mode=o.RECOVER_ARGMAX,
                                flags=o.FLAG_BONUS)
-    assert np.isinf(f["cdf_margin"]).all()
+    assert np.isfinite(f["cdf_margin"]).all() and f["cdf_margin"][1] == 0.0 and f["rec_token"][1] == 77
