@@ -1,7 +1,9 @@
 """GPU parity of greedy recovery (SPECSTEER_RECOVER_ARGMAX: the token of largest h_rec, Eq. 8; the paper decodes
-greedily) with the oracle.  Both sides form h_rec in float32 with one fused multiply-add, so the token must be
-identical on every request whose accepted length agrees (an accept decision may still differ where the oracle's
-margin is below 1e-5; compare() then forces it in the oracle); no margin applies to the token itself.
+greedily) with the oracle.  The oracle orders h_rec in double; the GPU forms it in float32 with one fused
+multiply-add.  compare() demands the oracle's token wherever the gap to the runner-up exceeds the float32 rounding
+of the three terms, a token inside that near-tie set otherwise, and in every case the token the documented float32
+tie-break picks.  An accept decision may differ where the oracle's margin is below 1e-5 (it is then forced in the
+oracle).
 """
 import numpy as np
 import pytest
@@ -23,13 +25,14 @@ def env(oracle_mod):
     ctx.close()
 
 
-def _check(env, inputs, flags=1, accept_mode=0, V=None, sel=None):
+def _check(env, inputs, flags=1, accept_mode=0, V=None, sel=None, near_ties=0):
     gpu = P.run_gpu(env["ctx"], inputs, accept_mode, ARGMAX, flags, V=V)
     npin = P.to_np_inputs(inputs, None if sel is None else torch.as_tensor(sel, device="cuda"))
     if V is not None:
         npin = {k: (np.ascontiguousarray(v[..., :V]) if k.startswith("h_") else v) for k, v in npin.items()}
     stats = P.compare(env["oracle"], gpu, npin, accept_mode, ARGMAX, flags, P.TOL[inputs["h_llm"].dtype], V=V, sel=sel)
-    assert stats["excused_token"] == 0
+    print("greedy", stats)
+    assert stats["excused_token"] <= near_ties     # tokens that differ from the double-precision order (near-ties)
     return gpu
 
 
@@ -87,20 +90,31 @@ def test_ragged_no_bonus_exact_rule_and_bad_requests(env):
     assert ((gpu["rec_token"] >= 0) == (gpu["accept_len"] < dl))[ok].all()
 
 
-def test_full_size_float32_sampled(env):
-    synth = env["synth"]
-    spec = synth.CONFIGS[3]
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_full_size_every_request(env, cfg):
+    """The two largest configurations, every request: one-pass greedy round with every output, then the two-phase
+    greedy round against the oracle round that reads only what Algorithm 1 reads."""
+    synth, b = env["synth"], env["binding"]
+    spec = synth.CONFIGS[cfg]
     inputs = synth.make_round(spec, device="cuda", seed=0)
-    sel = np.unique(np.linspace(0, spec.B - 1, 10).astype(int))
-    gpu = _check(env, inputs, sel=sel)
-    P.invariants(gpu, inputs, 1, P.TOL[torch.float32])
-    # every request, against a float32 restatement on the device, as a property that holds at any size
-    n = torch.as_tensor(gpu["accept_len"], device="cuda").long()
-    rows = torch.arange(spec.B, device="cuda")
-    l, p, m = (inputs[k][rows, n] for k in ("h_llm", "h_slm_plus", "h_slm_minus"))
-    r = torch.addcmul(l, inputs["beta"][:, None], p - m)
-    got = r[rows, torch.as_tensor(gpu["rec_token"], device="cuda").long()]
-    assert ((r.max(dim=1).values - got) <= 1e-5).all()      # torch may round the product and the sum separately
+    gpu = _check(env, inputs, near_ties=spec.B // 64)
+    P.invariants(gpu, inputs, 1, P.TOL[inputs["h_llm"].dtype])
+    keys = ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "rec_token", "rec_logprob", "out_tokens",
+            "n_out", "req_status")
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k in keys}
+    d = b.make_desc(inputs, outs, recover_mode=ARGMAX, flags=1)
+    before = env["ctx"].launch_count
+    env["ctx"].verify_round(d)
+    env["ctx"].recover_sample(d)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 3
+    two = {k: v.cpu().numpy() for k, v in outs.items()}
+    stats = P.compare(env["oracle"], two, P.to_np_inputs(inputs), 0, ARGMAX, 1, P.TOL[inputs["h_llm"].dtype], alg1=True,
+                      keys=keys)
+    print(spec.name, "two-phase greedy", stats)
+    assert stats["requests"] == spec.B and stats["excused_token"] <= spec.B // 64
+    for k in ("accept_len", "rec_token", "n_out", "out_tokens", "req_status", "accept_flags"):
+        assert np.array_equal(two[k], gpu[k]), k
 
 
 def test_host_round_in_greedy_mode(env):
@@ -132,7 +146,7 @@ def test_two_phase_greedy_round(env, dtype, flags):
     inputs["h_slm_plus"][3, 0, 5] = float("inf")
     inputs["lam"][4] = 1e30
     inputs["h_slm_plus"][4, 0, :] = float("-inf")    # h_SLM+ is -inf throughout the recovery row: only that pass can tell
-    ora = P.run_oracle(env["oracle"], P.to_np_inputs(inputs), 0, ARGMAX, flags)
+    ora = P.run_oracle(env["oracle"], P.to_np_inputs(inputs), 0, ARGMAX, flags, alg1=True)
     hp = inputs["h_slm_plus"].clone()
     keep = torch.zeros(hp.shape[:2], dtype=torch.bool, device="cuda")
     for r in range(spec.B):
@@ -142,8 +156,9 @@ def test_two_phase_greedy_round(env, dtype, flags):
     hp[~keep] = float("nan")
     poisoned = dict(inputs)
     poisoned["h_slm_plus"] = hp
-    skip = ("logp_plus", "logp_star", "log_z")
-    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k not in skip}
+    keys = ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "rec_token", "rec_logprob", "out_tokens",
+            "n_out", "req_status")
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k in keys}
     d = b.make_desc(poisoned, outs, recover_mode=ARGMAX, flags=flags | b.FLAG_TWO_PHASE)
     before = env["ctx"].launch_count
     env["ctx"].verify_round(d)
@@ -152,18 +167,12 @@ def test_two_phase_greedy_round(env, dtype, flags):
     assert env["ctx"].device_error() == 0
     assert env["ctx"].launch_count - before == 3
     gpu = {k: v.cpu().numpy() for k, v in outs.items()}
-    safe = (ora["accept_margin"] > P.MARGIN).all(axis=1)
-    assert safe.sum() >= spec.B - 1
-    for k in ("accept_len", "rec_token", "n_out", "req_status", "out_tokens"):
-        assert np.array_equal(gpu[k][safe], ora[k][safe]), k
+    # every request, the poisoned tensors on both sides: the oracle round that reads what Algorithm 1 reads
+    stats = P.compare(env["oracle"], gpu, P.to_np_inputs(poisoned), 0, ARGMAX, flags, P.TOL[inputs["h_llm"].dtype],
+                      alg1=True, keys=keys)
+    assert stats["requests"] == spec.B and stats["excused_token"] == 0
     assert gpu["req_status"][3] == b.REQ_NONFINITE and gpu["rec_token"][3] == -1 and gpu["accept_len"][3] == 0
     assert gpu["req_status"][4] == b.REQ_NONFINITE and gpu["rec_token"][4] == -1 and gpu["accept_len"][4] == 0
-    safe[3] = safe[4] = False   # their per-position diagnostics differ by design: the oracle reads h_SLM+ on drafted rows
-    tol = P.TOL[inputs["h_llm"].dtype]
-    for k in ("alpha", "logp_llm", "logp_minus", "rec_logprob"):
-        fin = np.isfinite(ora[k]) & (safe[:, None] if ora[k].ndim == 2 else safe)
-        assert np.array_equal(np.isnan(gpu[k][safe]), np.isnan(ora[k][safe])), k
-        assert np.abs(gpu[k][fin] - ora[k][fin]).max(initial=0.0) <= tol, k
 
 
 def test_two_phase_greedy_full_size_equals_one_pass(env):
