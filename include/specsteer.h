@@ -78,7 +78,8 @@ enum {
                                    below which its two extra launches cost more than the bytes it saves */
 };
 
-/* bits of req_status[b] */
+/* bits of req_status[b].  Every problem a request shows is reported: a bad length together with a bad parameter gives
+ * both bits (BAD_LEN | BAD_PARAM); BAD_TOKEN and NONFINITE are reported only for rows up to the first rejection. */
 enum {
   SPECSTEER_REQ_BAD_TOKEN = 1,      /* a reached draft token outside [0,V): that position is a rejection, alpha 0 */
   SPECSTEER_REQ_BAD_LEN = 2,        /* draft_len outside [0,K]: treated as 0 */
@@ -294,9 +295,10 @@ specsteer_status specsteer_round_host(specsteer_ctx *ctx, const specsteer_round_
  * a workspace; this call instead keeps its workspace in a fixed 8 MiB array that is part of the library's
  * device image, so every GPU that loads the library holds those 8 MiB until the process exits.
  *
- * It runs the same two kernels as specsteer_verify_round (same descriptor, same outputs, same error
- * behaviour, device pointers, the current CUDA device) and calls no cudaMalloc, cudaFree or other allocating
- * routine.  specsteer_recover_sample needs a context and cannot follow it.
+ * It runs the same two kernels as specsteer_verify_round (same descriptor, same host-side checks, same outputs,
+ * device pointers, the current CUDA device; every recover_mode is accepted, since verification does not depend on
+ * it, and u_recover may be NULL) and calls no cudaMalloc, cudaFree or other allocating routine.
+ * specsteer_recover_sample needs a context and cannot follow it.
  *   - Limits: B <= 1024, B*(K+1) <= 16384, and B*(K+1)*ceil(V/C) <= 229376 with C = 512 for float32 and
  *     1024 for bf16 logits.  Larger shapes return SPECSTEER_ERR_STATIC_LIMIT and launch nothing.
  *   - The first call on each device resolves the array's device address (cudaGetSymbolAddress) and reads

@@ -163,6 +163,28 @@ def alloc_outputs(B: int, K: int, device, pin: bool = False) -> Dict[str, torch.
     return out
 
 
+def _fill_request_arrays(d: RoundDesc, inputs, outputs, B: int, K: int):
+    """The per-request inputs and the outputs of a round descriptor (shared by both kinds of descriptor)."""
+    def ptr(t, dt, n):
+        if t.dtype != dt or not t.is_contiguous() or t.numel() != n:
+            raise ValueError("bad auxiliary tensor: dtype %s, numel %d (want %s, %d)" % (t.dtype, t.numel(), dt, n))
+        return t.data_ptr() if n else None
+
+    d.draft_tokens = ptr(inputs["draft_tokens"], torch.int32, B * K)
+    d.draft_len = ptr(inputs["draft_len"], torch.int32, B)
+    d.lam = ptr(inputs["lam"], torch.float32, B)
+    d.beta = ptr(inputs["beta"], torch.float32, B)
+    d.temperature = ptr(inputs["temperature"], torch.float32, B)
+    d.u_accept = ptr(inputs["u_accept"], torch.float32, B * K)
+    d.u_recover = ptr(inputs["u_recover"], torch.float32, B)
+    for name, (dt, shp) in _OUT_SPECS.items():
+        t = outputs.get(name)
+        n = B
+        for s in shp(K):
+            n *= s
+        setattr(d, name, ptr(t, dt, n) if t is not None else None)
+
+
 def make_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor], *, accept_mode=ACCEPT_RATIO,
               recover_mode=RECOVER_STEER, flags=0, V: Optional[int] = None) -> RoundDesc:
     """Fill a descriptor from tensors.  Logits: [B, K+1, ld_row] (last dim contiguous); pass V if ld_row > V."""
@@ -182,26 +204,7 @@ def make_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.Tensor],
     d.dtype = F32 if hl.dtype == torch.float32 else BF16
     d.accept_mode, d.recover_mode, d.flags = int(accept_mode), int(recover_mode), int(flags)
     d.h_llm, d.h_slm_plus, d.h_slm_minus = hl.data_ptr(), hp.data_ptr(), hm.data_ptr()
-
-    def ptr(t, dt, n):
-        if t.dtype != dt or not t.is_contiguous() or t.numel() != n:
-            raise ValueError("bad auxiliary tensor: dtype %s, numel %d (want %s, %d)" % (t.dtype, t.numel(), dt, n))
-        return t.data_ptr() if n else None
-
-    K = K1 - 1
-    d.draft_tokens = ptr(inputs["draft_tokens"], torch.int32, B * K)
-    d.draft_len = ptr(inputs["draft_len"], torch.int32, B)
-    d.lam = ptr(inputs["lam"], torch.float32, B)
-    d.beta = ptr(inputs["beta"], torch.float32, B)
-    d.temperature = ptr(inputs["temperature"], torch.float32, B)
-    d.u_accept = ptr(inputs["u_accept"], torch.float32, B * K)
-    d.u_recover = ptr(inputs["u_recover"], torch.float32, B)
-    for name, (dt, shp) in _OUT_SPECS.items():
-        t = outputs.get(name)
-        n = B
-        for s in shp(K):
-            n *= s
-        setattr(d, name, ptr(t, dt, n) if t is not None else None)
+    _fill_request_arrays(d, inputs, outputs, B, K1 - 1)
     return d
 
 
@@ -225,25 +228,7 @@ def make_lmhead_desc(inputs: Dict[str, torch.Tensor], outputs: Dict[str, torch.T
     d.B, d.K, d.V = B, K, V
     d.ld_row, d.ld_req, d.dtype = V, K1 * V, F32
     d.accept_mode, d.recover_mode, d.flags = int(accept_mode), int(recover_mode), int(flags)
-
-    def ptr(t, dt, n):
-        if t.dtype != dt or not t.is_contiguous() or t.numel() != n:
-            raise ValueError("bad auxiliary tensor: dtype %s, numel %d (want %s, %d)" % (t.dtype, t.numel(), dt, n))
-        return t.data_ptr() if n else None
-
-    d.draft_tokens = ptr(inputs["draft_tokens"], torch.int32, B * K)
-    d.draft_len = ptr(inputs["draft_len"], torch.int32, B)
-    d.lam = ptr(inputs["lam"], torch.float32, B)
-    d.beta = ptr(inputs["beta"], torch.float32, B)
-    d.temperature = ptr(inputs["temperature"], torch.float32, B)
-    d.u_accept = ptr(inputs["u_accept"], torch.float32, B * K)
-    d.u_recover = ptr(inputs["u_recover"], torch.float32, B)
-    for name, (dt, shp) in _OUT_SPECS.items():
-        t = outputs.get(name)
-        n = B
-        for s in shp(K):
-            n *= s
-        setattr(d, name, ptr(t, dt, n) if t is not None else None)
+    _fill_request_arrays(d, inputs, outputs, B, K)
     ld.x_llm, ld.w_llm = xl.data_ptr(), wl.data_ptr()
     ld.x_slm_plus, ld.w_slm_plus = xp.data_ptr(), wp.data_ptr()
     ld.x_slm_minus, ld.w_slm_minus = xm.data_ptr(), wm.data_ptr()

@@ -48,6 +48,43 @@ struct specsteer_ctx {
 static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
 static_assert(sizeof(specsteer_lmhead_desc) == 288, "the Python mirror of the LM-head descriptor assumes this layout");
 
+namespace specsteer {
+
+specsteer_status check_round_desc(const specsteer_round_desc* d, bool need_u_recover) {
+  if (!d) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->ld_row < d->V || d->ld_req < (int64_t)(d->K + 1) * d->ld_row) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->dtype != SPECSTEER_F32 && d->dtype != SPECSTEER_BF16) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z)
+    return SPECSTEER_ERR_INVALID_ARG;
+  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL &&
+      d->recover_mode != SPECSTEER_RECOVER_ARGMAX)
+    return SPECSTEER_ERR_INVALID_ARG;
+  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->B > 0) {
+    if (!d->h_llm || !d->h_slm_plus || !d->h_slm_minus || !d->draft_len || !d->lambda || !d->beta ||
+        !d->temperature || !d->accept_len)
+      return SPECSTEER_ERR_INVALID_ARG;
+    if (need_u_recover && !d->u_recover) return SPECSTEER_ERR_INVALID_ARG;
+    if (d->K > 0 && (!d->draft_tokens || !d->u_accept)) return SPECSTEER_ERR_INVALID_ARG;
+  }
+  return SPECSTEER_OK;
+}
+
+int sums_wanted(const specsteer_round_desc* d) {
+  return (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
+          d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? SUM_ALL : (SUM_L | SUM_M | SUM_R);
+}
+
+bool rows_aligned(const specsteer_round_desc* d) {
+  const size_t es = d->dtype == SPECSTEER_F32 ? 4 : 2;
+  auto a16 = [](const void* p) { return ((uintptr_t)p & 15u) == 0; };
+  return a16(d->h_llm) && a16(d->h_slm_plus) && a16(d->h_slm_minus) && ((size_t)d->ld_row * es) % 16 == 0 &&
+         ((size_t)d->ld_req * es) % 16 == 0;
+}
+
+}  // namespace specsteer
+
 namespace {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -70,21 +107,8 @@ int n_chunks_of(int V, int tile) { return (V + tile - 1) / tile; }
 
 specsteer_status check_desc(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
   if (!ctx || !d) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->ld_row < d->V || d->ld_req < (int64_t)(d->K + 1) * d->ld_row) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->dtype != SPECSTEER_F32 && d->dtype != SPECSTEER_BF16) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z)
-    return SPECSTEER_ERR_INVALID_ARG;
-  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL &&
-      d->recover_mode != SPECSTEER_RECOVER_ARGMAX)
-    return SPECSTEER_ERR_INVALID_ARG;
-  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->B > 0) {
-    if (!d->h_llm || !d->h_slm_plus || !d->h_slm_minus || !d->draft_len || !d->lambda || !d->beta ||
-        !d->temperature || !d->u_recover || !d->accept_len)
-      return SPECSTEER_ERR_INVALID_ARG;
-    if (d->K > 0 && (!d->draft_tokens || !d->u_accept)) return SPECSTEER_ERR_INVALID_ARG;
-  }
+  specsteer_status st = check_round_desc(d, true);
+  if (st != SPECSTEER_OK) return st;
   if (d->B > ctx->max_B || d->K > ctx->max_K || d->V > ctx->max_V) return SPECSTEER_ERR_UNSUPPORTED;
   // tiles of one launch are indexed with 31 bits
   const size_t slab_b = d->B < kMaxSlabB ? d->B : kMaxSlabB;
@@ -102,8 +126,7 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
   p.B = nb; p.K = K; p.V = d->V;
   p.ld_row = d->ld_row; p.ld_req = d->ld_req;
   p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
-  p.sums = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
-            d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? SUM_ALL : (SUM_L | SUM_M | SUM_R);
+  p.sums = sums_wanted(d);
   p.row_mode = ROWS_ALL;
   p.tile = tile_of(d->dtype);
   p.n_chunks = n_chunks_of(d->V, p.tile);
@@ -125,13 +148,6 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
 #undef OFF
   p.dev_error = ctx->dev_error;
   return p;
-}
-
-bool rows_aligned(const specsteer_round_desc* d) {
-  const size_t es = d->dtype == SPECSTEER_F32 ? 4 : 2;
-  auto a16 = [](const void* p) { return ((uintptr_t)p & 15u) == 0; };
-  return a16(d->h_llm) && a16(d->h_slm_plus) && a16(d->h_slm_minus) && ((size_t)d->ld_row * es) % 16 == 0 &&
-         ((size_t)d->ld_req * es) % 16 == 0;
 }
 
 // Verification needs the normalisers of h_LLM and h_SLM- only (Eq. 7); when nobody asks for a quantity of the

@@ -81,6 +81,18 @@ struct LmheadOperands {
   int d_llm, d_slm;
 };
 
+}  // namespace specsteer
+#include "specsteer.h"
+namespace specsteer {
+
+// Host-side checks of a round descriptor that every entry point shares: sizes, strides, enums, flags and the
+// pointers verification needs.  need_u_recover: the caller will (or may) run a recovery step on this descriptor.
+specsteer_status check_round_desc(const specsteer_round_desc* d, bool need_u_recover);
+// Which normalisers the streaming pass forms for a descriptor (SUM_* bits), from the outputs and modes it asks for.
+int sums_wanted(const specsteer_round_desc* d);
+// Every row of the three logit tensors starts on a 16-byte boundary (the bulk-copy path).
+bool rows_aligned(const specsteer_round_desc* d);
+
 struct LaunchInfo {
   int device;
   int sm_count;

@@ -12,6 +12,8 @@
 //                          128 logits of that chunk on the CUDA cores and samples within it (Eq. 8).
 #include <cuda.h>
 
+#include <atomic>
+
 #include "common.cuh"
 #include "internal.h"
 #include "specsteer.h"
@@ -625,11 +627,11 @@ cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float*
   k.argmax_keys = reinterpret_cast<u64*>(argmax_keys);
   k.shared_head = (op.w_plus == op.w_minus) ? 1 : 0;
   k.vocab_offset = p.vocab_offset;
-  static bool attr_set[64] = {};
-  if (li.device < 64 && !attr_set[li.device]) {
+  static std::atomic<bool> attr_set[64];   // per device; two host threads that both find it clear set the same value
+  if (!attr_set[li.device & 63].load(std::memory_order_acquire)) {
     cudaError_t e = cudaFuncSetAttribute(lmhead_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
-    attr_set[li.device] = true;
+    attr_set[li.device & 63].store(true, std::memory_order_release);
   }
   const int mb = (R + kBM - 1) / kBM, nb = (p.V + kBN - 1) / kBN;
   const long long tiles = (long long)mb * nb;

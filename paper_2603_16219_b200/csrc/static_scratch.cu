@@ -58,26 +58,16 @@ specsteer_status setup_device(int dev, DeviceSetup** out) {
 }  // namespace
 
 extern "C" specsteer_status specsteer_verify_round_static(const specsteer_round_desc* d, void* cuda_stream) {
-  if (!d) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->ld_row < d->V || d->ld_req < (int64_t)(d->K + 1) * d->ld_row) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->dtype != SPECSTEER_F32 && d->dtype != SPECSTEER_BF16) return SPECSTEER_ERR_INVALID_ARG;
-  if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z)
-    return SPECSTEER_ERR_INVALID_ARG;
-  if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL)
-    return SPECSTEER_ERR_INVALID_ARG;
-  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
+  // the same host-side checks as specsteer_verify_round (every recovery mode is accepted: verification does not
+  // depend on it; u_recover is not needed here)
+  specsteer_status chk = check_round_desc(d, false);
+  if (chk != SPECSTEER_OK) return chk;
   const int tile = d->dtype == SPECSTEER_F32 ? kChunkF32 : kChunkBF16;
   const int n_chunks = (d->V + tile - 1) / tile;
   const long long rows = (long long)d->B * (d->K + 1);
   if (d->B > kStaticMaxB || rows > kStaticMaxRows || rows * n_chunks > kStaticMaxRecords)
     return SPECSTEER_ERR_STATIC_LIMIT;
   if (d->B == 0) return SPECSTEER_OK;
-  if (!d->h_llm || !d->h_slm_plus || !d->h_slm_minus || !d->draft_len || !d->lambda || !d->beta ||
-      !d->temperature || !d->accept_len)
-    return SPECSTEER_ERR_INVALID_ARG;
-  if (d->K > 0 && (!d->draft_tokens || !d->u_accept)) return SPECSTEER_ERR_INVALID_ARG;
-
 
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess) return SPECSTEER_ERR_CUDA;
@@ -89,8 +79,7 @@ extern "C" specsteer_status specsteer_verify_round_static(const specsteer_round_
   p.B = d->B; p.K = d->K; p.V = d->V;
   p.ld_row = d->ld_row; p.ld_req = d->ld_req;
   p.accept_mode = d->accept_mode; p.recover_mode = d->recover_mode; p.flags = d->flags;
-  p.sums = (d->logp_plus || d->log_z || d->accept_mode == SPECSTEER_ACCEPT_EXACT_Z ||
-            d->recover_mode == SPECSTEER_RECOVER_RESIDUAL) ? SUM_ALL : (SUM_L | SUM_M | SUM_R);
+  p.sums = sums_wanted(d);
   p.row_mode = ROWS_ALL;
   p.tile = tile; p.n_chunks = n_chunks;
   p.h_llm = d->h_llm; p.h_plus = d->h_slm_plus; p.h_minus = d->h_slm_minus;
@@ -108,10 +97,7 @@ extern "C" specsteer_status specsteer_verify_round_static(const specsteer_round_
   p.status_ws = reinterpret_cast<int*>(su->base + kPartBytes + kLseBytes);
   p.dev_error = reinterpret_cast<int*>(su->base + kPartBytes + kLseBytes + kStatusBytes);
 
-  const size_t es = d->dtype == SPECSTEER_F32 ? 4 : 2;
-  auto a16 = [](const void* q) { return ((uintptr_t)q & 15u) == 0; };
-  const bool aligned = a16(d->h_llm) && a16(d->h_slm_plus) && a16(d->h_slm_minus) &&
-                       ((size_t)d->ld_row * es) % 16 == 0 && ((size_t)d->ld_req * es) % 16 == 0;
+  const bool aligned = rows_aligned(d);
   int nl = 0;
   if (launch_verify(p, d->dtype, aligned, su->li, (cudaStream_t)cuda_stream, &nl) != cudaSuccess) {
     cudaGetLastError();

@@ -11,6 +11,8 @@
 // log-probabilities and alpha; the accept flags are then scanned for accept_len
 // (Algorithm 1 Phase 2; Eq. 6 / Eq. 7).  With a sharded vocabulary the rows come from the shards' gathered
 // partials instead of the records.
+#include <atomic>
+
 #include "common.cuh"
 #include "internal.h"
 #include "records.cuh"
@@ -18,17 +20,6 @@
 
 namespace specsteer {
 
-// How many of the four pairs per batch of the h_SLM- stream take the FMA-pipe polynomial instead of ex2.approx
-// for 16-bit logits (all outputs / without the h_SLM+ normaliser).  0: measured no faster at any setting,
-// because the polynomial costs as many issue slots as it frees on the special-function unit.
-#ifndef SPECSTEER_POLY_PAIRS_BF16
-#define SPECSTEER_POLY_PAIRS_BF16 0
-#endif
-constexpr int kPolyPairsBF16 = SPECSTEER_POLY_PAIRS_BF16;
-#ifndef SPECSTEER_POLY_PAIRS_BF16_LEAN
-#define SPECSTEER_POLY_PAIRS_BF16_LEAN 0
-#endif
-constexpr int kPolyPairsBF16Lean = SPECSTEER_POLY_PAIRS_BF16_LEAN;
 constexpr float kSlack = 16.f;  // careful path: the reference exponent may lag the running maximum by this much
 
 struct TileMeta {
@@ -115,44 +106,13 @@ __device__ __forceinline__ float max8(const f32x2 (&v)[4]) {
   return fmaxf(max3(max3(x[0], x[1], x[2]), max3(x[3], x[4], x[5]), x[6]), x[7]);
 }
 
-// 2^a for a pair of arguments a < 127.5 on the FMA pipe (no special-function unit): a is clamped to
-// >= -126, split into round(a) + f with f in [-0.5, 0.5] by the 1.5*2^23 trick, 2^f is a degree-5
-// polynomial (relative error 2.1e-7 in float32 Horner form), and round(a) is added to the exponent field.
-__device__ __forceinline__ f32x2 exp2_poly2(f32x2 a) {
-  const float kMagic = 12582912.f;  // 1.5 * 2^23
-  float a0, a1;
-  unpack2(a, a0, a1);
-  const f32x2 ac = pack2(fmaxf(a0, -126.f), fmaxf(a1, -126.f));
-  const f32x2 magic2 = pack2(kMagic, kMagic);
-  const f32x2 t = add2(ac, magic2);
-  const f32x2 f = sub2(ac, sub2(t, magic2));
-  f32x2 q = pack2(0.001327645150013268f, 0.001327645150013268f);
-  q = fma2(q, f, pack2(0.009675540030002594f, 0.009675540030002594f));
-  q = fma2(q, f, pack2(0.05550713464617729f, 0.05550713464617729f));
-  q = fma2(q, f, pack2(0.24022120237350464f, 0.24022120237350464f));
-  q = fma2(q, f, pack2(0.6931469440460205f, 0.6931469440460205f));
-  q = fma2(q, f, pack2(1.0000001192092896f, 1.0000001192092896f));
-  float q0, q1, t0, t1;
-  unpack2(q, q0, q1);
-  unpack2(t, t0, t1);
-  return pack2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(t0) << 23)),
-               __uint_as_float(__float_as_uint(q1) + (__float_as_uint(t1) << 23)));
-}
-
-// sum += 2^(x*c - ref) over eight entries of one stream; the first POLY_N of the four pairs take the
-// FMA-pipe polynomial, the others ex2.approx
-template <int POLY_N>
+// sum += 2^(x*c - ref) over eight entries of one stream
 __device__ __forceinline__ void exp_sum8(f32x2& s2, const f32x2 (&x)[4], f32x2 c2, f32x2 nref2) {
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
-    const f32x2 arg = fma2(x[i], c2, nref2);
-    if (i < POLY_N) {
-      s2 = add2(s2, exp2_poly2(arg));
-    } else {
-      float a0, a1;
-      unpack2(arg, a0, a1);
-      s2 = add2(s2, pack2(ex2(a0), ex2(a1)));
-    }
+    float a0, a1;
+    unpack2(fma2(x[i], c2, nref2), a0, a1);
+    s2 = add2(s2, pack2(ex2(a0), ex2(a1)));
   }
 }
 
@@ -185,10 +145,10 @@ __device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32
     const bool upd = (bm[0] > a.thr[0]) | (bm[1] > a.thr[1]) | (bm[2] > a.thr[2]) | (bm[3] > a.thr[3]);
     if (__any_sync(kFullMask, upd)) acc_raise(a, bm, c, inv_c, lane);
   }
-  if (SUMS & SUM_L) exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-  if (SUMS & SUM_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-  if (SUMS & SUM_M) exp_sum8<0>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-  if (SUMS & SUM_R) exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+  if (SUMS & SUM_L) exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+  if (SUMS & SUM_P) exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+  if (SUMS & SUM_M) exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+  if (SUMS & SUM_R) exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
 }
 
 // ---- one chunk (half a tile) from shared memory, one warp ---------------------------------------
@@ -250,16 +210,14 @@ __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, con
 // The fast variant for a full chunk.  Only the first batch computes maxima: the references are set kBias
 // binades above them, so that later entries may exceed the first batch's maximum by 2^(kBias + 120)
 // before a sum overflows, while entries down to 2^-(126 - kBias) of it still count.  Nothing is tested
-// inside the chunk; at its end a sum that is not below 2^120 (or is NaN), or a polynomial argument
-// that left the polynomial's range, makes the warp return false and the caller redoes the chunk with
-// chunk_pass, which tests every batch.
+// inside the chunk; at its end a sum that is not below 2^120 (or is NaN) makes the warp return false and
+// the caller redoes the chunk with chunk_pass, which tests every batch.
 constexpr float kBias = 60.f;
 
-template <typename T, int CHUNK, int POLY_N, int SUMS>
+template <typename T, int CHUNK, int SUMS>
 __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, const T* sm, int lane, float beta,
                                            float c, float inv_c) {
   const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
-  float run_m = kNegInf;  // running maximum of the stream that takes the polynomial
   constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;   // the h_SLM+ slot is filled and read
   {
     f32x2 l[4], p[4], m[4], r[4];
@@ -273,11 +231,10 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     const float bm[4] = {(SUMS & SUM_L) ? max8(l) : kNegInf, (SUMS & SUM_P) ? max8(p) : kNegInf,
                          (SUMS & SUM_M) ? max8(m) : kNegInf, (SUMS & SUM_R) ? max8(r) : kNegInf};
     acc_start(a, bm, c, inv_c, lane, kBias);
-    run_m = bm[Q_M];
-    if (SUMS & SUM_L) exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    if (SUMS & SUM_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-    if (SUMS & SUM_M) exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-    if (SUMS & SUM_R) exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+    if (SUMS & SUM_L) exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+    if (SUMS & SUM_P) exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (SUMS & SUM_M) exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+    if (SUMS & SUM_R) exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
 #pragma unroll 1
   for (int it = 1; it < CHUNK / 256; ++it) {
@@ -289,11 +246,10 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
 #pragma unroll
       for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
     }
-    if (POLY_N > 0 && (SUMS & SUM_M)) run_m = fmaxf(run_m, max8(m));
-    if (SUMS & SUM_L) exp_sum8<0>(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    if (SUMS & SUM_P) exp_sum8<0>(a.s2[Q_P], p, c2, a.nref2[Q_P]);
-    if (SUMS & SUM_M) exp_sum8<POLY_N>(a.s2[Q_M], m, c2, a.nref2[Q_M]);
-    if (SUMS & SUM_R) exp_sum8<0>(a.s2[Q_R], r, c2, a.nref2[Q_R]);
+    if (SUMS & SUM_L) exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
+    if (SUMS & SUM_P) exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (SUMS & SUM_M) exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
+    if (SUMS & SUM_R) exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
   const float kBig = 1.329227995784916e36f;  // 2^120
   bool bad = false;
@@ -302,11 +258,6 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     float s0, s1;
     unpack2(a.s2[q], s0, s1);
     bad |= !(s0 + s1 < kBig);
-  }
-  if (POLY_N > 0 && (SUMS & SUM_M)) {
-    float n0, n1;
-    unpack2(a.nref2[Q_M], n0, n1);
-    bad |= !(fmaf(run_m, c, n0) < 120.f);
   }
   return !__any_sync(kFullMask, bad);
 }
@@ -367,8 +318,10 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
     if (p.n_shards == 0 && !p.tok_logits && y >= 0 && y < p.V) {
       const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
       gl = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
-      gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
       gm = load_logit<T>(reinterpret_cast<const T*>(p.h_minus), off);
+      // Eq. 7 needs nothing of h_SLM+: when verification forms neither its normaliser nor the one of h_rec (the
+      // two-phase round), that tensor is not touched on a drafted row at all
+      if (p.sums & (SUM_P | SUM_R)) gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
     }
   }
   pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
@@ -534,9 +487,6 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
   constexpr int TILE = 2 * CHUNK;
-  // 16-bit logits carry half the bytes per power of two, so there the special-function unit binds before
-  // HBM does: the h_SLM- stream takes the FMA-pipe polynomial for POLY_N of its four pairs per batch
-  constexpr int POLY_N = sizeof(T) == 2 ? ((SUMS & SUM_P) ? kPolyPairsBF16 : kPolyPairsBF16Lean) : 0;
   constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;  // h_SLM+ is read at all
   constexpr int NPAIR = NCW / 2;
   static_assert(NCW % 2 == 0 && STAGES % NPAIR == 0, "each stage belongs to one fixed pair of consumer warps");
@@ -709,7 +659,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       const T* sl = tiles + (size_t)stage * NSLOT * TILE + half * CHUNK;
       Acc a;
       if (nv >= CHUNK) {
-        if (!chunk_fast<T, CHUNK, POLY_N, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, mt.beta, mt.c, mt.inv_c))
+        if (!chunk_fast<T, CHUNK, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, mt.beta, mt.c, mt.inv_c))
           chunk_pass<T, CHUNK, false, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
       } else if (nv > 0) chunk_pass<T, CHUNK, true, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
@@ -752,13 +702,15 @@ static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cud
                        STAGES * sizeof(TileMeta) + 16;
   const size_t smem = fixed + (size_t)(5 * p.B + 1) * sizeof(int);
   auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS>;
-  static bool attr_set_dev[64] = {};  // per instantiation and device; sized for the largest slab
-  bool& attr_set = attr_set_dev[li.device & 63];
-  if (!attr_set) {
+  // per instantiation and device; sized for the largest slab.  Contexts may be driven from different host threads:
+  // the flag is atomic, and two threads that both find it clear merely set the same attribute twice.
+  static std::atomic<bool> attr_set_dev[64];
+  std::atomic<bool>& attr_set = attr_set_dev[li.device & 63];
+  if (!attr_set.load(std::memory_order_acquire)) {
     const size_t smem_max = fixed + (size_t)(5 * kMaxSlabB + 1) * sizeof(int);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
-    attr_set = true;
+    attr_set.store(true, std::memory_order_release);
   }
   kern<<<li.sm_count, (NCW + NPW) * 32, smem, s>>>(p);
   return cudaGetLastError();

@@ -17,15 +17,25 @@ VERIFY_OUTPUTS = ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus
                   "log_z", "req_status")
 
 
-def _both(binding, synth, ctx, spec, seed, accept_mode):
+def _both(binding, synth, ctx, spec, seed, accept_mode, recover_mode=0):
     inputs = synth.make_round(spec, device="cuda", seed=seed)
     ref = binding.alloc_outputs(spec.B, spec.K, "cuda")
     got = binding.alloc_outputs(spec.B, spec.K, "cuda")
     for t in got.values():                      # poison: the call must write every verify output itself
         t.view(torch.uint8).fill_(0xA5)
-    ctx.verify_round(binding.make_desc(inputs, ref, accept_mode=accept_mode, flags=binding.FLAG_BONUS))
-    binding.verify_round_static(binding.make_desc(inputs, got, accept_mode=accept_mode, flags=binding.FLAG_BONUS))
+    ctx.verify_round(binding.make_desc(inputs, ref, accept_mode=accept_mode, recover_mode=recover_mode,
+                                       flags=binding.FLAG_BONUS))
+    desc = binding.make_desc(inputs, got, accept_mode=accept_mode, recover_mode=recover_mode, flags=binding.FLAG_BONUS)
+    binding.verify_round_static(desc)           # warm-up: the first call on a device resolves the scratch array's
+    torch.cuda.synchronize()                    # address, and the first launch of a kernel loads its code
+    for t in got.values():
+        t.view(torch.uint8).fill_(0xA5)
     torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]  # the driver's own count of free device memory
+    binding.verify_round_static(desc)
+    torch.cuda.synchronize()
+    # the property the entry point exists for: the call took no device memory
+    assert torch.cuda.mem_get_info()[0] == free_before, spec.name
     for k in VERIFY_OUTPUTS:
         a, b = ref[k].cpu().numpy(), got[k].cpu().numpy()
         assert np.array_equal(a, b, equal_nan=True), (spec.name, k)
@@ -44,6 +54,9 @@ def test_static_entry_point_matches_context_entry_point_on_consecutive_calls():
     out_big = _both(binding, synth, ctx, big, 1, binding.ACCEPT_RATIO)
     _both(binding, synth, ctx, small, 2, binding.ACCEPT_EXACT_Z)
     _both(binding, synth, ctx, big, 3, binding.ACCEPT_EXACT_Z)
+    # a greedy-decoding descriptor (the paper's experimental setting) is served like any other: verification does
+    # not depend on the recovery mode
+    _both(binding, synth, ctx, small, 4, binding.ACCEPT_RATIO, recover_mode=binding.RECOVER_ARGMAX)
     assert int(out_big["accept_len"].sum()) > 0
     ctx.close()
 
