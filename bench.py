@@ -26,13 +26,11 @@ METRIC = "verified_draft_positions_per_sec"
 UNIT = "positions/s"
 FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1400.0   # sustained, under the power cap
-N_SM = 148
-EX2_PER_CLK_PER_SM = 16
 NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per used row of the streaming kernel, from the ncu captures summarised under
-# profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows), keyed by
-# configuration.  Absent = not captured for the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_ROW = {3: 1858819, 4: 1558613}
+# profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows, so the figure for a
+# full launch is an extrapolation), keyed by configuration.  Absent = not captured for the kernel as it stands.
+NCU_TRAFFIC_BYTES_PER_ROW = {}
 
 
 def _peaks():
@@ -130,17 +128,17 @@ def run_reference(args, rank, world):
     spec = synth.CONFIGS[args.config]
     cores = oracle.max_threads()
     # inputs for the sample only: generate a reduced batch of the same recipe on the CPU
-    probe_B = min(spec.B, 8)
+    probe_B = min(spec.B, max(8, cores))        # at least one request per host thread
     small = synth.RoundSpec(spec.name + "_sample", probe_B, spec.K, spec.V, spec.dtype, sigma_plus=spec.sigma_plus,
                             heavy_tail=spec.heavy_tail, ragged=spec.ragged, beta_choices=spec.beta_choices,
                             beta_uniform=spec.beta_uniform, temp_choices=spec.temp_choices, lam=spec.lam)
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     inputs = synth.make_round(small, device=dev, seed=0)
     flags = oracle.FLAG_BONUS
-    dt, _, _ = _oracle_time(oracle, synth, inputs, list(range(min(2, probe_B))), flags, cores)
-    per_req = dt / min(2, probe_B)
+    dt, _, _ = _oracle_time(oracle, synth, inputs, list(range(probe_B)), flags, cores)
+    per_req = dt / probe_B                        # wall time per request with every thread busy
     budget = 120.0 / max(1, args.steps + args.warmup)
-    n_req = int(max(1, min(probe_B, budget / max(per_req, 1e-6))))
+    n_req = int(max(min(probe_B, cores), min(probe_B, budget / max(per_req, 1e-6))))
     ends = [i // 2 if i % 2 == 0 else probe_B - 1 - i // 2 for i in range(probe_B)]   # alternate both regimes
     sel = sorted(ends[:n_req])
     for _ in range(args.warmup):
@@ -165,6 +163,169 @@ def run_reference(args, rank, world):
     print(json.dumps(line), flush=True)
 
 
+def _time_rounds(torch, ctx, descs, stream, steps, barrier, n_pairs=16):
+    """Times `steps` whole rounds (verify + recover) cycling over `descs`; on `n_pairs` of them the library also
+    records an event pair around the streaming kernel.  Returns (ms per step, streaming-kernel ms, wall window)."""
+    n_pairs = max(1, min(steps, n_pairs))
+    stride = max(1, steps // n_pairs)
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_pairs)]
+    for a, b in evs:
+        a.record(stream)
+        b.record(stream)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for i in range(3):
+        ctx.verify_round(descs[i % len(descs)], stream)
+        ctx.recover_sample(descs[i % len(descs)], stream)
+    barrier()
+    w0 = time.perf_counter()
+    e0.record(stream)
+    used = 0
+    for i in range(steps):
+        d = descs[i % len(descs)]
+        hook = i % stride == 0 and used < n_pairs
+        if hook:
+            ctx.time_streaming(*evs[used])
+        ctx.verify_round(d, stream)
+        ctx.recover_sample(d, stream)
+        if hook:
+            ctx.time_streaming(None, None)
+            used += 1
+    e1.record(stream)
+    barrier()
+    w1 = time.perf_counter()
+    kernel_ms = sum(a.elapsed_time(b) for a, b in evs[:used]) / used
+    return e0.elapsed_time(e1) / steps, kernel_ms, (w0, w1)
+
+
+def _ex2_rate(torch, binding, dev, stream, sampler):
+    """Measured ex2.approx throughput of this GPU: a few milliseconds of the library's probe kernel, CUDA events.
+    Returns (evaluations per second, wall window) - the window lets the clock sampler say at which SM clock."""
+    n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+    n_ctas, iters = 2 * n_sm, 4096
+    sink = torch.empty(n_ctas * 1024, dtype=torch.float32, device=dev)
+    binding.probe_ex2(n_ctas, 64, sink, stream)          # warm-up (loads the kernel)
+    torch.cuda.synchronize(dev)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0 = time.perf_counter()
+    a.record(stream)
+    n = 0
+    for _ in range(4):
+        n += binding.probe_ex2(n_ctas, iters, sink, stream)
+    b.record(stream)
+    torch.cuda.synchronize(dev)
+    w1 = time.perf_counter()
+    return n / (a.elapsed_time(b) * 1e-3), (w0, w1), n_sm
+
+
+def _largest_config(torch, binding, synth, dev, local_rank, stream, barrier, sampler, peak, steps):
+    """Config 4 (B=512, K=6, V=256000, bf16; 5.5 GB of logits): the round with every output, and the round asked for
+    Algorithm 1's outputs only (two-phase), each with the streaming launch timed by the library's event pair."""
+    spec = synth.CONFIGS[4]
+    inputs = synth.make_round(spec, device=dev, seed=0)
+    rows = synth.used_rows(spec, inputs["draft_len"], bonus=True)
+    positions = int(inputs["draft_len"].sum().item())
+    ctx = binding.Context(spec.B, spec.K, spec.V, device=local_rank)
+    flags = binding.FLAG_BONUS
+    outs = binding.alloc_outputs(spec.B, spec.K, dev)
+    lean_outs = {k: v for k, v in outs.items() if k not in ("logp_plus", "logp_star", "log_z")}
+    block = {"workload": spec.name, "dtype": "bf16", "B": spec.B, "K": spec.K, "V": spec.V,
+             "positions_per_step": positions, "l2": "inputs exceed L2"}
+    wins = []
+    # every output: three tensors, every used row, four normalisers
+    ms, kms, win = _time_rounds(torch, ctx, [binding.make_desc(inputs, outs, flags=flags)], stream, steps, barrier)
+    wins.append(win)
+    nbytes = spec.logit_bytes(rows)
+    ach = nbytes / (kms * 1e-3) / 1e9
+    block["all_outputs"] = {
+        "kernel": "verify_kernel", "kernel_ms": kms, "algorithmic_bytes_per_launch": nbytes, "achieved": ach, "unit": "GB/s",
+        "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "ms_per_step": ms,
+        "whole_step_gbs": nbytes / (ms * 1e-3) / 1e9, "whole_step_frac_of_nominal_8TBs": nbytes / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "positions_per_s": positions / (ms * 1e-3), "steps": steps}
+    acc_all = outs["accept_len"].clone()
+    # Algorithm 1's outputs only: verification streams h_LLM and h_SLM- over the drafted rows (Eq. 7), recovery then
+    # streams row accept_len of every request that takes a token, all three tensors (Eq. 8)
+    ms, kms, win = _time_rounds(torch, ctx, [binding.make_desc(inputs, lean_outs, flags=flags)], stream, steps, barrier)
+    wins.append(win)
+    vbytes = 2 * positions * spec.V * spec.elem_bytes
+    sampling = int((lean_outs["rec_token"] >= 0).sum().item())
+    rbytes = 3 * sampling * spec.V * spec.elem_bytes
+    ach = vbytes / (kms * 1e-3) / 1e9
+    block["algorithm1_only"] = {
+        "kernel": "verify_kernel (two tensors, drafted rows)", "kernel_ms": kms, "algorithmic_bytes_per_launch": vbytes,
+        "achieved": ach, "unit": "GB/s", "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
+        "ms_per_step": ms, "algorithmic_bytes_per_step": vbytes + rbytes,
+        "whole_step_gbs": (vbytes + rbytes) / (ms * 1e-3) / 1e9,
+        "whole_step_frac_of_nominal_8TBs": (vbytes + rbytes) / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "positions_per_s": positions / (ms * 1e-3), "steps": steps,
+        "same_accept_len_as_all_outputs": bool(torch.equal(lean_outs["accept_len"], acc_all))}
+    assert ctx.device_error() == 0
+    ctx.close()
+    del inputs
+    torch.cuda.empty_cache()
+    return block, wins
+
+
+def _vocab_sharded(torch, dist, binding, synth, sharding, dev, local_rank, rank, world, stream, barrier, steps):
+    """Config 3 with the vocabulary split over the ranks (a tensor-parallel LM head's layout): the round with one
+    all-gather of 64 bytes per row and rank and one MAX all-reduce of the per-request results (NCCL), and the same
+    with the three LM heads fused in front, their rows split over the ranks.  One batch for the whole job."""
+    spec = synth.CONFIGS[3]
+    out = {"workload": spec.name, "ranks": world, "collectives": "all_gather(64 B x rows x ranks) + all_reduce(MAX) of 4 small arrays (NCCL)"}
+    full = synth.make_round(spec, device=dev, seed=0)              # the same batch on every rank
+    positions = int(full["draft_len"].sum().item())
+    lo, hi = sharding.vocab_range(spec.V, rank, world, align=4)
+    local = dict(full)
+    for k in ("h_llm", "h_slm_plus", "h_slm_minus"):
+        local[k] = full[k][:, :, lo:hi].contiguous()
+    del full
+    torch.cuda.empty_cache()
+    ctx = binding.Context(spec.B, spec.K, max(hi - lo, 1), device=local_rank)
+    outs = binding.alloc_outputs(spec.B, spec.K, dev)
+    desc = binding.make_desc(local, outs, flags=binding.FLAG_BONUS)
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(n):
+            fn()
+        b.record(stream)
+        barrier()
+        t = torch.tensor([a.elapsed_time(b) / n], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    ms = timed(lambda: sharding.sharded_vocab_round(ctx, desc, outs, lo, spec.V, dist, stream), steps)
+    out["logits_split"] = {"ms_per_step": ms, "positions_per_s": positions / (ms * 1e-3), "steps": steps,
+                           "logit_bytes_per_rank": 3 * spec.rows * (hi - lo) * spec.elem_bytes,
+                           "bytes_exchanged_per_rank": spec.rows * 64 * world + spec.B * (4 + 4 + 4 * (spec.K + 1) + 4)}
+    assert ctx.device_error() == 0
+    ctx.close()
+    del local
+    torch.cuda.empty_cache()
+    # the fused form: hidden states replicated, the heads' rows split
+    dL, dS = 5120, 2048
+    lm = synth.make_lmhead_round(spec, dL, dS, device=dev, seed=0)
+    lo, hi = sharding.vocab_range(spec.V, rank, world, align=8)
+    lml = dict(lm)
+    for k in ("w_llm", "w_slm_plus", "w_slm_minus"):
+        lml[k] = lm[k][lo:hi].contiguous()
+    del lm
+    torch.cuda.empty_cache()
+    ctx = binding.Context(spec.B, spec.K, max(hi - lo, 1), device=local_rank)
+    ldesc = binding.make_lmhead_desc(lml, outs, flags=binding.FLAG_BONUS)
+    steps_lm = max(3, min(steps, 30))
+    ms = timed(lambda: sharding.sharded_lmhead_round(ctx, ldesc, outs, lo, spec.V, dist, stream), steps_lm)
+    out["heads_split"] = {"ms_per_step": ms, "positions_per_s": positions / (ms * 1e-3), "steps": steps_lm,
+                          "d_llm": dL, "d_slm": dS, "flops_per_rank": 2.0 * spec.rows * (hi - lo) * (dL + 2 * dS),
+                          "tflops_per_rank": 2.0 * spec.rows * (hi - lo) * (dL + 2 * dS) / (ms * 1e-3) / 1e12}
+    assert ctx.device_error() == 0
+    ctx.close()
+    return out
+
+
 def run_cuda(args, rank, world, local_rank):
     import torch
     from paper_2603_16219_b200 import binding, build, synth
@@ -174,7 +335,7 @@ def run_cuda(args, rank, world, local_rank):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
     dist = None
-    if world > 1:
+    if world > 1 or (args.vocab_sharded and "RANK" in os.environ):
         import torch.distributed as dist
         dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
 
@@ -421,6 +582,29 @@ def run_cuda(args, rank, world, local_rank):
                     "h2d_bytes_per_step": rows_copied * spec.V * spec.elem_bytes + h2d - 3 * spec.rows * spec.V * spec.elem_bytes,
                     "same_accept_len_and_tokens": bool(torch.equal(lean_host_out["accept_len"], host_out["accept_len"]) and
                                                        torch.equal(lean_host_out["rec_token"], host_out["rec_token"]))}
+    peak, peak_kind = _peaks()
+    # ---- the largest configuration beside the headline (1 GPU runs of the default workload)
+    largest = None
+    if world == 1 and args.config == 3 and not args.requests and not args.lean and not args.no_extras:
+        largest, wins = _largest_config(torch, binding, synth, dev, local_rank, stream, barrier, sampler, peak,
+                                        max(10, min(args.steps, 100)))
+        n0 = len(sampler.windows)
+        for w in wins:
+            sampler.window(*w)
+        only = ClockSampler.__new__(ClockSampler)      # the clocks of those two timed regions alone
+        only.samples, only.windows, only.max_mhz = sampler.samples, sampler.windows[n0:], sampler.max_mhz
+        largest["clocks"] = only.summary()
+    # ---- the measured special-function rate (the second ceiling of the streaming kernel)
+    ex2_per_s, ex2_win, n_sm = _ex2_rate(torch, binding, dev, stream, sampler)
+    probe_clk = ClockSampler.__new__(ClockSampler)
+    probe_clk.samples, probe_clk.windows, probe_clk.max_mhz = sampler.samples, [ex2_win], sampler.max_mhz
+    probe_clk = probe_clk.summary()
+    # ---- several GPUs: the same configuration with the vocabulary split over the ranks
+    sharded = None
+    if dist is not None and (world > 1 or args.vocab_sharded) and args.config == 3 and not args.requests and not args.no_extras:
+        from paper_2603_16219_b200 import sharding
+        sharded = _vocab_sharded(torch, dist, binding, synth, sharding, dev, local_rank, rank, world, stream, barrier,
+                                 max(10, min(args.steps, 100)))
     sampler.stop()
 
     if rank != 0:
@@ -429,25 +613,31 @@ def run_cuda(args, rank, world, local_rank):
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = _peaks()
     achieved = logit_bytes / (kernel_ms * 1e-3) / 1e9
     roofline = {
         "bound": "hbm", "kernel": "verify_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-        "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.config] * rows if args.config in NCU_TRAFFIC_BYTES_PER_ROW
+        "frac": achieved / peak,
+        "peak_source": "of " + peak_kind + " (a read+write copy: a read-only kernel can exceed it)",
+        "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.config] * rows if args.config in NCU_TRAFFIC_BYTES_PER_ROW
                     and not args.requests else None),
+        "traffic_source": ("extrapolated: ncu dram bytes per row on a 32-request capture x rows of this launch"
+                           if args.config in NCU_TRAFFIC_BYTES_PER_ROW and not args.requests else None),
         "algorithmic_bytes_per_launch": logit_bytes, "kernel_ms": kernel_ms,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "whole_step_gbs": logit_bytes / (ms_per_step * 1e-3) / 1e9,
+        "whole_step_frac": logit_bytes / (ms_per_step * 1e-3) / 1e9 / peak,
+        "whole_step_frac_of_nominal_8TBs": logit_bytes / (ms_per_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
     }
-    # The second ceiling of the streaming kernel: one ex2 per normaliser and vocabulary entry on the
-    # special-function unit (16 results per clock and SM: 4 per sub-partition), at the clock sampled under load.
+    # The second ceiling of the streaming kernel: one ex2.approx per normaliser and vocabulary entry on the
+    # special-function unit, against the rate the probe kernel reached on this GPU a moment ago.
     clk = sampler.summary()
-    if not args.lean and clk.get("sm_mhz"):
+    if not args.lean:
         n_ex2 = 4.0 * rows * spec.V
-        sfu_peak = N_SM * EX2_PER_CLK_PER_SM * clk["sm_mhz"] * 1e6
-        roofline["sfu"] = {"ex2_per_launch": n_ex2, "achieved": n_ex2 / (kernel_ms * 1e-3), "peak": sfu_peak,
-                           "unit": "ex2/s", "frac": n_ex2 / (kernel_ms * 1e-3) / sfu_peak,
-                           "peak_source": "derived: 16 ex2 per clock per SM x 148 SMs x median SM clock under load"}
+        roofline["sfu"] = {"ex2_per_launch": n_ex2, "achieved": n_ex2 / (kernel_ms * 1e-3), "peak": ex2_per_s,
+                           "unit": "ex2/s", "frac": n_ex2 / (kernel_ms * 1e-3) / ex2_per_s,
+                           "peak_source": "measured: specsteer_probe_ex2, CUDA events",
+                           "peak_per_clk_per_sm": (ex2_per_s / (probe_clk["sm_mhz"] * 1e6) / n_sm) if probe_clk.get("sm_mhz") else None,
+                           "probe_sm_mhz": probe_clk.get("sm_mhz")}
     cpu = None
     if world == 1:
         import oracle
@@ -470,7 +660,7 @@ def run_cuda(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(3, args.warmup),
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": spec.dtype, "data": "synthetic",
         "config": {"workload": spec.name, "B": spec.B, "K": spec.K, "V": spec.V, "logit_dtype": spec.dtype,
                    "requests_per_gpu": spec.B, "rows_read_per_gpu": rows, "positions_per_step_per_gpu": positions,
                    "accept_mode": "ratio", "recover_mode": "steer", "bonus_row": True, "lambda": spec.lam,
@@ -485,6 +675,8 @@ def run_cuda(args, rank, world, local_rank):
                 "ms_per_step": 1e3 * e2e_s, "steps": e2e_steps, "api": "specsteer_round_host (pinned host buffers)",
                 "algorithm1_outputs_only": e2e_alg1},
         "algorithm1_outputs_only": alg1,
+        "largest_config": largest,
+        "vocab_sharded": sharded,
         "gpu_launches": int(gpu_launches),
         "clocks": sampler.summary(),
     }
@@ -624,6 +816,10 @@ def main():
                     help="with --kernels-only: also time the top-k split recovery (cloud + edge kernels) with this k")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the device-resident steps and print a short line (profiling aid)")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the blocks beside the headline (the largest configuration; the vocabulary-sharded rounds)")
+    ap.add_argument("--vocab-sharded", action="store_true",
+                    help="under torchrun with one rank: still time the vocabulary-sharded rounds (a check of that leg)")
     ap.add_argument("--greedy", action="store_true",
                     help="with --kernels-only: greedy recovery (the token of largest h_rec) instead of sampling")
     ap.add_argument("--lmhead", action="store_true",

@@ -322,6 +322,13 @@ specsteer_status specsteer_ctx_device_error(specsteer_ctx *ctx);
  * switch the hook off.  Errors: INVALID_ARG (NULL ctx, or only one event given). */
 specsteer_status specsteer_ctx_time_streaming(specsteer_ctx *ctx, void *ev_begin, void *ev_end);
 
+/* Measurement aid (the paper has no counterpart): launches n_ctas CTAs of 1024 threads on the current device, each
+ * thread evaluating 8 * iters ex2.approx (the special-function instruction every normaliser of the streaming kernel
+ * costs once per vocabulary entry), so that a benchmark can time it with its own events and state a measured
+ * special-function rate instead of an assumed one.  sink: DEVICE, n_ctas * 1024 floats, overwritten.
+ * Total evaluations: n_ctas * 1024 * 8 * iters.  Errors: INVALID_ARG, CUDA. */
+specsteer_status specsteer_probe_ex2(int32_t n_ctas, int32_t iters, float *sink, void *cuda_stream);
+
 /* Bytes of device workspace owned by the context. */
 size_t specsteer_ctx_workspace_bytes(const specsteer_ctx *ctx);
 

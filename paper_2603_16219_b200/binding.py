@@ -33,6 +33,7 @@ EXPORTS = (
     "specsteer_lmhead_round",
     "specsteer_lmhead_shard_local", "specsteer_lmhead_shard_combine", "specsteer_lmhead_shard_recover",
     "specsteer_shard_greedy_local", "specsteer_lmhead_shard_greedy_local", "specsteer_shard_greedy_finish",
+    "specsteer_probe_ex2",
 )
 SHARD_PARTIAL_BYTES = 64
 MAX_SHARDS = 32
@@ -119,6 +120,8 @@ def load_library(path: Optional[str] = None):
     for fn in (lib.specsteer_lmhead_shard_combine, lib.specsteer_lmhead_shard_recover):
         fn.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         fn.restype = C.c_int
+    lib.specsteer_probe_ex2.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+    lib.specsteer_probe_ex2.restype = C.c_int
     lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
     lib.specsteer_ctx_time_streaming.restype = C.c_int
     lib.specsteer_ctx_launch_count.argtypes = [C.c_void_p]
@@ -391,6 +394,18 @@ class Context:
     @property
     def launch_count(self) -> int:
         return int(self._lib.specsteer_ctx_launch_count(self._h))
+
+
+def probe_ex2(n_ctas: int, iters: int, sink: torch.Tensor, stream=None) -> int:
+    """Launch the ex2.approx rate probe (a measurement aid) on the current stream; returns the evaluations it makes."""
+    if not torch.cuda.is_available():
+        raise RuntimeError("specsteer needs a CUDA device; there is no CPU fallback")
+    if sink.dtype != torch.float32 or not sink.is_contiguous() or sink.numel() < n_ctas * 1024:
+        raise ValueError("sink must be a contiguous float32 tensor of at least n_ctas * 1024 elements")
+    s = stream if stream is not None else torch.cuda.current_stream()
+    _check(load_library().specsteer_probe_ex2(int(n_ctas), int(iters), C.c_void_p(sink.data_ptr()), C.c_void_p(s.cuda_stream)),
+           "specsteer_probe_ex2")
+    return int(n_ctas) * 1024 * 8 * int(iters)
 
 
 def verify_round_static(desc: RoundDesc, stream=None):

@@ -9,7 +9,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libspecsteer.so")
-SOURCES = ["api.cu", "verify.cu", "recover.cu", "topk.cu", "lmhead.cu", "static_scratch.cu"]
+SOURCES = ["api.cu", "verify.cu", "recover.cu", "topk.cu", "lmhead.cu", "static_scratch.cu", "probe.cu"]
 HEADERS = ["common.cuh", "internal.h", "records.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v"]

@@ -20,6 +20,7 @@ struct specsteer_ctx {
   float* lse2;
   int* status_ws;
   int* dev_error;
+  float* row_ref;     // [max_B*(max_K+1)][4] reference exponents per row for the streaming kernel of large rounds
   void* topk_lists;   // [max_B][kTopkMaxSplit][32] keys of the split top-k selection
   int* topk_count;    // [max_B], zero between launches
   // last verified round, for the order check
@@ -153,6 +154,11 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
 // Verification needs the normalisers of h_LLM and h_SLM- only (Eq. 7); when nobody asks for a quantity of the
 // fused target on the drafted rows, the h_SLM+ tensor is left unread there and the recovery call forms the
 // normalisers of its one row itself (Eq. 8 on the row of the first rejection).
+bool large_round(const specsteer_round_desc* d) {
+  const double bytes = 3.0 * d->B * (d->K + 1) * (double)d->V * (d->dtype == SPECSTEER_F32 ? 4 : 2);
+  return bytes >= 128.0 * 1024 * 1024;
+}
+
 bool two_phase(const specsteer_round_desc* d) {
   const bool eligible = d->accept_mode == SPECSTEER_ACCEPT_RATIO &&
                         (d->recover_mode == SPECSTEER_RECOVER_STEER || d->recover_mode == SPECSTEER_RECOVER_ARGMAX) &&
@@ -160,8 +166,7 @@ bool two_phase(const specsteer_round_desc* d) {
   if (!eligible) return false;
   if (d->flags & SPECSTEER_FLAG_TWO_PHASE) return true;
   // one more launch and a short second pass (about 10 us) against a fifth of the bytes: worth it from roughly 128 MB of logits upwards
-  const double bytes = 3.0 * d->B * (d->K + 1) * (double)d->V * (d->dtype == SPECSTEER_F32 ? 4 : 2);
-  return bytes >= 128.0 * 1024 * 1024;
+  return large_round(d);
 }
 
 // Verification of the requests [b0, b0 + nb).  lean: two tensors over the drafted rows, in the larger chunks of that
@@ -175,6 +180,10 @@ specsteer_status verify_slab(specsteer_ctx* ctx, const specsteer_round_desc* d, 
     p.tile = d->dtype == SPECSTEER_F32 ? kChunkRatioF32 : kChunkRatioBF16;
     p.n_chunks = n_chunks_of(d->V, p.tile);
   }
+  // Large rounds take the reference exponents of a row from its drafted token (one small launch in front of the
+  // streaming kernel), so that heavy-tailed rows at low temperature stay on the streaming kernel's fast path; below
+  // about 128 MB of logits the extra launch costs more than it can save.
+  if (large_round(d) && rows_aligned(d)) p.row_ref = ctx->row_ref + (size_t)b0 * (d->K + 1) * 4;
   int nl = 0;
   if (launch_verify(p, d->dtype, rows_aligned(d), ctx->li, s, &nl, ev_begin, ev_end) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   ctx->launches += nl;
@@ -254,7 +263,7 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   const size_t b_st = align_up((size_t)max_B * sizeof(int), 256);
   const size_t b_tl = align_up((size_t)max_B * kTopkMaxSplit * 32 * sizeof(unsigned long long), 256);
   const size_t b_tc = align_up((size_t)max_B * sizeof(int), 256);
-  c->ws_bytes = b_part + b_lse + b_st + 256 + b_tl + b_tc;
+  c->ws_bytes = b_part + 2 * b_lse + b_st + 256 + b_tl + b_tc;
   if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
     cudaGetLastError();
     delete c;
@@ -263,6 +272,7 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   char* w = (char*)c->ws;
   c->part = (float*)w; w += b_part;
   c->lse2 = (float*)w; w += b_lse;
+  c->row_ref = (float*)w; w += b_lse;
   c->status_ws = (int*)w; w += b_st;
   c->dev_error = (int*)w; w += 256;
   c->topk_lists = (void*)w; w += b_tl;

@@ -61,6 +61,8 @@ struct RoundParams {
   float* lse2;        // [B*(K+1)][4]            base-2 log-normalisers {L,P,M,R}
   int* status_ws;     // [B]                     request status when the caller passes no req_status
   int* dev_error;     // [1]                     set when a bounded wait gave up
+  float* row_ref;     // [B*(K+1)][4]            reference exponents per row {L,P,M,R} (row_ref_kernel), or null: the
+                      //                         chunks take their references from their own first batch
   // vocabulary-sharded path (n_shards == 0: the tensors hold the whole vocabulary)
   const ShardPartial* shard_parts;  // [n_shards][B][K+1] gathered partials
   int n_shards, shard_rank;
@@ -119,6 +121,8 @@ cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_
                               void* lists_ws, int* count_ws, int sm_count, cudaStream_t s);
 cudaError_t launch_edge_resample(const RoundParams& p, int dtype, int k, const int* topk_idx, const float* topk_val,
                                  cudaStream_t s);
+// the reference exponents of every row (p.row_ref), for the streaming kernel launched next on the same stream
+cudaError_t launch_row_ref(const RoundParams& p, int dtype, cudaStream_t s);
 // the streaming kernel alone (partial records into the workspace), no epilogue
 cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s);
 // per-row ShardPartial of this shard from its partial records: out[B][K+1]

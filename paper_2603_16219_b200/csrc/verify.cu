@@ -22,10 +22,14 @@ namespace specsteer {
 
 constexpr float kSlack = 16.f;  // careful path: the reference exponent may lag the running maximum by this much
 
-struct TileMeta {
+struct alignas(16) TileMeta {
+  float ref[4];            // reference exponents of the row for the four normalisers (row_ref_kernel); ref[0] NaN: none.
+                           // First and 16-byte aligned: they arrive with the tile, as a fourth bulk copy
   int row, tile, n_valid;  // padded row index b*(K+1)+t, tile within the row, valid entries in the tile
   float beta, c, inv_c;    // beta_b, log2(e)/T_b and its reciprocal for the owning request
+  int pad[2];
 };
+static_assert(sizeof(TileMeta) == 48, "stage metadata: 16 bytes of references, then the tile's coordinates");
 
 // Packed pairs of float32 (sm_100 f32x2 arithmetic): one instruction, two lanes of a 64-bit register.
 typedef unsigned long long f32x2;
@@ -75,12 +79,10 @@ __device__ __forceinline__ void acc_set_ref(Acc& a, int q, float nr, float inv_c
 }
 
 // First batch of a chunk: the references come from the warp-wide maxima of this batch, plus `bias`.
-__device__ __forceinline__ void acc_start(Acc& a, const float (&bm)[4], float c, float inv_c, int lane,
-                                          float bias = 0.f) {
-  const float mine = warp_reduce4<true>(bm, lane);
+__device__ __forceinline__ void acc_start(Acc& a, const float (&bm)[4], float c, float inv_c, float bias = 0.f) {
 #pragma unroll
   for (int q = 0; q < 4; ++q) {
-    acc_set_ref(a, q, ceilf(__shfl_sync(kFullMask, mine, 8 * q) * c) + bias, inv_c);
+    acc_set_ref(a, q, ceilf(warp_max_redux(bm[q]) * c) + bias, inv_c);   // one warp-wide float maximum each
     a.s2[q] = 0ull;
   }
 }
@@ -116,6 +118,49 @@ __device__ __forceinline__ void exp_sum8(f32x2& s2, const f32x2 (&x)[4], f32x2 c
   }
 }
 
+// 2^a for a pair of arguments on the FMA and integer pipes instead of the special-function unit, which 16-bit
+// logits saturate (half the bytes per power of two): a is clamped below at -126, n = round(a) comes from the
+// 1.5 * 2^23 trick, 2^(a - n) from a cubic (relative error below 7.5e-5, 5e-6 on average), and n is added into the
+// exponent field.  Used for the normaliser of h_SLM+ alone, which no decision depends on under the ratio rule
+// (it feeds logp_plus and log_z).  amax collects the largest argument: the caller rejects the chunk when it is not
+// below 120, since above 127 the exponent field would overflow; a NaN argument is swallowed by the clamp, which is
+// why the caller also forms the normaliser of h_rec (NaN there whenever h_SLM+ is NaN) with ex2.
+__device__ __forceinline__ f32x2 exp2_cubic2(f32x2 a, float& amax) {
+  const float kMagic = 12582912.f;  // 1.5 * 2^23
+  float a0, a1;
+  unpack2(a, a0, a1);
+  amax = max3(amax, a0, a1);
+  const f32x2 ac = pack2(fmaxf(a0, -126.f), fmaxf(a1, -126.f));
+  const f32x2 magic2 = pack2(kMagic, kMagic);
+  const f32x2 y = add2(ac, magic2);
+  const f32x2 f = sub2(ac, sub2(y, magic2));   // in [-0.5, 0.5]
+  f32x2 q = pack2(0.05517147481441498f, 0.05517147481441498f);
+  q = fma2(q, f, pack2(0.24261066317558289f, 0.24261066317558289f));
+  q = fma2(q, f, pack2(0.6932609677314758f, 0.6932609677314758f));
+  q = fma2(q, f, pack2(0.9999281167984009f, 0.9999281167984009f));
+  float q0, q1, y0, y1;
+  unpack2(q, q0, q1);
+  unpack2(y, y0, y1);
+  return pack2(__uint_as_float(__float_as_uint(q0) + (__float_as_uint(y0) << 23)),
+               __uint_as_float(__float_as_uint(q1) + (__float_as_uint(y1) << 23)));
+}
+
+// exp_sum8 with the first NPOLY of the four pairs on the cubic
+template <int NPOLY>
+__device__ __forceinline__ void exp_sum8_mixed(f32x2& s2, const f32x2 (&x)[4], f32x2 c2, f32x2 nref2, float& amax) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const f32x2 arg = fma2(x[i], c2, nref2);
+    if (i < NPOLY) {
+      s2 = add2(s2, exp2_cubic2(arg, amax));
+    } else {
+      float a0, a1;
+      unpack2(arg, a0, a1);
+      s2 = add2(s2, pack2(ex2(a0), ex2(a1)));
+    }
+  }
+}
+
 // Eight vocabulary entries per lane of the three streams: r = l + beta (p - m)  (Eq. 8), then the four sums.
 template <bool MASKED, bool FIRST, int SUMS>
 __device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32x2 (&m)[4], f32x2 beta2, f32x2 c2,
@@ -140,7 +185,7 @@ __device__ __forceinline__ void accum8(Acc& a, f32x2 (&l)[4], f32x2 (&p)[4], f32
   const float bm[4] = {(SUMS & SUM_L) ? max8(l) : kNegInf, (SUMS & SUM_P) ? max8(p) : kNegInf,
                        (SUMS & SUM_M) ? max8(m) : kNegInf, (SUMS & SUM_R) ? max8(r) : kNegInf};
   if (FIRST) {
-    acc_start(a, bm, c, inv_c, lane);
+    acc_start(a, bm, c, inv_c);
   } else {
     const bool upd = (bm[0] > a.thr[0]) | (bm[1] > a.thr[1]) | (bm[2] > a.thr[2]) | (bm[3] > a.thr[3]);
     if (__any_sync(kFullMask, upd)) acc_raise(a, bm, c, inv_c, lane);
@@ -207,19 +252,27 @@ __device__ __forceinline__ void chunk_pass(Acc& a, const T* sl, const T* sp, con
   }
 }
 
-// The fast variant for a full chunk.  Only the first batch computes maxima: the references are set kBias
-// binades above them, so that later entries may exceed the first batch's maximum by 2^(kBias + 120)
-// before a sum overflows, while entries down to 2^-(126 - kBias) of it still count.  Nothing is tested
-// inside the chunk; at its end a sum that is not below 2^120 (or is NaN) makes the warp return false and
-// the caller redoes the chunk with chunk_pass, which tests every batch.
+// The fast variant for a full chunk: nothing is tested inside it.  The reference exponents come from the row
+// (row_ref_kernel: kBias binades above the row's logits at its drafted token, which was sampled from Softmax(h_SLM+)
+// and so lies near the top of the row) or, when the row has none, from the maxima of the chunk's first batch plus
+// kBias.  Either way later entries may exceed the value the reference was taken from by 2^(kBias + 120) before a sum
+// overflows, while entries down to 2^-(126 - kBias) of it still count (what is dropped is below 2^-66 of an entry
+// of the row).  At the chunk's end a sum that is not below 2^120 (or is NaN), or a cubic argument that left its
+// range, makes the warp return false and the caller redoes the chunk with chunk_pass, which tests every batch.
+// POLY: the first POLY of the four pairs per batch of h_SLM+ take the cubic instead of ex2.approx.
 constexpr float kBias = 60.f;
 
-template <typename T, int CHUNK, int SUMS>
+template <typename T, int CHUNK, int SUMS, int POLY, bool REF>
 __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, const T* sm, int lane, float beta,
-                                           float c, float inv_c) {
+                                           float c, float inv_c, const float* row_ref) {
   const f32x2 beta2 = pack2(beta, beta), c2 = pack2(c, c);
   constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;   // the h_SLM+ slot is filled and read
-  {
+  static_assert(POLY == 0 || (SUMS & SUM_R), "a NaN in h_SLM+ must still reach a sum formed with ex2");
+  float amax = kNegInf;
+  if (REF) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { acc_set_ref(a, q, (SUMS & (1 << q)) ? row_ref[q] : kNegInf, inv_c); a.s2[q] = 0ull; }
+  } else {   // the first batch apart: it also gives the references
     f32x2 l[4], p[4], m[4], r[4];
     Batch<T>::load(sl, 0, lane, l);
     if (kPlus) Batch<T>::load(sp, 0, lane, p);
@@ -230,14 +283,17 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     }
     const float bm[4] = {(SUMS & SUM_L) ? max8(l) : kNegInf, (SUMS & SUM_P) ? max8(p) : kNegInf,
                          (SUMS & SUM_M) ? max8(m) : kNegInf, (SUMS & SUM_R) ? max8(r) : kNegInf};
-    acc_start(a, bm, c, inv_c, lane, kBias);
+    acc_start(a, bm, c, inv_c, kBias);
     if (SUMS & SUM_L) exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    if (SUMS & SUM_P) exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (SUMS & SUM_P) {
+      if (POLY > 0) exp_sum8_mixed<POLY>(a.s2[Q_P], p, c2, a.nref2[Q_P], amax);
+      else exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    }
     if (SUMS & SUM_M) exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
     if (SUMS & SUM_R) exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
 #pragma unroll 1
-  for (int it = 1; it < CHUNK / 256; ++it) {
+  for (int it = REF ? 0 : 1; it < CHUNK / 256; ++it) {
     f32x2 l[4], p[4], m[4], r[4];
     Batch<T>::load(sl, it, lane, l);
     if (kPlus) Batch<T>::load(sp, it, lane, p);
@@ -247,7 +303,10 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
       for (int i = 0; i < 4; ++i) r[i] = fma2(beta2, sub2(p[i], m[i]), l[i]);
     }
     if (SUMS & SUM_L) exp_sum8(a.s2[Q_L], l, c2, a.nref2[Q_L]);
-    if (SUMS & SUM_P) exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    if (SUMS & SUM_P) {
+      if (POLY > 0) exp_sum8_mixed<POLY>(a.s2[Q_P], p, c2, a.nref2[Q_P], amax);
+      else exp_sum8(a.s2[Q_P], p, c2, a.nref2[Q_P]);
+    }
     if (SUMS & SUM_M) exp_sum8(a.s2[Q_M], m, c2, a.nref2[Q_M]);
     if (SUMS & SUM_R) exp_sum8(a.s2[Q_R], r, c2, a.nref2[Q_R]);
   }
@@ -259,6 +318,7 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
     unpack2(a.s2[q], s0, s1);
     bad |= !(s0 + s1 < kBig);
   }
+  if (POLY > 0) bad |= !(amax < 120.f);
   return !__any_sync(kFullMask, bad);
 }
 
@@ -484,7 +544,7 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 // producer thread that owns the stages congruent to its index modulo NPW (one thread cannot issue tiles
 // fast enough for a whole SM).  Every stage is always consumed by the same pair of warps, so a waiting
 // warp is never a whole barrier phase ahead of the data.
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS, int POLY>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
   constexpr int TILE = 2 * CHUNK;
   constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;  // h_SLM+ is read at all
@@ -569,6 +629,8 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
     int cr = g0 / tiles_per_row, tr = g0 % tiles_per_row;
     int b = 0;
     const int K1 = K + 1;
+    const float4 no_ref = make_float4(__int_as_float(0x7fc00000), 0.f, 0.f, 0.f);
+    if (p.row_ref) pdl_wait();   // the row references come from the kernel launched just before this one
     if (BULK) {
       if (lane == 0) {  // one elected thread issues the bulk copies
         int issued = 0;
@@ -585,19 +647,27 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
           const int n_valid = min(TILE, p.V - tr * TILE);
           const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + (long long)tr * TILE;
           T* dst = tiles + (size_t)stage * NSLOT * TILE;
-          meta[stage] = TileMeta{b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b]};
+          TileMeta* mt = &meta[stage];
+          mt->row = b * K1 + t; mt->tile = tr; mt->n_valid = n_valid;
+          mt->beta = beta_s[b]; mt->c = c_s[b]; mt->inv_c = ic_s[b];
+          // the row's reference exponents travel with the tile: a fourth bulk copy, 16 bytes, onto the same barrier
+          const uint32_t ref_bytes = p.row_ref ? 16u : 0u;
+          if (!p.row_ref) mt->ref[0] = no_ref.x;
           const int n_bulk = (int)(((size_t)n_valid * sizeof(T)) & ~(size_t)15) / (int)sizeof(T);
           for (int e = n_bulk; e < n_valid; ++e) {  // ragged end of the last tile: < 16 bytes per stream
             dst[e] = hl[off + e]; dst[MSLOT * TILE + e] = hm[off + e];
             if (kPlus) dst[TILE + e] = hp[off + e];
           }
           const uint32_t bytes = (uint32_t)(n_bulk * sizeof(T));
+          if (bytes + ref_bytes) {
+            mbar_arrive_expect_tx(&full[stage], (kPlus ? 3 : 2) * bytes + ref_bytes);
+            if (ref_bytes) bulk_g2s(mt->ref, p.row_ref + 4ll * (b * K1 + t), 16u, &full[stage]);
+          }
           if (bytes) {
-            mbar_arrive_expect_tx(&full[stage], (kPlus ? 3 : 2) * bytes);
             bulk_g2s(dst, hl + off, bytes, &full[stage]);
             if (kPlus) bulk_g2s(dst + TILE, hp + off, bytes, &full[stage]);
             bulk_g2s(dst + MSLOT * TILE, hm + off, bytes, &full[stage]);
-          } else {
+          } else if (!ref_bytes) {
             mbar_arrive(&full[stage]);
           }
           ++issued;
@@ -634,7 +704,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
         }
         __syncwarp();
         if (lane == 0) {
-          meta[stage] = TileMeta{b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b]};
+          meta[stage] = TileMeta{{no_ref.x, 0.f, 0.f, 0.f}, b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b], {0, 0}};
           mbar_arrive(&full[stage]);
         }
         cr += step_rows; tr += step_tiles;
@@ -659,7 +729,10 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       const T* sl = tiles + (size_t)stage * NSLOT * TILE + half * CHUNK;
       Acc a;
       if (nv >= CHUNK) {
-        if (!chunk_fast<T, CHUNK, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, mt.beta, mt.c, mt.inv_c))
+        const bool fast = (mt.ref[0] == mt.ref[0])
+            ? chunk_fast<T, CHUNK, SUMS, POLY, true>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, mt.beta, mt.c, mt.inv_c, mt.ref)
+            : chunk_fast<T, CHUNK, SUMS, POLY, false>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, mt.beta, mt.c, mt.inv_c, mt.ref);
+        if (!fast)
           chunk_pass<T, CHUNK, false, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, CHUNK, mt.beta, mt.c, mt.inv_c);
       } else if (nv > 0) chunk_pass<T, CHUNK, true, SUMS>(a, sl, sl + TILE, sl + MSLOT * TILE, lane, nv, mt.beta, mt.c, mt.inv_c);
       __syncwarp();
@@ -696,12 +769,12 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
 }
 
 // ---- launch -------------------------------------------------------------------------------------------
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS, int POLY = 0>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
   const size_t fixed = (size_t)STAGES * ((SUMS & (SUM_P | SUM_R)) ? 3 : 2) * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
                        STAGES * sizeof(TileMeta) + 16;
   const size_t smem = fixed + (size_t)(5 * p.B + 1) * sizeof(int);
-  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS>;
+  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS, POLY>;
   // per instantiation and device; sized for the largest slab.  Contexts may be driven from different host threads:
   // the flag is atomic, and two threads that both find it clear merely set the same attribute twice.
   static std::atomic<bool> attr_set_dev[64];
@@ -712,7 +785,68 @@ static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cud
     if (e != cudaSuccess) return e;
     attr_set.store(true, std::memory_order_release);
   }
-  kern<<<li.sm_count, (NCW + NPW) * 32, smem, s>>>(p);
+  if (!p.row_ref) {
+    kern<<<li.sm_count, (NCW + NPW) * 32, smem, s>>>(p);
+    return cudaGetLastError();
+  }
+  // The row references were written by row_ref_kernel, launched just before on the same stream: this kernel may
+  // start while that one drains (its producers wait for it before they read a reference).
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(li.sm_count);
+  cfg.blockDim = dim3((NCW + NPW) * 32);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, p);
+}
+
+// ---- reference exponents per row ------------------------------------------------------------------------
+// One thread per row (b, t) that will be streamed: the row's pivot is its drafted token (for the row a recovery pass
+// streams: the token that was rejected there), which was drawn from Softmax(h_SLM+ / T) and therefore sits near the
+// top of the row in all three tensors.  The references are kBias binades above the pivot's scaled logits, so a chunk
+// overflows the fast path only if it holds an entry 2^(kBias + 120) above the pivot - with per-chunk references it
+// is the first 256 entries of every chunk that have to be representative, which heavy-tailed rows at low
+// temperature are not.  A row without a usable pivot (the bonus row, a bad token, non-finite logits) gets NaN and
+// its chunks fall back to their own first batch.
+template <typename T>
+__global__ void __launch_bounds__(128) row_ref_kernel(const RoundParams p, float4* out) {
+  pdl_launch_dependents();
+  const int K = p.K, K1 = K + 1;
+  const int row = blockIdx.x * 128 + threadIdx.x;
+  if (row >= p.B * K1) return;
+  const int b = row / K1, t = row - b * K1;
+  float4 ref = make_float4(__int_as_float(0x7fc00000), 0.f, 0.f, 0.f);
+  int len = p.draft_len[b];
+  if (len < 0 || len > K) len = 0;
+  const float Tmp = p.temperature[b], beta = p.beta[b];
+  if (t < len && Tmp > 0.f) {
+    const int y = p.draft_tokens[(long long)b * K + t];
+    if (y >= 0 && y < p.V) {
+      const long long off = (long long)b * p.ld_req + (long long)t * p.ld_row + y;
+      const float l = load_logit<T>(reinterpret_cast<const T*>(p.h_llm), off);
+      const float m = load_logit<T>(reinterpret_cast<const T*>(p.h_minus), off);
+      // the two-phase verification never touches h_SLM+ on a drafted row
+      const float pp = (p.sums & (SUM_P | SUM_R)) ? load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off) : l;
+      const float c = kLog2e / Tmp;
+      const float4 cand = make_float4(ceilf(l * c) + kBias, ceilf(pp * c) + kBias, ceilf(m * c) + kBias,
+                                      ceilf(fmaf(beta, pp - m, l) * c) + kBias);
+      const float big = 1e30f;
+      if (fabsf(cand.x) < big && fabsf(cand.y) < big && fabsf(cand.z) < big && fabsf(cand.w) < big) ref = cand;
+    }
+  }
+  out[row] = ref;
+}
+
+cudaError_t launch_row_ref(const RoundParams& p, int dtype, cudaStream_t s) {
+  const int rows = p.B * (p.K + 1);
+  if (rows == 0 || !p.row_ref) return cudaSuccess;
+  float4* out = reinterpret_cast<float4*>(p.row_ref);
+  if (dtype == SPECSTEER_F32) row_ref_kernel<float><<<(rows + 127) / 128, 128, 0, s>>>(p, out);
+  else row_ref_kernel<uint16_t><<<(rows + 127) / 128, 128, 0, s>>>(p, out);
   return cudaGetLastError();
 }
 
@@ -780,6 +914,11 @@ cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, 
     return launch_stream<float, kChunkRatioF32, 12, 12, 3, true, kRatio>(p, li, s);
   }
   if (!aligned) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, false, SUM_ALL>(p, li, s);
+  // 16-bit logits with all four normalisers are bound by the special-function unit: under the ratio rule, where the
+  // normaliser of h_SLM+ decides nothing, three of its four pairs per batch take the cubic (5574 against 5274 GB/s
+  // on the largest benchmark shape; one, two and four pairs gave 5363, 5512 and 5500)
+  if (sums == SUM_ALL && p.accept_mode == SPECSTEER_ACCEPT_RATIO)
+    return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL, 3>(p, li, s);
   if (sums == SUM_ALL) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL>(p, li, s);
   if (sums == kNoPlus) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kNoPlus>(p, li, s);
   return launch_stream<uint16_t, kChunkRatioBF16, 16, 16, 4, true, kRatio>(p, li, s);
@@ -805,6 +944,10 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
                           int* n_launches, cudaEvent_t ev_begin, cudaEvent_t ev_end) {
   *n_launches = 2;
   cudaError_t e;
+  if (p.row_ref) {
+    if ((e = launch_row_ref(p, dtype, s)) != cudaSuccess) return e;
+    *n_launches = 3;
+  }
   if (ev_begin && (e = cudaEventRecord(ev_begin, s)) != cudaSuccess) return e;
   if ((e = launch_verify_stream(p, dtype, aligned, li, s)) != cudaSuccess) return e;
   if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;

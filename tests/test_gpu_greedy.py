@@ -107,7 +107,7 @@ def test_full_size_every_request(env, cfg):
     env["ctx"].verify_round(d)
     env["ctx"].recover_sample(d)
     torch.cuda.synchronize()
-    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 3
+    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 4   # row references, stream, epilogue, argmax
     two = {k: v.cpu().numpy() for k, v in outs.items()}
     stats = P.compare(env["oracle"], two, P.to_np_inputs(inputs), 0, ARGMAX, 1, P.TOL[inputs["h_llm"].dtype], alg1=True,
                       keys=keys)
@@ -188,7 +188,7 @@ def test_two_phase_greedy_full_size_equals_one_pass(env):
     env["ctx"].verify_round(d)
     env["ctx"].recover_sample(d)
     torch.cuda.synchronize()
-    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 3
+    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == 4
     for k in ("accept_len", "rec_token", "n_out", "out_tokens", "req_status", "accept_flags"):
         assert np.array_equal(outs[k].cpu().numpy(), full[k]), k
     assert np.abs(outs["rec_logprob"].cpu().numpy() - full["rec_logprob"]).max() <= 1e-5

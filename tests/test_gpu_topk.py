@@ -17,7 +17,7 @@ def env(oracle_mod):
     from paper_2603_16219_b200 import binding, build, synth
     assert torch.cuda.is_available()
     build.build()
-    ctx = binding.Context(max_B=64, max_K=8, max_V=160000, device=0)
+    ctx = binding.Context(max_B=512, max_K=8, max_V=262144, device=0)
     yield {"binding": binding, "synth": synth, "oracle": oracle_mod, "ctx": ctx}
     ctx.close()
 
@@ -69,7 +69,7 @@ def _run(env, inputs, k, flags, V=None, cloud_only_verification=False):
         if gpu["rec_token"][r] >= 0:
             assert gpu["out_tokens"][r][n] == gpu["rec_token"][r]
         assert (gpu["out_tokens"][r][want_n:] == -1).all()
-    assert n_checked >= B - 1
+    assert n_checked >= B - max(1, B // 64)
     return gpu, top
 
 
@@ -111,14 +111,13 @@ def test_topk_unaligned_rows(env):
     _run(env, inputs, 32, 1, V=1001)
 
 
-@pytest.mark.parametrize("cfg", [0, 2])
+@pytest.mark.parametrize("cfg", [0, 2, 3, 4])
 def test_topk_on_benchmark_shapes(env, cfg):
-    import dataclasses
+    """The benchmark configurations at their full batch size, every request."""
     spec = env["synth"].CONFIGS[cfg]
-    spec = dataclasses.replace(spec, B=min(spec.B, 12))
     inputs = env["synth"].make_round(spec, device="cuda", seed=cfg)
     gpu, top = _run(env, inputs, 32, 1)
-    assert (gpu["rec_token"] >= 0).all()
+    assert (gpu["rec_token"] >= 0).all() and gpu["rec_token"].shape[0] == spec.B
 
 
 def test_topk_after_verification_without_h_slm_plus(env):

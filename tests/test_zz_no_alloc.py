@@ -73,6 +73,7 @@ def test_static_entry_point_rejects_shapes_beyond_its_scratch():
     # too many partial records: 16 requests x 9 rows x ceil(2_000_000 / 1024) chunks
     desc = binding.make_desc(inputs, outs)
     desc.B, desc.K, desc.V, desc.ld_row, desc.ld_req = 16, 8, 2_000_000, 2_000_000, 9 * 2_000_000
+    desc.draft_tokens = desc.u_accept = desc.lam      # K > 0 wants these two set; the call is refused before any launch
     with pytest.raises(binding.SpecSteerError) as e:
         binding.verify_round_static(desc)
     assert e.value.code == binding.ERR_STATIC_LIMIT
