@@ -314,6 +314,16 @@ specsteer_status specsteer_verify_round_static(const specsteer_round_desc *desc,
  * SPECSTEER_OK or SPECSTEER_ERR_TIMEOUT (sticky until the context is destroyed). */
 specsteer_status specsteer_ctx_device_error(specsteer_ctx *ctx);
 
+/* Test hook for the library's only failure detector.  Every wait inside the streaming kernel (a consumer warp for a
+ * tile's bytes, a producer thread for a free stage) is bounded: after `sm_clocks` SM clocks it gives up, the CTA records
+ * the error, waits for the copies it has in flight and returns, and specsteer_ctx_device_error reports
+ * SPECSTEER_ERR_TIMEOUT.  The default (0 restores it) is 2^33 clocks, a few seconds, which no healthy run reaches; a
+ * limit of a few hundred clocks makes the first wait for data run out, which is how the give-up path is exercised
+ * without hanging or faulting anything.  Outputs of a round that gave up are undefined (but every access stays in
+ * bounds).  Applies to specsteer_verify_round / _recover_sample / _round_host / the sharded logit rounds of this
+ * context.  Errors: INVALID_ARG (NULL ctx, negative limit). */
+specsteer_status specsteer_ctx_set_wait_limit(specsteer_ctx *ctx, int64_t sm_clocks);
+
 /* Profiling hook: from now on specsteer_verify_round records the two caller-owned CUDA events (cudaEvent_t
  * passed as void*, created with timing enabled) on its stream just before and just after the streaming
  * kernel, the launch that reads all the logits, so that a benchmark can time that kernel alone; the per-request

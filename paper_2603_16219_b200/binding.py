@@ -33,7 +33,7 @@ EXPORTS = (
     "specsteer_lmhead_round",
     "specsteer_lmhead_shard_local", "specsteer_lmhead_shard_combine", "specsteer_lmhead_shard_recover",
     "specsteer_shard_greedy_local", "specsteer_lmhead_shard_greedy_local", "specsteer_shard_greedy_finish",
-    "specsteer_probe_ex2",
+    "specsteer_probe_ex2", "specsteer_ctx_set_wait_limit",
 )
 SHARD_PARTIAL_BYTES = 64
 MAX_SHARDS = 32
@@ -120,6 +120,8 @@ def load_library(path: Optional[str] = None):
     for fn in (lib.specsteer_lmhead_shard_combine, lib.specsteer_lmhead_shard_recover):
         fn.argtypes = [C.c_void_p, C.POINTER(LmheadDesc), C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_void_p]
         fn.restype = C.c_int
+    lib.specsteer_ctx_set_wait_limit.argtypes = [C.c_void_p, C.c_int64]
+    lib.specsteer_ctx_set_wait_limit.restype = C.c_int
     lib.specsteer_probe_ex2.argtypes = [C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
     lib.specsteer_probe_ex2.restype = C.c_int
     lib.specsteer_ctx_time_streaming.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
@@ -383,6 +385,11 @@ class Context:
         a = C.c_void_p(ev_begin.cuda_event) if ev_begin is not None else None
         b = C.c_void_p(ev_end.cuda_event) if ev_end is not None else None
         _check(self._lib.specsteer_ctx_time_streaming(self._h, a, b), "specsteer_ctx_time_streaming")
+
+    def set_wait_limit(self, sm_clocks: int):
+        """Give-up limit of the streaming kernel's bounded waits, in SM clocks (0 = the default of a few seconds).
+        A test hook: see specsteer_ctx_set_wait_limit."""
+        _check(self._lib.specsteer_ctx_set_wait_limit(self._h, int(sm_clocks)), "specsteer_ctx_set_wait_limit")
 
     def device_error(self) -> int:
         return int(self._lib.specsteer_ctx_device_error(self._h))

@@ -28,6 +28,7 @@ struct specsteer_ctx {
   int v_B, v_K, v_V, v_dtype;
   const void* v_h_llm;
   uint64_t launches;
+  long long wait_cycles;   // give-up limit of the streaming kernel's waits (specsteer_ctx_set_wait_limit)
   bool poisoned;
   bool shard_streamed;   // specsteer_shard_verify_local ran for the shape in v_*
   bool v_two_phase;      // the last verify_round left the recovery rows unread (see two_phase())
@@ -148,6 +149,7 @@ RoundParams slab_params(const specsteer_ctx* ctx, const specsteer_round_desc* d,
   p.status_ws = ctx->status_ws + b0;
 #undef OFF
   p.dev_error = ctx->dev_error;
+  p.wait_cycles = ctx->wait_cycles;
   return p;
 }
 
@@ -250,6 +252,7 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   if (!c) return SPECSTEER_ERR_WORKSPACE;
   memset(c, 0, sizeof *c);
   c->device = device; c->max_B = max_B; c->max_K = max_K; c->max_V = max_V;
+  c->wait_cycles = kDefaultWaitCycles;
   c->li.device = device;
   if (cudaDeviceGetAttribute(&c->li.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
       cudaDeviceGetAttribute(&c->li.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) {
@@ -837,6 +840,12 @@ specsteer_status specsteer_ctx_device_error(specsteer_ctx* ctx) {
   if (cudaMemcpy(&flag, ctx->dev_error, sizeof flag, cudaMemcpyDeviceToHost) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   if (flag) ctx->poisoned = true;
   return flag ? SPECSTEER_ERR_TIMEOUT : SPECSTEER_OK;
+}
+
+specsteer_status specsteer_ctx_set_wait_limit(specsteer_ctx* ctx, int64_t sm_clocks) {
+  if (!ctx || sm_clocks < 0) return SPECSTEER_ERR_INVALID_ARG;
+  ctx->wait_cycles = sm_clocks == 0 ? kDefaultWaitCycles : (long long)sm_clocks;
+  return SPECSTEER_OK;
 }
 
 specsteer_status specsteer_ctx_time_streaming(specsteer_ctx* ctx, void* ev_begin, void* ev_end) {

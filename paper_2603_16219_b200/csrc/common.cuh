@@ -92,18 +92,37 @@ __device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity, uint32
       : "memory");
   return ok != 0;
 }
-// Bounded wait: gives up once kWaitCycles SM clocks (a few seconds) have passed and returns false;
-// the caller then records an error and unwinds.
+// The phase test that never blocks.
+__device__ __forceinline__ bool mbar_test_nonblocking(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: gives up once `limit` SM clocks have passed (default: a few seconds) and returns false; the caller
+// then records an error and unwinds.  The blocking form of the test may keep a thread suspended for longer than any
+// hint says, so a limit of a few thousand clocks or less (the give-up path under test) polls with the form that
+// never blocks: such a wait ends within its limit whatever the barrier does.
 constexpr long long kWaitCycles = 1ll << 33;
 constexpr uint32_t kSuspendNs = 2000;
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, long long limit = kWaitCycles) {
+  if (limit < 8192) {
+    const long long t0 = clock64();
+    for (;;) {
+      if (mbar_test_nonblocking(bar, parity)) return true;
+      if (clock64() - t0 > limit) return false;
+    }
+  }
   if (mbar_test(bar, parity, kSuspendNs)) return true;
   const long long t0 = clock64();
   for (;;) {
-#pragma unroll 1
-    for (int i = 0; i < 256; ++i)
-      if (mbar_test(bar, parity, kSuspendNs)) return true;
-    if (clock64() - t0 > kWaitCycles) return false;
+    if (mbar_test(bar, parity, kSuspendNs)) return true;
+    if (clock64() - t0 > limit) return false;
   }
 }
 // 1-D bulk copy global -> shared of this CTA alone, completion counted in bytes on `bar`.

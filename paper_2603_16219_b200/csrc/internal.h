@@ -14,6 +14,8 @@ constexpr int kChunkMin = 512;
 // (3 KB per stream): fewer per-chunk set-ups and reductions per byte (measured on 3.15 GB of bf16: 570 -> 512 us).
 constexpr int kChunkRatioF32 = 768;
 constexpr int kChunkRatioBF16 = 1536;
+// A bounded device-side wait gives up after this many SM clocks (a few seconds) unless the context says otherwise.
+constexpr long long kDefaultWaitCycles = 1ll << 33;
 constexpr int kMaxSlabB = 1024;  // requests handled by one launch (per-request tables live in shared memory)
 
 // What one vocabulary shard knows about one row (64 bytes; the unit of the all-gather in the sharded path):
@@ -61,6 +63,7 @@ struct RoundParams {
   float* lse2;        // [B*(K+1)][4]            base-2 log-normalisers {L,P,M,R}
   int* status_ws;     // [B]                     request status when the caller passes no req_status
   int* dev_error;     // [1]                     set when a bounded wait gave up
+  long long wait_cycles;  // give-up limit of the streaming kernel's pipeline waits, in SM clocks
   float* row_ref;     // [B*(K+1)][4]            reference exponents per row {L,P,M,R} (row_ref_kernel), or null: the
                       //                         chunks take their references from their own first batch
   // vocabulary-sharded path (n_shards == 0: the tensors hold the whole vocabulary)

@@ -96,6 +96,7 @@ extern "C" specsteer_status specsteer_verify_round_static(const specsteer_round_
   p.lse2 = reinterpret_cast<float*>(su->base + kPartBytes);
   p.status_ws = reinterpret_cast<int*>(su->base + kPartBytes + kLseBytes);
   p.dev_error = reinterpret_cast<int*>(su->base + kPartBytes + kLseBytes + kStatusBytes);
+  p.wait_cycles = kDefaultWaitCycles;
 
   const bool aligned = rows_aligned(d);
   int nl = 0;

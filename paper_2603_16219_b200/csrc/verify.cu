@@ -637,7 +637,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
         for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
           const int stage = j % STAGES;
           const uint32_t phase = (uint32_t)((j / STAGES) & 1);
-          if (*reinterpret_cast<volatile int*>(abort_flag) || !mbar_wait(&empty[stage], phase ^ 1u)) {
+          if (*reinterpret_cast<volatile int*>(abort_flag) || !mbar_wait(&empty[stage], phase ^ 1u, p.wait_cycles)) {
             *reinterpret_cast<volatile int*>(abort_flag) = 1;
             atomicExch(p.dev_error, 1);
             break;
@@ -689,7 +689,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
         const int stage = j % STAGES;
         const uint32_t phase = (uint32_t)((j / STAGES) & 1);
-        const bool ok = __all_sync(kFullMask, mbar_wait(&empty[stage], phase ^ 1u));
+        const bool ok = __all_sync(kFullMask, mbar_wait(&empty[stage], phase ^ 1u, p.wait_cycles));
         if (!ok || *reinterpret_cast<volatile int*>(abort_flag)) {
           if (lane == 0) { *reinterpret_cast<volatile int*>(abort_flag) = 1; atomicExch(p.dev_error, 1); }
           break;
@@ -718,7 +718,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
       const int stage = j % STAGES;
       const uint32_t phase = (uint32_t)((j / STAGES) & 1);
       // every lane observes the phase itself: that is what makes the copied bytes visible to it
-      bool ok = !*reinterpret_cast<volatile int*>(abort_flag) && mbar_wait(&full[stage], phase);
+      bool ok = !*reinterpret_cast<volatile int*>(abort_flag) && mbar_wait(&full[stage], phase, p.wait_cycles);
       ok = __all_sync(kFullMask, ok);
       if (!ok) {
         if (lane == 0) { *reinterpret_cast<volatile int*>(abort_flag) = 1; atomicExch(p.dev_error, 1); }
