@@ -343,7 +343,8 @@ def run_cuda(args, rank, world, local_rank):
     if args.requests:   # a reduced batch of the same recipe, for profiler captures that must stay small
         import dataclasses
         spec = dataclasses.replace(spec, B=args.requests, name="%s_first%d" % (spec.name, args.requests))
-    flags = binding.FLAG_BONUS
+    flags = binding.FLAG_BONUS | (binding.FLAG_SEPARATE_LAUNCHES if args.separate else 0) | \
+        (binding.FLAG_ONE_LAUNCH if args.one_launch else 0)
     inputs = synth.make_round(spec, device=dev, seed=rank)     # every rank owns its own requests
     rows = synth.used_rows(spec, inputs["draft_len"], bonus=True)
     positions = int(inputs["draft_len"].sum().item())
@@ -469,6 +470,7 @@ def run_cuda(args, rank, world, local_rank):
         if rank == 0:
             line = {"workload": spec.name, "outputs": ("lean, two-phase" if two_phase else "lean, one pass") if args.lean else "all",
                     "recovery": "greedy (argmax of h_rec)" if args.greedy else "sampled", "ms_per_step": ms_per_step,
+                    "launches_per_step": gpu_launches / args.steps,
                     "verify_kernel_ms": kernel_ms, "verify_gbs": logit_bytes / (kernel_ms * 1e-3) / 1e9,
                     "positions_per_s": value, "clocks": sampler.summary()}
             line.update(extra)
@@ -816,6 +818,10 @@ def main():
                     help="with --kernels-only: also time the top-k split recovery (cloud + edge kernels) with this k")
     ap.add_argument("--kernels-only", action="store_true",
                     help="time only the device-resident steps and print a short line (profiling aid)")
+    ap.add_argument("--separate", action="store_true",
+                    help="keep verification and recovery in separate launches (small rounds otherwise run in one launch)")
+    ap.add_argument("--one-launch", action="store_true",
+                    help="take the one-launch round for a small batch of several requests too")
     ap.add_argument("--no-extras", action="store_true",
                     help="skip the blocks beside the headline (the largest configuration; the vocabulary-sharded rounds)")
     ap.add_argument("--vocab-sharded", action="store_true",

@@ -73,9 +73,20 @@ typedef enum {
 
 enum {
   SPECSTEER_FLAG_BONUS = 1u,    /* when all drafts are accepted, also sample one token (STEER) from row draft_len */
-  SPECSTEER_FLAG_TWO_PHASE = 2u /* take the two-phase round (see the outputs below) whenever it is eligible, however
+  SPECSTEER_FLAG_TWO_PHASE = 2u, /* take the two-phase round (see the outputs below) whenever it is eligible, however
                                    small the batch; without it the library takes it from 128 MB of logits upwards,
                                    below which its two extra launches cost more than the bytes it saves */
+  SPECSTEER_FLAG_SEPARATE_LAUNCHES = 4u, /* keep verification and recovery in launches of their own.  Without it a
+                                   round of ONE request (below 128 MB of logits, STEER recovery, 16-byte aligned rows)
+                                   runs in one launch: specsteer_verify_round then also samples the recovery token and
+                                   writes rec_token, rec_logprob, out_tokens and n_out, and the
+                                   specsteer_recover_sample that follows launches nothing.  Same outputs, bit for bit.
+                                   Set it when something else than specsteer_recover_sample follows
+                                   (specsteer_cloud_topk: the sample would be wasted work) or when the recovery outputs
+                                   must not be written before that call. */
+  SPECSTEER_FLAG_ONE_LAUNCH = 8u /* take the one-launch round for a small batch of several requests too (slower than three
+                                   launches on the shapes measured, see above; kept for callers to whom the number of
+                                   launches matters more than the time) */
 };
 
 /* bits of req_status[b].  Every problem a request shows is reported: a bad length together with a bad parameter gives

@@ -21,6 +21,8 @@ ACCEPT_RATIO, ACCEPT_EXACT_Z = 0, 1
 RECOVER_STEER, RECOVER_RESIDUAL, RECOVER_ARGMAX = 0, 1, 2
 FLAG_BONUS = 1
 FLAG_TWO_PHASE = 2
+FLAG_SEPARATE_LAUNCHES = 4
+FLAG_ONE_LAUNCH = 8
 REQ_BAD_TOKEN, REQ_BAD_LEN, REQ_NONFINITE, REQ_RESIDUAL_EMPTY, REQ_BAD_PARAM = 1, 2, 4, 8, 16
 
 EXPORTS = (

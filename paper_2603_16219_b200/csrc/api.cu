@@ -21,6 +21,8 @@ struct specsteer_ctx {
   int* status_ws;
   int* dev_error;
   float* row_ref;     // [max_B*(max_K+1)][4] reference exponents per row for the streaming kernel of large rounds
+  int* req_done;      // [max_B] chunks retired per request in the one-launch round; zero between launches
+  bool v_fused;       // the last verify_round ran the whole round (recover_sample then has nothing to launch)
   void* topk_lists;   // [max_B][kTopkMaxSplit][32] keys of the split top-k selection
   int* topk_count;    // [max_B], zero between launches
   // last verified round, for the order check
@@ -62,7 +64,7 @@ specsteer_status check_round_desc(const specsteer_round_desc* d, bool need_u_rec
   if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_RESIDUAL &&
       d->recover_mode != SPECSTEER_RECOVER_ARGMAX)
     return SPECSTEER_ERR_INVALID_ARG;
-  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE | SPECSTEER_FLAG_SEPARATE_LAUNCHES | SPECSTEER_FLAG_ONE_LAUNCH)) return SPECSTEER_ERR_INVALID_ARG;
   if (d->B > 0) {
     if (!d->h_llm || !d->h_slm_plus || !d->h_slm_minus || !d->draft_len || !d->lambda || !d->beta ||
         !d->temperature || !d->accept_len)
@@ -214,7 +216,32 @@ specsteer_status recover_slab(specsteer_ctx* ctx, const specsteer_round_desc* d,
   return SPECSTEER_OK;
 }
 
+// A round of a single request (the paper's own regime: one user, one drafted block per round) with STEER recovery
+// runs in one launch: the streaming kernel also does the request's epilogue and its recovery sample.  With more
+// requests the one launch loses: the requests' last chunks are retired by whichever CTAs run last, a few CTAs end up
+// with most of the epilogues and run them one after the other (measured on 16 requests: 113 us against 38 us in three
+// launches), so those rounds keep their three launches unless SPECSTEER_FLAG_ONE_LAUNCH asks otherwise.
+bool fused_round(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
+  if (d->flags & SPECSTEER_FLAG_SEPARATE_LAUNCHES) return false;
+  if (large_round(d) || two_phase(d) || !rows_aligned(d) || d->recover_mode != SPECSTEER_RECOVER_STEER) return false;
+  if (d->B > kMaxSlabB || !d->u_recover) return false;
+  if (d->B != 1 && !(d->flags & SPECSTEER_FLAG_ONE_LAUNCH)) return false;
+  RoundParams p = slab_params(ctx, d, 0, d->B);
+  return fused_round_fits(p, d->dtype);
+}
+
 specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
+  ctx->v_fused = false;
+  if (fused_round(ctx, d)) {
+    RoundParams p = slab_params(ctx, d, 0, d->B);
+    p.req_done = ctx->req_done;
+    if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    if (launch_verify_fused(p, d->dtype, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+    ctx->launches += 1;
+    ctx->v_fused = true;
+    return SPECSTEER_OK;
+  }
   const bool lean = two_phase(d);
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
@@ -227,6 +254,7 @@ specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cu
 }
 
 specsteer_status do_recover(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
+  if (ctx->v_fused && d->recover_mode == SPECSTEER_RECOVER_STEER) return SPECSTEER_OK;   // the one launch did it
   const bool lean = ctx->v_two_phase;   // what the verification of this round did, not what this descriptor says
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
@@ -266,7 +294,7 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   const size_t b_st = align_up((size_t)max_B * sizeof(int), 256);
   const size_t b_tl = align_up((size_t)max_B * kTopkMaxSplit * 32 * sizeof(unsigned long long), 256);
   const size_t b_tc = align_up((size_t)max_B * sizeof(int), 256);
-  c->ws_bytes = b_part + 2 * b_lse + b_st + 256 + b_tl + b_tc;
+  c->ws_bytes = b_part + 2 * b_lse + 2 * b_st + 256 + b_tl + b_tc;
   if (cudaMalloc(&c->ws, c->ws_bytes) != cudaSuccess) {
     cudaGetLastError();
     delete c;
@@ -277,6 +305,7 @@ specsteer_status specsteer_ctx_create(specsteer_ctx** out, int device, int32_t m
   c->lse2 = (float*)w; w += b_lse;
   c->row_ref = (float*)w; w += b_lse;
   c->status_ws = (int*)w; w += b_st;
+  c->req_done = (int*)w; w += b_st;
   c->dev_error = (int*)w; w += 256;
   c->topk_lists = (void*)w; w += b_tl;
   c->topk_count = (int*)w;
@@ -471,7 +500,7 @@ specsteer_status prep_lmhead(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld
   if (d->B < 0 || d->K < 0 || d->V <= 0) return SPECSTEER_ERR_INVALID_ARG;
   if (d->accept_mode != SPECSTEER_ACCEPT_RATIO && d->accept_mode != SPECSTEER_ACCEPT_EXACT_Z) return SPECSTEER_ERR_INVALID_ARG;
   if (d->recover_mode != SPECSTEER_RECOVER_STEER && d->recover_mode != SPECSTEER_RECOVER_ARGMAX) return SPECSTEER_ERR_UNSUPPORTED;
-  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE)) return SPECSTEER_ERR_INVALID_ARG;
+  if (d->flags & ~(uint32_t)(SPECSTEER_FLAG_BONUS | SPECSTEER_FLAG_TWO_PHASE | SPECSTEER_FLAG_SEPARATE_LAUNCHES | SPECSTEER_FLAG_ONE_LAUNCH)) return SPECSTEER_ERR_INVALID_ARG;
   if (ld->d_llm <= 0 || ld->d_slm <= 0) return SPECSTEER_ERR_INVALID_ARG;
   if (ld->d_llm % 8 || ld->d_slm % 8) return SPECSTEER_ERR_UNSUPPORTED;   // rows of the operands must be 16-byte multiples
   if (d->B > 0) {

@@ -63,6 +63,7 @@ struct RoundParams {
   float* lse2;        // [B*(K+1)][4]            base-2 log-normalisers {L,P,M,R}
   int* status_ws;     // [B]                     request status when the caller passes no req_status
   int* dev_error;     // [1]                     set when a bounded wait gave up
+  int* req_done;      // [B]                     chunks retired per request (one-launch round); zero between launches
   long long wait_cycles;  // give-up limit of the streaming kernel's pipeline waits, in SM clocks
   float* row_ref;     // [B*(K+1)][4]            reference exponents per row {L,P,M,R} (row_ref_kernel), or null: the
                       //                         chunks take their references from their own first batch
@@ -124,6 +125,11 @@ cudaError_t launch_cloud_topk(const RoundParams& p, int dtype, int k, int* topk_
                               void* lists_ws, int* count_ws, int sm_count, cudaStream_t s);
 cudaError_t launch_edge_resample(const RoundParams& p, int dtype, int k, const int* topk_idx, const float* topk_val,
                                  cudaStream_t s);
+// The whole round of a small batch in one launch: streaming, per-request epilogue and STEER recovery sample.
+// p: ROWS_ALL, sums with SUM_R, 16-byte aligned rows, p.req_done set.  fused_round_fits: the vocabulary is small enough
+// for the chunk weights of a row to sit in the ring.
+bool fused_round_fits(const RoundParams& p, int dtype);
+cudaError_t launch_verify_fused(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s);
 // the reference exponents of every row (p.row_ref), for the streaming kernel launched next on the same stream
 cudaError_t launch_row_ref(const RoundParams& p, int dtype, cudaStream_t s);
 // the streaming kernel alone (partial records into the workspace), no epilogue

@@ -55,14 +55,15 @@ __device__ __forceinline__ double log2_pos(double x) {
 }
 
 // One warp: the largest exponent per normaliser over the row's records and the float64 sums relative to it
-// (pass 2 finds the lines of pass 1 in L1); every lane gets the results.
+// (read through L2: in the one-launch round the records come from other SMs of the same kernel); every lane gets the
+// results.
 __device__ __forceinline__ void row_sums_from_records(const RoundParams& p, const float* rec, int lane, float (&M)[4],
                                                       double (&S)[4]) {
   float Ml[4] = {kNegInf, kNegInf, kNegInf, kNegInf};
 #pragma unroll 4
   for (int ch = lane; ch < p.n_chunks; ch += 32) {
-    const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
-    const float4 z = __ldg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
+    const float4 x = __ldcg(reinterpret_cast<const float4*>(rec + ch * 8));
+    const float4 z = __ldcg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
     Ml[0] = fmaxf(Ml[0], x.x); Ml[1] = fmaxf(Ml[1], x.z); Ml[2] = fmaxf(Ml[2], z.x); Ml[3] = fmaxf(Ml[3], z.z);
   }
   const float mine = warp_reduce4<true>(Ml, lane);
@@ -70,8 +71,8 @@ __device__ __forceinline__ void row_sums_from_records(const RoundParams& p, cons
   for (int q = 0; q < 4; ++q) { M[q] = __shfl_sync(kFullMask, mine, 8 * q); S[q] = 0.0; }
 #pragma unroll 4
   for (int ch = lane; ch < p.n_chunks; ch += 32) {
-    const float4 x = __ldg(reinterpret_cast<const float4*>(rec + ch * 8));
-    const float4 z = __ldg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
+    const float4 x = __ldcg(reinterpret_cast<const float4*>(rec + ch * 8));
+    const float4 z = __ldcg(reinterpret_cast<const float4*>(rec + ch * 8 + 4));
     const float mm[4] = {x.x, x.z, z.x, z.z}, ss[4] = {x.y, x.w, z.y, z.w};
 #pragma unroll
     for (int q = 0; q < 4; ++q) {

@@ -16,6 +16,7 @@
 #include "common.cuh"
 #include "internal.h"
 #include "records.cuh"
+#include "recover_steer.cuh"
 #include "specsteer.h"
 
 namespace specsteer {
@@ -27,7 +28,7 @@ struct alignas(16) TileMeta {
                            // First and 16-byte aligned: they arrive with the tile, as a fourth bulk copy
   int row, tile, n_valid;  // padded row index b*(K+1)+t, tile within the row, valid entries in the tile
   float beta, c, inv_c;    // beta_b, log2(e)/T_b and its reciprocal for the owning request
-  int pad[2];
+  int req, pad;            // the owning request
 };
 static_assert(sizeof(TileMeta) == 48, "stage metadata: 16 bytes of references, then the tile's coordinates");
 
@@ -325,6 +326,7 @@ __device__ __forceinline__ bool chunk_fast(Acc& a, const T* sl, const T* sp, con
 // ---- per-request epilogue: Eq. 6/7 and the accepted length ------------------------------------------
 constexpr int kEpiWarps = 8;
 constexpr int kEpiMaxRows = 64;  // rows of one request held in shared memory; more run in several rounds
+constexpr int kFusedTailBytes = 8192;  // one-launch round: row results and sampling state at the start of the ring, chunk weights behind
 
 struct RowResult {
   double lse[4];
@@ -364,7 +366,7 @@ __device__ __forceinline__ double pow2_nonpos_int_d(float d) {
 
 // One warp: combine the partial records of `row` (exact power-of-two rescale, sums in double) and, for a
 // drafted row, the log-probabilities, alpha and the accept decision.
-template <typename T>
+template <typename T, bool PDL>
 __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float beta, float lam, float c, int lane,
                              RowResult* out) {
   const int K = p.K, K1 = K + 1;
@@ -384,7 +386,7 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
       if (p.sums & (SUM_P | SUM_R)) gp = load_logit<T>(reinterpret_cast<const T*>(p.h_plus), off);
     }
   }
-  pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
+  if (PDL) pdl_wait();  // everything above read inputs only; the records come from the streaming kernel
   if (p.tok_logits && y >= 0 && y < p.V) {  // fused LM-head path: the tensor-core pass left them in the workspace
     const float4 g = ld_cg_f4(p.tok_logits + row * 4);
     gl = g.x; gp = g.y; gm = g.z;
@@ -462,11 +464,19 @@ __device__ void epilogue_row(const RoundParams& p, int b, int t, int len, float 
   if (lane == 0) *out = r;
 }
 
-template <typename T>
-__global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundParams p) {
-  __shared__ RowResult res[kEpiMaxRows];
-  pdl_launch_dependents();  // the recovery kernel may be set up behind this one
-  const int b = blockIdx.x, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+// The barrier of the NT threads that work on one request: the whole CTA (BAR = 0) or the named barrier BAR.
+template <int BAR, int NT>
+__device__ __forceinline__ void epi_sync() {
+  if (BAR == 0) __syncthreads();
+  else asm volatile("bar.sync %0, %1;" ::"n"(BAR), "n"(NT) : "memory");
+}
+
+// One request, NT threads (tid = 0 .. NT - 1; res: kEpiMaxRows RowResults of shared memory): every warp combines
+// the records of one row at a time, then the rows are scanned in order for accept_len and the status word.
+template <typename T, int BAR, int NT, bool PDL>
+__device__ __forceinline__ void request_epilogue(const RoundParams& p, int b, int tid, RowResult* res) {
+  constexpr int NW = NT / 32;
+  const int warp = tid >> 5, lane = tid & 31;
   const int K = p.K, K1 = K + 1;
   int status = 0;
   int len = p.draft_len[b];
@@ -478,7 +488,7 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
   const float c = kLog2e / Tmp;
   const float qnan = __int_as_float(0x7fc00000);
 
-  for (int t = tid; t < K; t += kEpiWarps * 32) {
+  for (int t = tid; t < K; t += NT) {
     const long long i = (long long)b * K + t;
     if (p.accept_flags) p.accept_flags[i] = 0;
     if (p.alpha) p.alpha[i] = 0.f;
@@ -487,7 +497,7 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
     if (p.logp_plus) p.logp_plus[i] = qnan;
     if (p.logp_star) p.logp_star[i] = qnan;
   }
-  for (int t = tid; t <= K; t += kEpiWarps * 32)
+  for (int t = tid; t <= K; t += NT)
     if (p.log_z) p.log_z[(long long)b * K1 + t] = qnan;
 
   int n = len;
@@ -495,11 +505,11 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
   if (!params_ok) { status |= SPECSTEER_REQ_BAD_PARAM; n = 0; }
   for (int t0 = 0; t0 < R; t0 += kEpiMaxRows) {
     const int nr = min(kEpiMaxRows, R - t0);
-    __syncthreads();  // defaults written / previous round consumed
-    for (int k = warp; k < nr; k += kEpiWarps) epilogue_row<T>(p, b, t0 + k, len, beta, lam, c, lane, &res[k]);
-    __syncthreads();
+    epi_sync<BAR, NT>();  // defaults written / previous round consumed
+    for (int k = warp; k < nr; k += NW) epilogue_row<T, PDL>(p, b, t0 + k, len, beta, lam, c, lane, &res[k]);
+    epi_sync<BAR, NT>();
     // outputs of these rows (any thread), then the sequential scan (every thread, same result)
-    for (int k = tid; k < nr; k += kEpiWarps * 32) {
+    for (int k = tid; k < nr; k += NT) {
       const int t = t0 + k;
       const RowResult& r = res[k];
       if (r.fin && p.log_z) p.log_z[(long long)b * K1 + t] = (float)r.logz;
@@ -537,6 +547,13 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
   }
 }
 
+template <typename T>
+__global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundParams p) {
+  __shared__ RowResult res[kEpiMaxRows];
+  pdl_launch_dependents();  // the recovery kernel may be set up behind this one
+  request_epilogue<T, 0, kEpiWarps * 32, true>(p, blockIdx.x, threadIdx.x, res);
+}
+
 // ---- the persistent streaming kernel --------------------------------------------------------------
 // A tile is 2*CHUNK vocabulary entries of one used row, all three streams (three bulk copies, one stage).
 // Warps [0, NCW) consume: warps 2k and 2k+1 share the tiles congruent to k modulo NCW/2 and each reduces
@@ -544,7 +561,12 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
 // producer thread that owns the stages congruent to its index modulo NPW (one thread cannot issue tiles
 // fast enough for a whole SM).  Every stage is always consumed by the same pair of warps, so a waiting
 // warp is never a whole barrier phase ahead of the data.
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS, int POLY>
+// FUSED (small rounds): the whole round in this one launch.  Every chunk that is retired is counted per request; the
+// warp that retires a request's last chunk puts the request on its CTA's list, and when a CTA has streamed all its
+// tiles its consumer warps run the epilogue and the recovery sample (STEER) of the requests on its list - the same
+// device code the two stand-alone kernels run, so the outputs are the same bits.  Nobody waits for anybody: the
+// counters are only ever incremented, and a request with no rows at all belongs to CTA (request mod grid).
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS, int POLY, bool FUSED>
 __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const RoundParams p) {
   constexpr int TILE = 2 * CHUNK;
   constexpr bool kPlus = (SUMS & (SUM_P | SUM_R)) != 0;  // h_SLM+ is read at all
@@ -565,6 +587,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   float* c_s = beta_s + p.B;                                      // [B]  log2(e) / T_b
   float* ic_s = c_s + p.B;                                        // [B]  T_b / log2(e)
   int* first_s = reinterpret_cast<int*>(ic_s + p.B);              // [B]  first row of the request that is read
+  int* todo = first_s + p.B;                                      // FUSED: [B] requests this CTA finishes, [B] = how many
 
   pdl_launch_dependents();  // the epilogue's CTAs may take over SMs as this grid's CTAs retire
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -578,6 +601,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 2); }
     *abort_flag = 0;
     row_start[0] = 0;
+    if (FUSED) todo[p.B] = 0;
     fence_barrier_init();
   }
   for (int b = tid; b < p.B; b += nthreads) {
@@ -616,6 +640,10 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
   __syncthreads();
   const int total_tiles = row_start[p.B] * tiles_per_row;  // the host guarantees this fits in 31 bits
   const int cta = blockIdx.x, G = gridDim.x;
+  if (FUSED) {   // a request that streams nothing still gets its epilogue (defaults, accept_len, status)
+    for (int b = tid; b < p.B; b += nthreads)
+      if (row_start[b + 1] == row_start[b] && b % G == cta) todo[atomicAdd(&todo[p.B], 1)] = b;
+  }
 
   if (warp >= NCW) {
     // ================= producer warps =================
@@ -649,7 +677,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
           T* dst = tiles + (size_t)stage * NSLOT * TILE;
           TileMeta* mt = &meta[stage];
           mt->row = b * K1 + t; mt->tile = tr; mt->n_valid = n_valid;
-          mt->beta = beta_s[b]; mt->c = c_s[b]; mt->inv_c = ic_s[b];
+          mt->beta = beta_s[b]; mt->c = c_s[b]; mt->inv_c = ic_s[b]; mt->req = b;
           // the row's reference exponents travel with the tile: a fourth bulk copy, 16 bytes, onto the same barrier
           const uint32_t ref_bytes = p.row_ref ? 16u : 0u;
           if (!p.row_ref) mt->ref[0] = no_ref.x;
@@ -704,7 +732,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
         }
         __syncwarp();
         if (lane == 0) {
-          meta[stage] = TileMeta{{no_ref.x, 0.f, 0.f, 0.f}, b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b], {0, 0}};
+          meta[stage] = TileMeta{{no_ref.x, 0.f, 0.f, 0.f}, b * K1 + t, tr, n_valid, beta_s[b], c_s[b], ic_s[b], b, 0};
           mbar_arrive(&full[stage]);
         }
         cr += step_rows; tr += step_tiles;
@@ -763,24 +791,57 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
           float* rec = p.part + ((long long)mt.row * p.n_chunks + (mt.tile * 2 + half)) * 8;
           *reinterpret_cast<float2*>(rec + 2 * q) = make_float2(m_out, s_out);
         }
+        if (FUSED) {   // one more chunk of the request is in the workspace
+          __threadfence();
+          __syncwarp();
+          if (lane == 0) {
+            const int total = (row_start[mt.req + 1] - row_start[mt.req]) * p.n_chunks;
+            if (atomicAdd(p.req_done + mt.req, 1) + 1 == total) {
+              p.req_done[mt.req] = 0;   // nobody else touches it any more: left at zero for the next launch
+              __threadfence();          // what the other CTAs wrote before they counted is visible from here on
+              todo[atomicAdd(&todo[p.B], 1)] = mt.req;
+            }
+          }
+        }
+      }
+    }
+    if (FUSED) {
+      // ---- the requests this CTA finishes: epilogue (Eq. 6 / 7, accept_len) and recovery sample (Eq. 8) ----
+      constexpr int NT = NCW * 32;
+      epi_sync<1, NT>();   // every consumer warp has read its last stage; the ring is free
+      if (!*reinterpret_cast<volatile int*>(abort_flag)) {
+        const int n_todo = *reinterpret_cast<volatile int*>(&todo[p.B]);
+        RowResult* res = reinterpret_cast<RowResult*>(smem_raw);
+        PickShared* psh = reinterpret_cast<PickShared*>(smem_raw + kEpiMaxRows * sizeof(RowResult));
+        double* lse_fin = reinterpret_cast<double*>(smem_raw + kEpiMaxRows * sizeof(RowResult) + 256);
+        double* cw = reinterpret_cast<double*>(smem_raw + kFusedTailBytes);
+        for (int i = 0; i < n_todo; ++i) {
+          const int b = todo[i];
+          __threadfence();
+          request_epilogue<T, 1, NT, false>(p, b, tid, res);
+          epi_sync<1, NT>();   // accept_len, the status word and the row normalisers of the request are written
+          if (tid < kRecThreads) recover_steer_request<T, CHUNK, false, 2>(p, b, tid, cw, *psh, lse_fin);
+          epi_sync<1, NT>();   // the shared memory is reused by the next request
+        }
       }
     }
   }
 }
 
 // ---- launch -------------------------------------------------------------------------------------------
-template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS, int POLY = 0>
+template <typename T, int CHUNK, int STAGES, int NCW, int NPW, bool BULK, int SUMS, int POLY = 0, bool FUSED = false>
 static cudaError_t launch_stream(const RoundParams& p, const LaunchInfo& li, cudaStream_t s) {
-  const size_t fixed = (size_t)STAGES * ((SUMS & (SUM_P | SUM_R)) ? 3 : 2) * 2 * CHUNK * sizeof(T) + 2 * STAGES * sizeof(uint64_t) +
-                       STAGES * sizeof(TileMeta) + 16;
-  const size_t smem = fixed + (size_t)(5 * p.B + 1) * sizeof(int);
-  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS, POLY>;
+  const size_t ring = (size_t)STAGES * ((SUMS & (SUM_P | SUM_R)) ? 3 : 2) * 2 * CHUNK * sizeof(T);
+  const size_t fixed = ring + 2 * STAGES * sizeof(uint64_t) + STAGES * sizeof(TileMeta) + 16;
+  const size_t smem = fixed + (size_t)(6 * p.B + 2) * sizeof(int);
+  if (FUSED && (size_t)kFusedTailBytes + (size_t)p.n_chunks * sizeof(double) > ring) return cudaErrorInvalidValue;
+  auto kern = verify_kernel<T, CHUNK, STAGES, NCW, NPW, BULK, SUMS, POLY, FUSED>;
   // per instantiation and device; sized for the largest slab.  Contexts may be driven from different host threads:
   // the flag is atomic, and two threads that both find it clear merely set the same attribute twice.
   static std::atomic<bool> attr_set_dev[64];
   std::atomic<bool>& attr_set = attr_set_dev[li.device & 63];
   if (!attr_set.load(std::memory_order_acquire)) {
-    const size_t smem_max = fixed + (size_t)(5 * kMaxSlabB + 1) * sizeof(int);
+    const size_t smem_max = fixed + (size_t)(6 * kMaxSlabB + 2) * sizeof(int);
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max);
     if (e != cudaSuccess) return e;
     attr_set.store(true, std::memory_order_release);
@@ -922,6 +983,26 @@ cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, 
   if (sums == SUM_ALL) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL>(p, li, s);
   if (sums == kNoPlus) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kNoPlus>(p, li, s);
   return launch_stream<uint16_t, kChunkRatioBF16, 16, 16, 4, true, kRatio>(p, li, s);
+}
+
+// The whole round of a small batch in one launch (ROWS_ALL, STEER recovery, 16-byte aligned rows): see verify_kernel.
+bool fused_round_fits(const RoundParams& p, int dtype) {
+  // the chunk weights of one row share the ring with the row results (see launch_stream)
+  const size_t ring = dtype == SPECSTEER_F32 ? (size_t)12 * 3 * 2 * kChunkF32 * 4 : (size_t)16 * 3 * 2 * kChunkBF16 * 2;
+  return (size_t)kFusedTailBytes + (size_t)p.n_chunks * sizeof(double) <= ring;
+}
+
+cudaError_t launch_verify_fused(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s) {
+  constexpr int kNoPlus = SUM_L | SUM_M | SUM_R;
+  const bool all = (p.sums & SUM_P) != 0;
+  if (dtype == SPECSTEER_F32) {
+    if (all) return launch_stream<float, kChunkF32, 12, 12, 3, true, SUM_ALL, 0, true>(p, li, s);
+    return launch_stream<float, kChunkF32, 12, 12, 3, true, kNoPlus, 0, true>(p, li, s);
+  }
+  if (all && p.accept_mode == SPECSTEER_ACCEPT_RATIO)
+    return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL, 3, true>(p, li, s);
+  if (all) return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, SUM_ALL, 0, true>(p, li, s);
+  return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kNoPlus, 0, true>(p, li, s);
 }
 
 cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s) {

@@ -527,3 +527,51 @@ def test_host_round_with_algorithm1_outputs_edge_shapes(env, B, K, V):
         for k, v in host_out.items():
             assert np.array_equal(outs[k].cpu().numpy(), v.numpy(), equal_nan=True), (k, recover_mode)
         assert (host_out["rec_token"].numpy() >= 0).all()
+
+
+# ------------------------------------------------------------------ the one-launch round of small batches
+@pytest.mark.parametrize("cfg", [0, 1])
+@pytest.mark.parametrize("mode", MODES, ids=[m[0] for m in MODES])
+def test_one_launch_round_equals_separate_launches_on_configs(env, cfg, mode):
+    """The one-launch round (streaming, epilogue and STEER sample in the streaming kernel: the default for a single
+    request, FLAG_ONE_LAUNCH for more) against the same round in three launches.  Same device code per request: every
+    output byte equal."""
+    b, synth = env["binding"], env["synth"]
+    inputs = synth.make_round(synth.CONFIGS[cfg], device="cuda", seed=0)
+    _, am, rm, fl = mode
+    got = []
+    for extra, want in ((b.FLAG_ONE_LAUNCH, 1 if rm == 0 else 3), (b.FLAG_SEPARATE_LAUNCHES, 3 if rm == 0 else 4)):
+        before = env["ctx"].launch_count
+        out = P.run_gpu(env["ctx"], inputs, am, rm, fl | extra)
+        if rm == 0:
+            assert env["ctx"].launch_count - before == want
+        got.append(out)
+    for k in got[0]:
+        assert np.array_equal(got[0][k], got[1][k], equal_nan=True), k
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_one_launch_round_edge_cases(env, dtype):
+    """Requests that stream nothing (no drafts and no bonus row; bad parameters), bad tokens, non-finite rows, ragged
+    drafts, a ragged last chunk, more requests than CTAs: one launch against three, and against the oracle."""
+    b, synth = env["binding"], env["synth"]
+    spec, inputs = _small(synth, 200, 3, 2600, dtype, seed=77, ragged=True, beta_choices=(0.5, 1.0, 2.0),
+                          temp_choices=(0.7, 1.0))
+    inputs["draft_len"][0] = 0
+    inputs["draft_len"][7] = 0
+    inputs["temperature"][3] = 0.0
+    inputs["draft_tokens"][4, 0] = 2600
+    inputs["h_llm"][5, 1, 9] = float("nan")
+    inputs["draft_len"][6] = 9
+    for fl in (0, 1):
+        for am in (0, 1):
+            one = P.run_gpu(env["ctx"], inputs, am, 0, fl | b.FLAG_ONE_LAUNCH)
+            three = P.run_gpu(env["ctx"], inputs, am, 0, fl | b.FLAG_SEPARATE_LAUNCHES)
+            for k in one:
+                assert np.array_equal(one[k], three[k], equal_nan=True), (k, fl, am)
+            P.compare(env["oracle"], one, P.to_np_inputs(inputs), am, 0, fl, P.TOL[inputs["h_llm"].dtype])
+    # repeated launches leave the per-request counters at zero: the next round is right again
+    again = P.run_gpu(env["ctx"], inputs, 0, 0, 1 | b.FLAG_ONE_LAUNCH)
+    ref = P.run_gpu(env["ctx"], inputs, 0, 0, 1 | b.FLAG_SEPARATE_LAUNCHES)
+    for k in again:
+        assert np.array_equal(again[k], ref[k], equal_nan=True), k
