@@ -30,7 +30,7 @@ NOMINAL_HBM_GBS = 8000.0
 # DRAM bytes (read + write) per used row of the streaming kernel, from the ncu captures summarised under
 # profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows, so the figure for a
 # full launch is an extrapolation), keyed by configuration.  Absent = not captured for the kernel as it stands.
-NCU_TRAFFIC_BYTES_PER_ROW = {}
+NCU_TRAFFIC_BYTES_PER_ROW = {3: 1856690, 4: 1561579}
 
 
 def _peaks():
@@ -193,8 +193,8 @@ def _time_rounds(torch, ctx, descs, stream, steps, barrier, n_pairs=16):
     e1.record(stream)
     barrier()
     w1 = time.perf_counter()
-    kernel_ms = sum(a.elapsed_time(b) for a, b in evs[:used]) / used
-    return e0.elapsed_time(e1) / steps, kernel_ms, (w0, w1)
+    ks = [a.elapsed_time(b) for a, b in evs[:used]]
+    return e0.elapsed_time(e1) / steps, (sum(ks) / used, min(ks)), (w0, w1)
 
 
 def _ex2_rate(torch, binding, dev, stream, sampler):
@@ -232,26 +232,28 @@ def _largest_config(torch, binding, synth, dev, local_rank, stream, barrier, sam
              "positions_per_step": positions, "l2": "inputs exceed L2"}
     wins = []
     # every output: three tensors, every used row, four normalisers
-    ms, kms, win = _time_rounds(torch, ctx, [binding.make_desc(inputs, outs, flags=flags)], stream, steps, barrier)
+    ms, (kms, kmin), win = _time_rounds(torch, ctx, [binding.make_desc(inputs, outs, flags=flags)], stream, steps, barrier)
     wins.append(win)
     nbytes = spec.logit_bytes(rows)
     ach = nbytes / (kms * 1e-3) / 1e9
     block["all_outputs"] = {
-        "kernel": "verify_kernel", "kernel_ms": kms, "algorithmic_bytes_per_launch": nbytes, "achieved": ach, "unit": "GB/s",
+        "kernel": "verify_kernel", "kernel_ms": kms, "kernel_ms_fastest_launch": kmin,
+        "algorithmic_bytes_per_launch": nbytes, "achieved": ach, "unit": "GB/s",
         "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS, "ms_per_step": ms,
         "whole_step_gbs": nbytes / (ms * 1e-3) / 1e9, "whole_step_frac_of_nominal_8TBs": nbytes / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
         "positions_per_s": positions / (ms * 1e-3), "steps": steps}
     acc_all = outs["accept_len"].clone()
     # Algorithm 1's outputs only: verification streams h_LLM and h_SLM- over the drafted rows (Eq. 7), recovery then
     # streams row accept_len of every request that takes a token, all three tensors (Eq. 8)
-    ms, kms, win = _time_rounds(torch, ctx, [binding.make_desc(inputs, lean_outs, flags=flags)], stream, steps, barrier)
+    ms, (kms, kmin), win = _time_rounds(torch, ctx, [binding.make_desc(inputs, lean_outs, flags=flags)], stream, steps, barrier)
     wins.append(win)
     vbytes = 2 * positions * spec.V * spec.elem_bytes
     sampling = int((lean_outs["rec_token"] >= 0).sum().item())
     rbytes = 3 * sampling * spec.V * spec.elem_bytes
     ach = vbytes / (kms * 1e-3) / 1e9
     block["algorithm1_only"] = {
-        "kernel": "verify_kernel (two tensors, drafted rows)", "kernel_ms": kms, "algorithmic_bytes_per_launch": vbytes,
+        "kernel": "verify_kernel (two tensors, drafted rows)", "kernel_ms": kms, "kernel_ms_fastest_launch": kmin,
+        "algorithmic_bytes_per_launch": vbytes,
         "achieved": ach, "unit": "GB/s", "frac": ach / peak, "frac_of_nominal_8TBs": ach / NOMINAL_HBM_GBS,
         "ms_per_step": ms, "algorithmic_bytes_per_step": vbytes + rbytes,
         "whole_step_gbs": (vbytes + rbytes) / (ms * 1e-3) / 1e9,
