@@ -722,6 +722,10 @@ def run_lmhead(args, local_rank):
     positions = int(inputs["draft_len"].sum().item())
     ctx = binding.Context(B, K, V, device=local_rank)
     outs = binding.alloc_outputs(B, K, dev)
+    if args.lean:   # only Algorithm 1's outputs: the two-phase round (h_LLM and h_SLM- in verification, all three products
+        # on the compacted recovery rows)
+        for name in ("logp_plus", "logp_star", "log_z"):
+            outs.pop(name)
     desc = binding.make_lmhead_desc(inputs, outs, flags=binding.FLAG_BONUS,
                                     recover_mode=binding.RECOVER_ARGMAX if args.greedy else binding.RECOVER_STEER)
     stream = torch.cuda.current_stream(dev)
@@ -789,12 +793,15 @@ def run_lmhead(args, local_rank):
     sampler.stop()
     peak, peak_kind = _tensor_peak()
     flops = 2.0 * rows * V * (dL + 2 * dS)
+    if args.lean:   # what the two tensor-core launches actually multiply: two products on every row, three on one row per request
+        flops = 2.0 * rows * V * (dL + dS) + 2.0 * B * V * (dL + 2 * dS)
     achieved = flops / (kernel_ms * 1e-3) / 1e12
     line = {
         "workload": "%s_lmhead_dllm%d_dslm%d" % (spec.name, dL, dS), "metric": METRIC,
+        "outputs": "Algorithm 1 only (two-phase: lmhead_ratio_kernel on every row, lmhead_kernel on the compacted recovery rows)" if args.lean else "all",
         "recovery": "greedy (argmax of h_rec)" if args.greedy else "sampled",
         "value": positions / (fused_ms * 1e-3), "unit": UNIT, "ms_per_step": fused_ms, "steps": steps, "dtype": "bf16",
-        "roofline": {"bound": "tensor", "kernel": "lmhead_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+        "roofline": {"bound": "tensor", "kernel": "lmhead_ratio_kernel + lmhead_kernel" if args.lean else "lmhead_kernel", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
                      "frac": achieved / peak, "peak_source": "of " + peak_kind, "traffic": None,
                      "algorithmic_flops_per_launch": flops, "kernel_ms": kernel_ms},
         "unfused": {"ms_per_step": unfused_ms, "what": "three torch.matmul (library GEMM) products from the same bf16 operands, "

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "libspecsteer.so")
 SOURCES = ["api.cu", "verify.cu", "recover.cu", "topk.cu", "lmhead.cu", "static_scratch.cu", "probe.cu"]
-HEADERS = ["common.cuh", "internal.h", "records.cuh"]
+HEADERS = ["common.cuh", "internal.h", "records.cuh", "recover_steer.cuh"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-shared", "-Xptxas", "-v"]
 

@@ -47,6 +47,9 @@ struct specsteer_ctx {
   float* lm_part;
   float* lm_tok;
   void* lm_keys;      // [rows][chunks of 128] per-tile keys of the largest h_rec, for greedy recovery
+  // two-phase round on that path: the recovery rows' hidden states, compacted, and three small per-request arrays
+  void* lm_x2;
+  size_t lm_x2_bytes;
 };
 
 static_assert(sizeof(specsteer_round_desc) == 232, "the Python mirror of the descriptor assumes this layout");
@@ -327,6 +330,7 @@ specsteer_status specsteer_ctx_destroy(specsteer_ctx* ctx) {
   }
   if (ctx->stage) cudaFree(ctx->stage);
   if (ctx->lm_ws) cudaFree(ctx->lm_ws);
+  if (ctx->lm_x2) cudaFree(ctx->lm_x2);
   if (ctx->ws) cudaFree(ctx->ws);
   delete ctx;
   return SPECSTEER_OK;
@@ -547,6 +551,73 @@ specsteer_status prep_lmhead(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld
 }
 }  // namespace
 
+namespace {
+// The two-phase round on the LM-head path (only Algorithm 1's outputs wanted: the ratio rule, STEER or ARGMAX recovery,
+// none of logp_plus, logp_star, log_z): verification forms h_LLM and h_SLM- alone, in tiles twice as wide (Eq. 7);
+// then the hidden states of row accept_len of every request that takes a token are compacted and the three-product
+// kernel forms all three logit rows of just those positions (Eq. 8), from which the token is sampled (or the argmax
+// taken) exactly as in the one-pass round.
+bool lmhead_two_phase(const specsteer_round_desc* d) {
+  return d->accept_mode == SPECSTEER_ACCEPT_RATIO &&
+         (d->recover_mode == SPECSTEER_RECOVER_STEER || d->recover_mode == SPECSTEER_RECOVER_ARGMAX) && !d->logp_plus &&
+         !d->logp_star && !d->log_z && !(d->flags & SPECSTEER_FLAG_SEPARATE_LAUNCHES);
+}
+
+specsteer_status lmhead_round_two_phase(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, RoundParams p, LmheadOperands op,
+                                        cudaStream_t s) {
+  const specsteer_round_desc* d = &ld->round;
+  const int B = d->B;
+  // compact operands and per-request scratch (grown when a call needs more)
+  const size_t x_bytes = align_up((size_t)ctx->max_B * (size_t)(op.d_llm + 2 * op.d_slm) * 2, 256);
+  const size_t need = x_bytes + 3 * align_up((size_t)ctx->max_B * sizeof(int), 256);
+  if (need > ctx->lm_x2_bytes) {
+    if (ctx->lm_x2) { cudaStreamSynchronize(s); cudaFree(ctx->lm_x2); ctx->lm_x2 = nullptr; ctx->lm_x2_bytes = 0; }
+    if (cudaMalloc(&ctx->lm_x2, need) != cudaSuccess) { (void)cudaGetLastError(); return SPECSTEER_ERR_WORKSPACE; }
+    ctx->lm_x2_bytes = need;
+    ctx->ws_bytes += need;
+  }
+  uint16_t* xl = (uint16_t*)ctx->lm_x2;
+  uint16_t* xp = xl + (size_t)ctx->max_B * op.d_llm;
+  uint16_t* xm = xp + (size_t)ctx->max_B * op.d_slm;
+  int* c_n = (int*)((char*)ctx->lm_x2 + x_bytes);
+  int* c_status = c_n + align_up((size_t)ctx->max_B * sizeof(int), 256) / sizeof(int);
+  int* c_token = c_status + align_up((size_t)ctx->max_B * sizeof(int), 256) / sizeof(int);
+  const bool greedy = d->recover_mode == SPECSTEER_RECOVER_ARGMAX;
+
+  // 1. verification alone: h_LLM, h_SLM- of every row; 2. the per-request epilogue over the drafted rows
+  RoundParams pv = p;
+  pv.sums = SUM_L | SUM_M;
+  pv.row_mode = ROWS_DRAFTED;
+  pv.tile = kLmheadRatioChunk;
+  pv.n_chunks = n_chunks_of(d->V, kLmheadRatioChunk);
+  if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_lmhead_ratio(pv, op, ctx->lm_tok, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_epilogue(pv, SPECSTEER_F32, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  // 3. the recovery rows, compacted; 4. all three products on them (one row per request: a round with K = 0)
+  if (launch_lmhead_gather_rows(p, op, xl, xp, xm, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  RoundParams pc = p;
+  pc.K = 0;
+  pc.flags = p.flags | SPECSTEER_FLAG_BONUS;
+  pc.sums = SUM_ALL;
+  pc.row_mode = ROWS_ALL;
+  pc.accept_len = c_n; pc.status_ws = c_status; pc.req_status = nullptr;
+  pc.accept_flags = nullptr; pc.alpha = nullptr; pc.logp_llm = nullptr; pc.logp_minus = nullptr; pc.logp_plus = nullptr;
+  pc.logp_star = nullptr; pc.log_z = nullptr; pc.out_tokens = nullptr; pc.n_out = nullptr;
+  pc.rec_token = c_token;
+  LmheadOperands oc = op;
+  oc.x_llm = xl; oc.x_plus = xp; oc.x_minus = xm;
+  if (launch_lmhead(pc, oc, ctx->lm_tok, greedy ? ctx->lm_keys : nullptr, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (ctx->ev_stream_end && cudaEventRecord(ctx->ev_stream_end, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  // 5. the normalisers of those rows (and whether they are finite); 6. the token; 7. the round's outputs
+  if (launch_epilogue(pc, SPECSTEER_F32, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if ((greedy ? launch_lmhead_argmax(pc, ctx->lm_keys, s) : launch_lmhead_recover(pc, oc, s)) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_lmhead_finish(p, c_status, c_token, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  ctx->launches += 7;
+  (void)B;
+  return SPECSTEER_OK;
+}
+}  // namespace
+
 specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhead_desc* ld, void* cuda_stream) {
   RoundParams p;
   LmheadOperands op;
@@ -558,6 +629,7 @@ specsteer_status specsteer_lmhead_round(specsteer_ctx* ctx, const specsteer_lmhe
   DeviceGuard g(ctx->device);
   if (!g.ok) return SPECSTEER_ERR_CUDA;
   cudaStream_t s = (cudaStream_t)cuda_stream;
+  if (lmhead_two_phase(&ld->round)) return lmhead_round_two_phase(ctx, ld, p, op, s);
   if (ctx->ev_stream_begin && cudaEventRecord(ctx->ev_stream_begin, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;
   const bool greedy = ld->round.recover_mode == SPECSTEER_RECOVER_ARGMAX;
   if (launch_lmhead(p, op, ctx->lm_tok, greedy ? ctx->lm_keys : nullptr, ctx->li, s) != cudaSuccess) return SPECSTEER_ERR_CUDA;

@@ -113,6 +113,16 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
 // or null when nobody needs them.
 cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float* tok_logits, void* argmax_keys,
                           const LaunchInfo& li, cudaStream_t s);
+// Two-phase round on the LM-head path.  Verification alone: h_LLM and h_SLM- of every row (tiles of 128 x 256, records
+// at 256 entries per chunk, slots of h_SLM+ and h_rec empty) and the drafted tokens' two logits.
+constexpr int kLmheadRatioChunk = 256;
+cudaError_t launch_lmhead_ratio(const RoundParams& p, const LmheadOperands& op, float* tok_logits, const LaunchInfo& li,
+                                cudaStream_t s);
+// the hidden states of row accept_len of every request that takes a token, compacted to [B][d] (zero rows otherwise)
+cudaError_t launch_lmhead_gather_rows(const RoundParams& p, const LmheadOperands& op, uint16_t* xl, uint16_t* xp, uint16_t* xm,
+                                      cudaStream_t s);
+// rec_token, rec_logprob, out_tokens, n_out and the status words from the compact pass's token and status
+cudaError_t launch_lmhead_finish(const RoundParams& p, const int* c_status, const int* c_token, cudaStream_t s);
 // Sharded greedy rounds, last step: the outputs from the keys every shard agreed on (MAX over shards).
 cudaError_t launch_greedy_finish(const RoundParams& p, const long long* keys, cudaStream_t s);
 // Greedy recovery from those keys.

@@ -389,6 +389,266 @@ lmhead_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__
   }
 }
 
+// ---- verification alone: h_LLM and h_SLM- (Eq. 7), tiles of 128 rows x 256 vocabulary entries -------------
+// Algorithm 1's verification reads P_LLM and P_SLM- only, so when nothing of the fused target is wanted on the drafted
+// rows this kernel forms just those two products.  Two accumulators of 256 columns fill tensor memory, which buys a tile
+// twice as wide: every hidden-state tile is used for 256 vocabulary entries, a third fewer operand bytes per flop than
+// 128 x 128 tiles with three accumulators (the 128 x 128 kernel is short of operand bytes, not of tensor throughput).
+// The two normalisers are independent, so the epilogue of h_LLM runs under the product of h_SLM- and the epilogue of
+// h_SLM- under the next tile's h_LLM product: no second copy of an accumulator is needed.  Records: one per row and
+// tile of 256 entries, {m, s} of h_LLM and h_SLM-, the other two slots empty.
+constexpr int kBN2 = 256;
+constexpr int kGroups2 = 4;                       // one step of 64 hidden entries each: {x (16 KB), W (32 KB)}
+constexpr int kGroupBytes2 = 3 * kTileBytes;
+constexpr int kSmemBytes2 = kGroups2 * kGroupBytes2 + 1024 /* alignment */ + 512 /* barriers */;
+constexpr uint32_t kIdesc2 = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kBN2 >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+
+struct LmShared2 {
+  uint64_t full[kGroups2], empty[kGroups2];
+  uint64_t tmem_full[2], tmem_empty[2], drain;
+  uint32_t tmem_slot;
+  int abort_flag;
+};
+__device__ __forceinline__ bool aborted2(const LmShared2* sh) { return *reinterpret_cast<const volatile int*>(&sh->abort_flag) != 0; }
+__device__ __forceinline__ void set_abort2(LmShared2* sh, int* dev_error) {
+  *reinterpret_cast<volatile int*>(&sh->abort_flag) = 1;
+  atomicExch(dev_error, 1);
+}
+
+// One accumulator of 256 columns, one row per thread: the record {m, s} of sum_v 2^(x_v c) over the valid columns, and
+// the logit in column `jtok` (if 0 <= jtok < n_valid) into *tok_out / *found.
+__device__ __forceinline__ float2 reduce_acc256(uint32_t taddr, int n_valid, float c, int jtok, uint32_t* tok_out, bool* found) {
+  float mx = kNegInf;
+#pragma unroll 1
+  for (int j0 = 0; j0 < kBN2; j0 += 32) {
+    uint32_t A[32];
+    tmem_ld32(taddr + j0, A);
+    tmem_ld_wait();
+    const int nv = n_valid - j0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < nv) mx = fmaxf(mx, __uint_as_float(A[j]));
+    const int jj = jtok - j0;
+    if (jj >= 0 && jj < 32 && jj < nv) {
+      uint32_t t = 0;
+#pragma unroll
+      for (int j = 0; j < 32; ++j)
+        if (j == jj) t = A[j];
+      *tok_out = t;
+      *found = true;
+    }
+  }
+  const float ref = ceilf(mx * c);
+  const float nref = (ref > kNegInf && ref < -kNegInf) ? -ref : 0.f;
+  float s = 0.f;
+#pragma unroll 1
+  for (int j0 = 0; j0 < kBN2; j0 += 32) {
+    uint32_t A[32];
+    tmem_ld32(taddr + j0, A);
+    tmem_ld_wait();
+    const int nv = n_valid - j0;
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (j < nv) s += ex2(fmaf(__uint_as_float(A[j]), c, nref));
+  }
+  return make_record(ref, s);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+lmhead_ratio_kernel(const __grid_constant__ CUtensorMap tm_xl, const __grid_constant__ CUtensorMap tm_wl,
+                    const __grid_constant__ CUtensorMap tm_xm, const __grid_constant__ CUtensorMap tm_wm,
+                    const LmKernelParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // operand tiles need 1024-byte alignment
+  LmShared2* sh = reinterpret_cast<LmShared2*>(smem_raw + (smem0 - smem_u32(smem_raw)) + kGroups2 * kGroupBytes2);
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int mb_count = (p.R + kBM - 1) / kBM, nb_count = (p.V + kBN2 - 1) / kBN2;
+  const int n_tiles = mb_count * nb_count;
+  const int nkL = (p.d_llm + kBK - 1) / kBK, nkS = (p.d_slm + kBK - 1) / kBK;
+
+  if (tid == 0) {
+    for (int s = 0; s < kGroups2; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&sh->tmem_full[a], 1); mbar_init(&sh->tmem_empty[a], 4); }
+    mbar_init(&sh->drain, 1);
+    sh->abort_flag = 0;
+    fence_barrier_init();
+  }
+  if (warp == 1) tmem_alloc(&sh->tmem_slot, kTmemCols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *reinterpret_cast<volatile uint32_t*>(&sh->tmem_slot);
+
+  if (warp == 0) {
+    // ================= TMA producer =================
+    if (lane == 0) {
+      int grp = 0;
+      bool ok = true;
+      auto steps = [&](const CUtensorMap* ta, const CUtensorMap* tb, int m0, int n0, int nk) {
+        for (int kb = 0; kb < nk && ok; ++kb, ++grp) {
+          const int gs = grp % kGroups2;
+          const uint32_t ph = (uint32_t)((grp / kGroups2) & 1);
+          if (aborted2(sh) || !mbar_wait(&sh->empty[gs], ph ^ 1u)) { set_abort2(sh, p.dev_error); ok = false; break; }
+          const uint32_t base = smem0 + gs * kGroupBytes2;
+          mbar_arrive_expect_tx(&sh->full[gs], 3 * kTileBytes);
+          tma_load_2d(base, ta, kb * kBK, m0, &sh->full[gs]);
+          tma_load_2d(base + kTileBytes, tb, kb * kBK, n0, &sh->full[gs]);   // 256 rows of the head: 32 KB
+        }
+      };
+      for (int g = blockIdx.x; g < n_tiles && ok; g += gridDim.x) {
+        const int mb = g % mb_count, nb = g / mb_count;  // row blocks fastest: CTAs running together share W tiles in L2
+        steps(&tm_xl, &tm_wl, mb * kBM, nb * kBN2, nkL);
+        steps(&tm_xm, &tm_wm, mb * kBM, nb * kBN2, nkS);
+      }
+      if (!ok) {  // copies already issued may still be landing: wait for them (bounded) before the CTA exits
+        for (int i = grp > kGroups2 ? grp - kGroups2 : 0; i < grp; ++i)
+          mbar_wait(&sh->full[i % kGroups2], (uint32_t)((i / kGroups2) & 1));
+      }
+    }
+  } else if (warp == 1) {
+    // ================= tensor-core issuer =================
+    if (lane == 0) {
+      int grp = 0, ti = 0;
+      bool ok = true;
+      auto product = [&](uint32_t col, int nk) {
+        for (int kb = 0; kb < nk && ok; ++kb, ++grp) {
+          const int gs = grp % kGroups2;
+          if (aborted2(sh) || !mbar_wait(&sh->full[gs], (uint32_t)((grp / kGroups2) & 1))) { set_abort2(sh, p.dev_error); ok = false; break; }
+          tc_fence_after();
+          const uint32_t base = smem0 + gs * kGroupBytes2;
+          const uint64_t ad = smem_desc_sw128(base), bd = smem_desc_sw128(base + kTileBytes);
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k)
+            umma_bf16(tmem_base + col, ad + (uint64_t)(2 * k), bd + (uint64_t)(2 * k), kIdesc2, (kb | k) != 0);
+          umma_commit(&sh->empty[gs]);  // the group is free once these have read it
+        }
+      };
+      for (int g = blockIdx.x; g < n_tiles && ok; g += gridDim.x, ++ti) {
+        for (int a = 0; a < 2 && ok; ++a) {
+          if (ti > 0) {   // the epilogue of the tile before has read this accumulator
+            if (aborted2(sh) || !mbar_wait(&sh->tmem_empty[a], (uint32_t)((ti - 1) & 1))) { set_abort2(sh, p.dev_error); ok = false; break; }
+            tc_fence_after();
+          }
+          product(a ? 256u : 0u, a ? nkS : nkL);
+          if (ok) umma_commit(&sh->tmem_full[a]);
+        }
+      }
+      if (!ok) {  // let everything issued finish before tensor memory is given back
+        umma_commit(&sh->drain);
+        mbar_wait(&sh->drain, 0);
+      }
+    }
+  } else {
+    // ================= epilogue warps: one row per thread =================
+    const int quarter = warp & 3;  // the lanes of tensor memory this warp may read
+    const int K1 = p.K + 1;
+    int ti = 0;
+    for (int g = blockIdx.x; g < n_tiles; g += gridDim.x, ++ti) {
+      const int mb = g % mb_count, nb = g / mb_count;
+      const int row = mb * kBM + quarter * 32 + lane, n0 = nb * kBN2;
+      const bool valid = row < p.R;
+      float c = 1.f;
+      int tok = -1;
+      if (valid) {
+        const int b = row / K1, t = row - b * K1;
+        c = kLog2e / p.temperature[b];
+        int len = p.draft_len[b];
+        if (len < 0 || len > p.K) len = 0;
+        if (t < len) tok = p.draft_tokens[(long long)b * p.K + t] - p.vocab_offset;   // id within the heads passed
+      }
+      const int n_valid = min(kBN2, p.V - n0);
+      float2 rec2[2];
+      uint32_t tl[2] = {0u, 0u};
+      bool found = false;
+      bool alive = true;
+      for (int a = 0; a < 2; ++a) {
+        bool ok = !aborted2(sh) && mbar_wait(&sh->tmem_full[a], (uint32_t)(ti & 1));
+        ok = __all_sync(kFullMask, ok);
+        if (!ok) {
+          if (lane == 0) set_abort2(sh, p.dev_error);
+          alive = false;
+          break;
+        }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (a ? 256u : 0u);
+        rec2[a] = reduce_acc256(taddr, n_valid, c, tok - n0, &tl[a], &found);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&sh->tmem_empty[a]);  // the accumulator may be overwritten
+      }
+      if (!alive) break;
+      if (valid) {
+        if (found) *reinterpret_cast<uint4*>(p.tok_logits + (long long)row * 4) = make_uint4(tl[0], 0u, tl[1], 1u);
+        float* rec = p.part + ((long long)row * p.n_chunks + nb) * 8;
+        *reinterpret_cast<float4*>(rec) = make_float4(rec2[0].x, rec2[0].y, kNegInf, 0.f);
+        *reinterpret_cast<float4*>(rec + 4) = make_float4(rec2[1].x, rec2[1].y, kNegInf, 0.f);
+      }
+    }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ---- two-phase round on this path: the recovery rows, compacted ----------------------------------------------
+// The hidden states of row accept_len of every request that takes a token, gathered into [B][d] arrays (zero rows for
+// the others), so that the three-accumulator kernel can form all three logit rows of exactly those positions (Eq. 8).
+__global__ void __launch_bounds__(256) lmhead_gather_rows_kernel(const RoundParams p, const LmheadOperands op, uint16_t* xl,
+                                                                 uint16_t* xp, uint16_t* xm) {
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int K = p.K, K1 = K + 1;
+  const int n = p.accept_len[b];
+  int len = p.draft_len[b];
+  if (len < 0 || len > K) len = 0;
+  const bool bad = (p.status_ws[b] & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+  const bool sample = !bad && n >= 0 && n <= len && (n < len || (p.flags & SPECSTEER_FLAG_BONUS));
+  const long long row = (long long)b * K1 + (sample ? n : 0);
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = tid * 8; i < op.d_llm; i += 256 * 8)
+    *reinterpret_cast<uint4*>(xl + (long long)b * op.d_llm + i) =
+        sample ? __ldg(reinterpret_cast<const uint4*>(op.x_llm + row * op.d_llm + i)) : zero;
+  for (int i = tid * 8; i < op.d_slm; i += 256 * 8) {
+    *reinterpret_cast<uint4*>(xp + (long long)b * op.d_slm + i) =
+        sample ? __ldg(reinterpret_cast<const uint4*>(op.x_plus + row * op.d_slm + i)) : zero;
+    *reinterpret_cast<uint4*>(xm + (long long)b * op.d_slm + i) =
+        sample ? __ldg(reinterpret_cast<const uint4*>(op.x_minus + row * op.d_slm + i)) : zero;
+  }
+}
+
+// Last step of the two-phase round: the compact pass sampled (or took the argmax of) one token per request into
+// rec_token / rec_logprob; this puts the round's outputs together from the real accepted lengths.  c_status: the status
+// words of the compact pass (a non-finite recovery row shows there).
+__global__ void __launch_bounds__(128) lmhead_finish_kernel(const RoundParams p, const int* c_status, const int* c_token) {
+  const int b = blockIdx.x * 128 + threadIdx.x;
+  if (b >= p.B) return;
+  const int K = p.K, K1 = K + 1;
+  const int n = p.accept_len[b];
+  int status = p.status_ws[b];
+  int len = p.draft_len[b];
+  if (len < 0 || len > K) len = 0;
+  const bool bad = (status & (SPECSTEER_REQ_BAD_PARAM | SPECSTEER_REQ_NONFINITE)) != 0;
+  bool sample = !bad && (n < len || (p.flags & SPECSTEER_FLAG_BONUS));
+  if (sample && (c_status[b] & SPECSTEER_REQ_NONFINITE)) {   // the recovery row has no distribution
+    status |= SPECSTEER_REQ_NONFINITE;
+    p.status_ws[b] = status;
+    if (p.req_status) p.req_status[b] = status;
+    sample = false;
+  }
+  int tok = sample ? c_token[b] : -1;   // c_token may be the caller's rec_token itself
+  if (!sample || tok < 0) {
+    tok = -1;
+    if (p.rec_logprob) p.rec_logprob[b] = __int_as_float(0x7fc00000);
+  }
+  if (p.rec_token) p.rec_token[b] = tok;
+  if (p.out_tokens)
+    for (int t = 0; t <= K; ++t)
+      p.out_tokens[(long long)b * K1 + t] = (t < n) ? p.draft_tokens[(long long)b * K + t] : ((t == n && tok >= 0) ? tok : -1);
+  if (p.n_out) p.n_out[b] = n + (tok >= 0 ? 1 : 0);
+}
+
 // ---- recovery ------------------------------------------------------------------------------------------
 constexpr int kRecT = 1024;  // 32 warps: recomputing the chunk is a chain of dependent loads per warp, so many warps
 struct LmRecShared {
@@ -597,12 +857,12 @@ EncodeTiledFn encode_fn() {
 }
 
 // [rows][d] bf16, row-major: boxes of 64 x 128 entries (128 bytes x 128 rows), 128-byte swizzle, zero fill outside
-bool encode_operand(CUtensorMap* tm, const void* base, int rows, int d) {
+bool encode_operand(CUtensorMap* tm, const void* base, int rows, int d, int box_rows = kBM) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
   const cuuint64_t strides[1] = {(cuuint64_t)d * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)kBM};
+  const cuuint32_t box[2] = {(cuuint32_t)kBK, (cuuint32_t)box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -637,6 +897,47 @@ cudaError_t launch_lmhead(const RoundParams& p, const LmheadOperands& op, float*
   const long long tiles = (long long)mb * nb;
   const int grid = (int)(tiles < li.sm_count ? tiles : li.sm_count);
   lmhead_kernel<<<grid, kThreads, kSmemBytes, s>>>(tm[0], tm[1], tm[2], tm[3], tm[4], tm[5], k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_lmhead_ratio(const RoundParams& p, const LmheadOperands& op, float* tok_logits, const LaunchInfo& li,
+                                cudaStream_t s) {
+  const int R = p.B * (p.K + 1);
+  if (R == 0) return cudaSuccess;
+  CUtensorMap tm[4];
+  if (!encode_operand(&tm[0], op.x_llm, R, op.d_llm) || !encode_operand(&tm[1], op.w_llm, p.V, op.d_llm, kBN2) ||
+      !encode_operand(&tm[2], op.x_minus, R, op.d_slm) || !encode_operand(&tm[3], op.w_minus, p.V, op.d_slm, kBN2))
+    return cudaErrorInvalidValue;
+  LmKernelParams k;
+  k.R = R; k.V = p.V; k.K = p.K; k.d_llm = op.d_llm; k.d_slm = op.d_slm; k.n_chunks = p.n_chunks;
+  k.draft_tokens = p.draft_tokens; k.draft_len = p.draft_len; k.beta = p.beta; k.temperature = p.temperature;
+  k.part = p.part; k.tok_logits = tok_logits; k.dev_error = p.dev_error;
+  k.argmax_keys = nullptr;
+  k.shared_head = 0;
+  k.vocab_offset = p.vocab_offset;
+  static std::atomic<bool> attr_set[64];
+  if (!attr_set[li.device & 63].load(std::memory_order_acquire)) {
+    cudaError_t e = cudaFuncSetAttribute(lmhead_ratio_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes2);
+    if (e != cudaSuccess) return e;
+    attr_set[li.device & 63].store(true, std::memory_order_release);
+  }
+  const int mb = (R + kBM - 1) / kBM, nb = (p.V + kBN2 - 1) / kBN2;
+  const long long tiles = (long long)mb * nb;
+  const int grid = (int)(tiles < li.sm_count ? tiles : li.sm_count);
+  lmhead_ratio_kernel<<<grid, kThreads, kSmemBytes2, s>>>(tm[0], tm[1], tm[2], tm[3], k);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_lmhead_gather_rows(const RoundParams& p, const LmheadOperands& op, uint16_t* xl, uint16_t* xp, uint16_t* xm,
+                                      cudaStream_t s) {
+  if (p.B == 0) return cudaSuccess;
+  lmhead_gather_rows_kernel<<<p.B, 256, 0, s>>>(p, op, xl, xp, xm);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_lmhead_finish(const RoundParams& p, const int* c_status, const int* c_token, cudaStream_t s) {
+  if (p.B == 0) return cudaSuccess;
+  lmhead_finish_kernel<<<(p.B + 127) / 128, 128, 0, s>>>(p, c_status, c_token);
   return cudaGetLastError();
 }
 

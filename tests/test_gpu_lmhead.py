@@ -126,9 +126,18 @@ def test_zero_drafts_and_bad_tokens(env):
 def test_outputs_can_be_left_out(env):
     inputs = env["synth"].make_lmhead_round(_spec(env, 0, B=7, K=3, V=1800), 128, 64, device="cuda", seed=7)
     full = _run_gpu(env, inputs)
-    lean = _run_gpu(env, inputs, drop=("logp_plus", "logp_star", "log_z", "alpha", "accept_flags", "req_status"))
+    lean = _run_gpu(env, inputs, drop=("logp_plus", "log_z", "alpha", "accept_flags", "req_status"))     # still one pass
     for k in lean:
         assert np.array_equal(full[k], lean[k], equal_nan=True), k
+    # without logp_star as well the round is two-phase (other tiles, other summation order): same decisions and tokens,
+    # floating-point outputs to rounding
+    lean = _run_gpu(env, inputs, drop=("logp_plus", "logp_star", "log_z", "alpha", "accept_flags", "req_status"))
+    for k in lean:
+        if lean[k].dtype.kind in "iu":
+            assert np.array_equal(full[k], lean[k]), k
+        else:
+            assert np.array_equal(np.isnan(full[k]), np.isnan(lean[k])), k
+            assert np.nanmax(np.abs(full[k] - lean[k]), initial=0.0) < 1e-4, k
 
 
 def test_repeated_calls_are_bit_identical(env):
@@ -329,3 +338,72 @@ def test_greedy_and_sampled_fused_rounds_share_the_verification(env):
     torch.cuda.synchronize()
     for k in ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "logp_plus", "logp_star", "log_z", "req_status"):
         assert np.array_equal(outs[k].cpu().numpy(), sampled[k], equal_nan=True), k
+
+
+# ------------------------------------------------------------------ the two-phase round on this path
+TWO_PHASE_KEYS = ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "rec_token", "rec_logprob", "out_tokens",
+                  "n_out", "req_status")
+
+
+def _two_phase_case(env, spec, d_llm, d_slm, seed, flags=1, recover_mode=0, mutate=None, launches=7):
+    """Only Algorithm 1's outputs requested: verification forms h_LLM and h_SLM- alone (tiles of 128 x 256), the
+    recovery rows are compacted and get all three products.  Every request against the oracle round that reads only
+    what Algorithm 1 reads, on float64 logits."""
+    b = env["binding"]
+    inputs = env["synth"].make_lmhead_round(spec, d_llm, d_slm, device="cuda", seed=seed)
+    if mutate:
+        mutate(inputs)
+    outs = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k in TWO_PHASE_KEYS}
+    desc = b.make_lmhead_desc(inputs, outs, recover_mode=recover_mode, flags=flags)
+    before = env["ctx"].launch_count
+    env["ctx"].lmhead_round(desc)
+    torch.cuda.synchronize()
+    assert env["ctx"].device_error() == 0 and env["ctx"].launch_count - before == launches
+    gpu = {k: v.cpu().numpy() for k, v in outs.items()}
+    stats = P.compare(env["oracle"], gpu, _np_inputs(env["oracle"], inputs), 0, recover_mode, flags, TOL, margin=MARGIN,
+                      alg1=True, keys=TWO_PHASE_KEYS)
+    return inputs, gpu, stats
+
+
+@pytest.mark.parametrize("recover_mode", [0, 2], ids=["sampled", "greedy"])
+def test_two_phase_round_small_ragged_vocabulary(env, recover_mode):
+    _, gpu, stats = _two_phase_case(env, _spec(env, 0, B=5, K=3, V=3001), 320, 128, seed=0, recover_mode=recover_mode)
+    assert (gpu["rec_token"] >= 0).all() and stats["max_logp_err"] < TOL
+
+
+def test_two_phase_round_several_row_blocks_odd_hidden_widths_no_bonus(env):
+    """280 rows = 2 blocks + 24 in verification, 70 compact rows in recovery; widths that end inside a stage of 64."""
+    spec = _spec(env, 4, B=70, K=3, V=1000, ragged=True)
+    inputs, gpu, _ = _two_phase_case(env, spec, 200, 72, seed=1, flags=0)
+    dl = inputs["draft_len"].cpu().numpy()
+    assert ((gpu["rec_token"] >= 0) == (gpu["accept_len"] < dl)).all()
+
+
+def test_two_phase_round_more_tiles_than_sms(env):
+    """188 vocabulary tiles of 256 on 148 CTAs: the accumulators are reused, each epilogue runs under the other product."""
+    _, gpu, _ = _two_phase_case(env, _spec(env, 1, B=20, K=5, V=48000), 256, 64, seed=2)
+    assert len(set(gpu["rec_token"].tolist())) > 5
+
+
+def test_two_phase_round_degenerate_requests(env):
+    def mutate(inputs):
+        inputs["draft_len"][0] = 0                   # nothing drafted: only the bonus row
+        inputs["draft_tokens"][1, 1] = -3            # bad tokens
+        inputs["draft_tokens"][2, 0] = 2500
+        inputs["temperature"][3] = 0.0               # bad parameter: nothing accepted, no token
+        inputs["u_accept"][4] = 0.0                  # everything accepted: the bonus row is the recovery row
+        inputs["lam"][5] = 1e30                      # rejected at once
+    _, gpu, _ = _two_phase_case(env, _spec(env, 0, B=8, K=3, V=2500), 128, 64, seed=6, mutate=mutate)
+    assert gpu["accept_len"][0] == 0 and gpu["rec_token"][0] >= 0
+    assert gpu["req_status"][1] & 1 and gpu["req_status"][2] & 1
+    assert gpu["req_status"][3] == 16 and gpu["rec_token"][3] == -1 and gpu["n_out"][3] == 0
+    assert gpu["accept_len"][4] == 3 and gpu["n_out"][4] == 4
+    assert gpu["accept_len"][5] == 0 and gpu["n_out"][5] == 1
+
+
+def test_two_phase_round_twice_gives_the_same_bits(env):
+    spec = _spec(env, 0, B=33, K=4, V=9000)
+    _, a, _ = _two_phase_case(env, spec, 320, 128, seed=8)
+    _, c, _ = _two_phase_case(env, spec, 320, 128, seed=8)
+    for k in a:
+        assert np.array_equal(a[k], c[k], equal_nan=True), k
