@@ -233,7 +233,13 @@ specsteer_status specsteer_shard_recover_local(specsteer_ctx *ctx, const specste
  *     (max_B*(max_K+1)*(16 + 40*ceil(max_V/128)) bytes); later calls allocate nothing.
  *   - Accuracy: the logits carry the rounding of a float32 accumulation over d bf16 products, so decisions may
  *     differ from exact arithmetic where their margin is below about 1e-4.
- * Three launches; stream-ordered; specsteer_ctx_time_streaming brackets the tensor-core kernel.
+ *   - With only Algorithm 1's outputs requested (RATIO, STEER or ARGMAX, logp_plus / logp_star / log_z NULL, and not
+ *     SPECSTEER_FLAG_SEPARATE_LAUNCHES) the round is two-phase: verification forms h_LLM and h_SLM- alone (Eq. 7) in
+ *     tiles twice as wide, then all three products of row accept_len of every request that takes a token (Eq. 8) from
+ *     compacted hidden states.  Seven launches, about a fifth faster; a further workspace of
+ *     max_B*(d_llm + 2*d_slm)*2 bytes is allocated by the first such call.  Same decisions and tokens as the one-pass
+ *     round up to the accuracy stated above.
+ * Three launches otherwise; stream-ordered; specsteer_ctx_time_streaming brackets the tensor-core kernel(s).
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, TIMEOUT, CUDA. */
 typedef struct {
   specsteer_round_desc round;
