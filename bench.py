@@ -31,6 +31,22 @@ NOMINAL_HBM_GBS = 8000.0
 # profiles/ (taken on 32 requests of the same recipe; traffic grows in proportion to the rows, so the figure for a
 # full launch is an extrapolation), keyed by configuration.  Absent = not captured for the kernel as it stands.
 NCU_TRAFFIC_BYTES_PER_ROW = {3: 1856690, 4: 1561579}
+# The streaming kernel's sources as they were when those counters were taken (sha256 over the files below, in this
+# order): when they have changed since, the traffic figure no longer describes the kernel and is reported as null.
+NCU_TRAFFIC_SOURCES = ("verify.cu", "common.cuh", "records.cuh", "internal.h")
+NCU_TRAFFIC_SOURCE_SHA256 = "496e09680e4e86e82c68c8f6a72941e50c3d778ba6e7a7afc3e35a43d45ba206"
+
+
+def _traffic_still_valid():
+    import hashlib
+    h = hashlib.sha256()
+    try:
+        for name in NCU_TRAFFIC_SOURCES:
+            with open(os.path.join(ROOT, "paper_2603_16219_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+    except OSError:
+        return False
+    return h.hexdigest() == NCU_TRAFFIC_SOURCE_SHA256
 
 
 def _peaks():
@@ -618,14 +634,14 @@ def run_cuda(args, rank, world, local_rank):
         return
 
     achieved = logit_bytes / (kernel_ms * 1e-3) / 1e9
+    traffic_ok = args.config in NCU_TRAFFIC_BYTES_PER_ROW and not args.requests and not args.lean and _traffic_still_valid()
     roofline = {
         "bound": "hbm", "kernel": "verify_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
         "frac": achieved / peak,
         "peak_source": "of " + peak_kind + " (a read+write copy: a read-only kernel can exceed it)",
-        "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.config] * rows if args.config in NCU_TRAFFIC_BYTES_PER_ROW
-                    and not args.requests else None),
+        "traffic": (NCU_TRAFFIC_BYTES_PER_ROW[args.config] * rows if traffic_ok else None),
         "traffic_source": ("extrapolated: ncu dram bytes per row on a 32-request capture x rows of this launch"
-                           if args.config in NCU_TRAFFIC_BYTES_PER_ROW and not args.requests else None),
+                           if traffic_ok else "none: not captured for this workload, or the kernel's sources changed since"),
         "algorithmic_bytes_per_launch": logit_bytes, "kernel_ms": kernel_ms,
         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
         "whole_step_gbs": logit_bytes / (ms_per_step * 1e-3) / 1e9,

@@ -20,6 +20,10 @@ TOL = 5e-4
 MARGIN = 2e-4
 
 
+TWO_PHASE_KEYS = ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "rec_token", "rec_logprob", "out_tokens",
+                  "n_out", "req_status")
+
+
 @pytest.fixture(scope="module")
 def env(oracle_mod):
     from paper_2603_16219_b200 import binding, build, synth
@@ -217,6 +221,13 @@ def test_full_size_sampled_requests():
         torch.cuda.synchronize()
         assert ctx.device_error() == 0
         gpu = {k: v.cpu().numpy() for k, v in outs.items()}
+        # the same batch with only Algorithm 1's outputs requested: the two-phase round, as `bench.py --lmhead --lean` times it
+        outs2 = {k: v for k, v in b.alloc_outputs(spec.B, spec.K, "cuda").items() if k in TWO_PHASE_KEYS}
+        before = ctx.launch_count
+        ctx.lmhead_round(b.make_lmhead_desc(inputs, outs2, flags=1))
+        torch.cuda.synchronize()
+        assert ctx.device_error() == 0 and ctx.launch_count - before == 7
+        gpu2 = {k: v.cpu().numpy() for k, v in outs2.items()}
     finally:
         ctx.close()
     P.invariants(gpu, {"draft_tokens": inputs["draft_tokens"], "draft_len": inputs["draft_len"]}, 1, TOL)
@@ -235,6 +246,12 @@ def test_full_size_sampled_requests():
     stats = P.compare(o, gpu, npin, 0, 0, 1, TOL, sel=sel, margin=MARGIN)
     print("lmhead full size", stats)
     assert stats["requests"] == 32
+    stats2 = P.compare(o, gpu2, npin, 0, 0, 1, TOL, sel=sel, margin=MARGIN, alg1=True, keys=TWO_PHASE_KEYS)
+    print("lmhead full size, two-phase", stats2)
+    assert stats2["requests"] == 32
+    # over the whole batch the two rounds agree wherever neither decision is near a margin (a handful may differ)
+    same = (gpu["accept_len"] == gpu2["accept_len"]) & (gpu["rec_token"] == gpu2["rec_token"])
+    assert same.mean() > 0.97, same.mean()
 
 
 def test_no_drafts_at_all_and_empty_batch(env):
@@ -341,10 +358,6 @@ def test_greedy_and_sampled_fused_rounds_share_the_verification(env):
 
 
 # ------------------------------------------------------------------ the two-phase round on this path
-TWO_PHASE_KEYS = ("accept_len", "accept_flags", "alpha", "logp_llm", "logp_minus", "rec_token", "rec_logprob", "out_tokens",
-                  "n_out", "req_status")
-
-
 def _two_phase_case(env, spec, d_llm, d_slm, seed, flags=1, recover_mode=0, mutate=None, launches=7):
     """Only Algorithm 1's outputs requested: verification forms h_LLM and h_SLM- alone (tiles of 128 x 256), the
     recovery rows are compacted and get all three products.  Every request against the oracle round that reads only
