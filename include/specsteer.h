@@ -76,11 +76,13 @@ enum {
   SPECSTEER_FLAG_TWO_PHASE = 2u, /* take the two-phase round (see the outputs below) whenever it is eligible, however
                                    small the batch; without it the library takes it from 128 MB of logits upwards,
                                    below which its two extra launches cost more than the bytes it saves */
-  SPECSTEER_FLAG_SEPARATE_LAUNCHES = 4u, /* keep verification and recovery in launches of their own.  Without it a
-                                   round of ONE request (below 128 MB of logits, STEER recovery, 16-byte aligned rows)
-                                   runs in one launch: specsteer_verify_round then also samples the recovery token and
-                                   writes rec_token, rec_logprob, out_tokens and n_out, and the
-                                   specsteer_recover_sample that follows launches nothing.  Same outputs, bit for bit.
+  SPECSTEER_FLAG_SEPARATE_LAUNCHES = 4u, /* keep verification and recovery in launches of their own.  Without it, when
+                                   recovery is the STEER sample, u_recover is given and the round is not two-phase,
+                                   the launch that runs the verification epilogue also samples the recovery token:
+                                   specsteer_verify_round then writes rec_token, rec_logprob, out_tokens and n_out
+                                   as well, and the specsteer_recover_sample that follows launches nothing.  A round
+                                   of ONE request (below 128 MB of logits, 16-byte aligned rows) runs in a single
+                                   launch altogether.  Same outputs, bit for bit.
                                    Set it when something else than specsteer_recover_sample follows
                                    (specsteer_cloud_topk: the sample would be wasted work) or when the recovery outputs
                                    must not be written before that call. */
@@ -157,7 +159,8 @@ specsteer_status specsteer_ctx_destroy(specsteer_ctx *ctx);
  * computes the four log-normalisers, then per position the log-probabilities, alpha and the accept flag,
  * and per request accept_len = the first t with u_accept > alpha (or draft_len).  Writes every output of
  * the descriptor except rec_token, rec_logprob, out_tokens, n_out (req_status is written here and may gain
- * bits in specsteer_recover_sample).  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
+ * bits in specsteer_recover_sample); unless SPECSTEER_FLAG_SEPARATE_LAUNCHES is set it may write those four as well
+ * (see the flag).  Errors: INVALID_ARG, UNSUPPORTED, CUDA. */
 specsteer_status specsteer_verify_round(specsteer_ctx *ctx, const specsteer_round_desc *desc, void *cuda_stream);
 
 /* Recovery (Algorithm 1 Phase 3; Eq. 8): for each request whose accept_len < draft_len (or always, with

@@ -179,7 +179,7 @@ bool two_phase(const specsteer_round_desc* d) {
 // Verification of the requests [b0, b0 + nb).  lean: two tensors over the drafted rows, in the larger chunks of that
 // launch shape (the two-phase round).
 specsteer_status verify_slab(specsteer_ctx* ctx, const specsteer_round_desc* d, int b0, int nb, bool lean, cudaStream_t s,
-                             cudaEvent_t ev_begin, cudaEvent_t ev_end) {
+                             cudaEvent_t ev_begin, cudaEvent_t ev_end, bool with_recover) {
   RoundParams p = slab_params(ctx, d, b0, nb);
   if (lean) {
     p.sums = SUM_L | SUM_M;
@@ -192,7 +192,8 @@ specsteer_status verify_slab(specsteer_ctx* ctx, const specsteer_round_desc* d, 
   // about 128 MB of logits the extra launch costs more than it can save.
   if (large_round(d) && rows_aligned(d)) p.row_ref = ctx->row_ref + (size_t)b0 * (d->K + 1) * 4;
   int nl = 0;
-  if (launch_verify(p, d->dtype, rows_aligned(d), ctx->li, s, &nl, ev_begin, ev_end) != cudaSuccess) return SPECSTEER_ERR_CUDA;
+  if (launch_verify(p, d->dtype, rows_aligned(d), ctx->li, s, &nl, ev_begin, ev_end, with_recover) != cudaSuccess)
+    return SPECSTEER_ERR_CUDA;
   ctx->launches += nl;
   return SPECSTEER_OK;
 }
@@ -233,6 +234,11 @@ bool fused_round(const specsteer_ctx* ctx, const specsteer_round_desc* d) {
   return fused_round_fits(p, d->dtype);
 }
 
+bool tail_in_one_launch(const specsteer_round_desc* d, bool lean) {
+  return !lean && d->recover_mode == SPECSTEER_RECOVER_STEER && d->u_recover != nullptr &&
+         !(d->flags & SPECSTEER_FLAG_SEPARATE_LAUNCHES);
+}
+
 specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cudaStream_t s) {
   ctx->v_fused = false;
   if (fused_round(ctx, d)) {
@@ -246,13 +252,18 @@ specsteer_status do_verify(specsteer_ctx* ctx, const specsteer_round_desc* d, cu
     return SPECSTEER_OK;
   }
   const bool lean = two_phase(d);
+  // A round whose verification reads every row and whose recovery is the STEER sample needs nothing between its
+  // epilogue and that sample: one launch does both (same device code, same bits), and the recovery call that follows
+  // finds its work done.
+  const bool tail = tail_in_one_launch(d, lean);
   for (int b0 = 0; b0 < d->B; b0 += kMaxSlabB) {
     const int nb = d->B - b0 < kMaxSlabB ? d->B - b0 : kMaxSlabB;
     const bool first = b0 == 0, last = b0 + nb >= d->B;
     specsteer_status st = verify_slab(ctx, d, b0, nb, lean, s, first ? ctx->ev_stream_begin : nullptr,
-                                      last ? ctx->ev_stream_end : nullptr);
+                                      last ? ctx->ev_stream_end : nullptr, tail);
     if (st != SPECSTEER_OK) return st;
   }
+  ctx->v_fused = tail;
   return SPECSTEER_OK;
 }
 
@@ -855,7 +866,7 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
       }
       CK(cudaEventRecord(ctx->ev_copied[idx2], ctx->copy_stream));
       CK(cudaStreamWaitEvent(s, ctx->ev_copied[idx2], 0));
-      if (verify_slab(ctx, &forced, b0, nb, true, s, nullptr, nullptr) != SPECSTEER_OK) fail = true;
+      if (verify_slab(ctx, &forced, b0, nb, true, s, nullptr, nullptr, false) != SPECSTEER_OK) fail = true;
     }
     int32_t* n_host = (int32_t*)malloc((size_t)B * 8);
     if (!n_host) fail = true;
@@ -905,8 +916,10 @@ specsteer_status specsteer_round_host(specsteer_ctx* ctx, const specsteer_round_
     CK(cudaStreamWaitEvent(s, ctx->ev_copied[idx], 0));
     RoundParams p = slab_params(ctx, &d, b0, nb);
     int nl = 0;
-    CK(launch_verify(p, d.dtype, rows_aligned(&d), ctx->li, s, &nl)); ctx->launches += nl;
-    if (d.recover_mode == SPECSTEER_RECOVER_ARGMAX) {
+    const bool tail = tail_in_one_launch(&d, false);   // epilogue and STEER sample in one launch
+    CK(launch_verify(p, d.dtype, rows_aligned(&d), ctx->li, s, &nl, nullptr, nullptr, tail)); ctx->launches += nl;
+    if (tail) {
+    } else if (d.recover_mode == SPECSTEER_RECOVER_ARGMAX) {
       CK(launch_recover_argmax(p, d.dtype, rows_aligned(&d), false, (char*)ctx->topk_lists + (size_t)b0 * kTopkMaxSplit * 32 * 8,
                                ctx->topk_count + b0, ctx->li.sm_count, s));
       ctx->launches += 1;

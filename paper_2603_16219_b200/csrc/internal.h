@@ -106,8 +106,10 @@ struct LaunchInfo {
 };
 
 // ev_begin / ev_end, when not null, are recorded on `s` just before and just after the streaming kernel.
+// with_recover: the launch that runs the epilogue also draws the STEER recovery sample (see launch_epilogue).
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
-                          int* n_launches, cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr);
+                          int* n_launches, cudaEvent_t ev_begin = nullptr, cudaEvent_t ev_end = nullptr,
+                          bool with_recover = false);
 // The tensor-core pass: partial records of every row at kLmheadChunk entries per chunk, and tok_logits.
 // argmax_keys: [B*(K+1)][n_chunks] 64-bit words that receive, per tile, the key of the largest h_rec (greedy recovery),
 // or null when nobody needs them.
@@ -146,8 +148,10 @@ cudaError_t launch_row_ref(const RoundParams& p, int dtype, cudaStream_t s);
 cudaError_t launch_verify_stream(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s);
 // per-row ShardPartial of this shard from its partial records: out[B][K+1]
 cudaError_t launch_shard_rows(const RoundParams& p, int dtype, ShardPartial* out, cudaStream_t s);
-// the per-request epilogue alone (reads p.shard_parts when p.n_shards > 0)
-cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s);
+// the per-request epilogue alone (reads p.shard_parts when p.n_shards > 0); with_recover: the same CTAs go on to the
+// STEER recovery sample of their request (p as for launch_recover without own_lse, records at the logit type's chunk
+// size), which saves the second launch of a round whose verification read every row
+cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s, bool with_recover = false);
 // own_lse: row accept_len has records but no normalisers yet (two-phase round); the STEER kernel forms them first.
 cudaError_t launch_recover(const RoundParams& p, int dtype, const LaunchInfo& li, cudaStream_t s, int* n_launches,
                            bool own_lse = false);

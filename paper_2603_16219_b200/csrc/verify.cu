@@ -554,6 +554,21 @@ __global__ void __launch_bounds__(kEpiWarps * 32) epilogue_kernel(const RoundPar
   request_epilogue<T, 0, kEpiWarps * 32, true>(p, blockIdx.x, threadIdx.x, res);
 }
 
+// The epilogue and the STEER recovery sample of a request in one CTA and one launch: the same device code as
+// epilogue_kernel followed by recover_steer_kernel (the outputs are the same bits), without the second launch.
+template <typename T, int TILE>
+__global__ void __launch_bounds__(kEpiWarps * 32) epilogue_recover_kernel(const RoundParams p) {
+  static_assert(kEpiWarps * 32 == kRecThreads, "one CTA shape serves both steps");
+  extern __shared__ double cw[];  // [n_chunks] chunk weights of the recovery row
+  __shared__ RowResult res[kEpiMaxRows];
+  __shared__ PickShared sh;
+  __shared__ double lse_fin[2];
+  pdl_launch_dependents();
+  request_epilogue<T, 0, kEpiWarps * 32, true>(p, blockIdx.x, threadIdx.x, res);
+  __syncthreads();   // accept_len, the status word and the row normalisers of the request are written
+  recover_steer_request<T, TILE, false, 0>(p, blockIdx.x, threadIdx.x, cw, sh, lse_fin);
+}
+
 // ---- the persistent streaming kernel --------------------------------------------------------------
 // A tile is 2*CHUNK vocabulary entries of one used row, all three streams (three bulk copies, one stage).
 // Warps [0, NCW) consume: warps 2k and 2k+1 share the tiles congruent to k modulo NCW/2 and each reduces
@@ -1005,24 +1020,28 @@ cudaError_t launch_verify_fused(const RoundParams& p, int dtype, const LaunchInf
   return launch_stream<uint16_t, kChunkBF16, 16, 16, 4, true, kNoPlus, 0, true>(p, li, s);
 }
 
-cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s) {
+cudaError_t launch_epilogue(const RoundParams& p, int dtype, cudaStream_t s, bool with_recover) {
   // programmatic dependent launch: the epilogue reads its inputs while the kernel before it drains
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(p.B);
   cfg.blockDim = dim3(kEpiWarps * 32);
-  cfg.dynamicSmemBytes = 0;
+  cfg.dynamicSmemBytes = with_recover ? (size_t)p.n_chunks * sizeof(double) : 0;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (with_recover) {
+    if (dtype == SPECSTEER_F32) return cudaLaunchKernelEx(&cfg, epilogue_recover_kernel<float, kChunkF32>, p);
+    return cudaLaunchKernelEx(&cfg, epilogue_recover_kernel<uint16_t, kChunkBF16>, p);
+  }
   if (dtype == SPECSTEER_F32) return cudaLaunchKernelEx(&cfg, epilogue_kernel<float>, p);
   return cudaLaunchKernelEx(&cfg, epilogue_kernel<uint16_t>, p);
 }
 
 cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const LaunchInfo& li, cudaStream_t s,
-                          int* n_launches, cudaEvent_t ev_begin, cudaEvent_t ev_end) {
+                          int* n_launches, cudaEvent_t ev_begin, cudaEvent_t ev_end, bool with_recover) {
   *n_launches = 2;
   cudaError_t e;
   if (p.row_ref) {
@@ -1032,7 +1051,7 @@ cudaError_t launch_verify(const RoundParams& p, int dtype, bool aligned, const L
   if (ev_begin && (e = cudaEventRecord(ev_begin, s)) != cudaSuccess) return e;
   if ((e = launch_verify_stream(p, dtype, aligned, li, s)) != cudaSuccess) return e;
   if (ev_end && (e = cudaEventRecord(ev_end, s)) != cudaSuccess) return e;
-  return launch_epilogue(p, dtype, s);
+  return launch_epilogue(p, dtype, s, with_recover);
 }
 
 }  // namespace specsteer

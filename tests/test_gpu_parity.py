@@ -540,7 +540,11 @@ def test_one_launch_round_equals_separate_launches_on_configs(env, cfg, mode):
     inputs = synth.make_round(synth.CONFIGS[cfg], device="cuda", seed=0)
     _, am, rm, fl = mode
     got = []
-    for extra, want in ((b.FLAG_ONE_LAUNCH, 1 if rm == 0 else 3), (b.FLAG_SEPARATE_LAUNCHES, 3 if rm == 0 else 4)):
+    # the library's own choice: one launch for a single request, otherwise the streaming kernel and one launch for
+    # epilogue + STEER sample
+    default = 1 if synth.CONFIGS[cfg].B == 1 else 2
+    for extra, want in ((b.FLAG_ONE_LAUNCH, 1 if rm == 0 else 3), (b.FLAG_SEPARATE_LAUNCHES, 3 if rm == 0 else 4),
+                        (0, default if rm == 0 else 3)):
         before = env["ctx"].launch_count
         out = P.run_gpu(env["ctx"], inputs, am, rm, fl | extra)
         if rm == 0:
@@ -548,6 +552,7 @@ def test_one_launch_round_equals_separate_launches_on_configs(env, cfg, mode):
         got.append(out)
     for k in got[0]:
         assert np.array_equal(got[0][k], got[1][k], equal_nan=True), k
+        assert np.array_equal(got[2][k], got[1][k], equal_nan=True), k
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
@@ -567,8 +572,10 @@ def test_one_launch_round_edge_cases(env, dtype):
         for am in (0, 1):
             one = P.run_gpu(env["ctx"], inputs, am, 0, fl | b.FLAG_ONE_LAUNCH)
             three = P.run_gpu(env["ctx"], inputs, am, 0, fl | b.FLAG_SEPARATE_LAUNCHES)
+            two = P.run_gpu(env["ctx"], inputs, am, 0, fl)   # streaming kernel, then epilogue + sample in one launch
             for k in one:
                 assert np.array_equal(one[k], three[k], equal_nan=True), (k, fl, am)
+                assert np.array_equal(two[k], three[k], equal_nan=True), (k, fl, am)
             P.compare(env["oracle"], one, P.to_np_inputs(inputs), am, 0, fl, P.TOL[inputs["h_llm"].dtype])
     # repeated launches leave the per-request counters at zero: the next round is right again
     again = P.run_gpu(env["ctx"], inputs, 0, 0, 1 | b.FLAG_ONE_LAUNCH)
