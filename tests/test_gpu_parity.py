@@ -582,3 +582,40 @@ def test_one_launch_round_edge_cases(env, dtype):
     ref = P.run_gpu(env["ctx"], inputs, 0, 0, 1 | b.FLAG_SEPARATE_LAUNCHES)
     for k in again:
         assert np.array_equal(again[k], ref[k], equal_nan=True), k
+
+
+# ------------------------------------------------------------------ the paper's comparison decoders, as inputs to this path
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_standard_speculative_decoding_as_an_input_special_case(env, dtype):
+    """Standard speculative decoding (the "Standard SD" row of the paper's efficiency table) is this path with the
+    drafter in both Specialist slots, beta = 0, the exact acceptance of Eq. 6 (target P_LLM, proposal P_SLM+) and the
+    residual fallback: alpha = min(1, P_LLM/Q) and the resample from max(0, P_LLM - Q).  The two Specialist pointers
+    name the same tensor."""
+    synth = env["synth"]
+    spec, inputs = _small(synth, 24, 4, 9000, dtype, seed=5, ragged=True, temp_choices=(0.7, 1.0))
+    inputs["h_slm_minus"] = inputs["h_slm_plus"]       # the same device memory behind both pointers
+    inputs["beta"].fill_(0.0)
+    inputs["lam"].fill_(1.0)
+    gpu = P.run_gpu(env["ctx"], inputs, 1, 1, 0)
+    npin = P.to_np_inputs(inputs)
+    P.compare(env["oracle"], gpu, npin, 1, 1, 0, P.TOL[inputs["h_llm"].dtype])
+    # with beta = 0 the fused target is P_LLM itself: log P* = log P_LLM and log Z = 0 on every verified row
+    n = gpu["accept_len"]
+    for b in range(spec.B):
+        rows = min(int(n[b]) + 1, int(npin["draft_len"][b]))
+        if gpu["req_status"][b] == 0 and rows > 0:
+            np.testing.assert_allclose(gpu["logp_star"][b, :rows], gpu["logp_llm"][b, :rows], atol=P.TOL[inputs["h_llm"].dtype])
+            np.testing.assert_allclose(gpu["log_z"][b, :rows], 0.0, atol=P.TOL[inputs["h_llm"].dtype])
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_always_on_steering_as_an_input_special_case(env, dtype):
+    """Steering at every step without drafts (the always-on logit steering the paper compares with): no drafted
+    tokens, FLAG_BONUS, so every request samples one token from Softmax(h_LLM + beta (h_SLM+ - h_SLM-)) (Eq. 8) on
+    row 0."""
+    synth = env["synth"]
+    spec, inputs = _small(synth, 40, 3, 12001, dtype, seed=6, beta_choices=(0.5, 1.0, 2.0), temp_choices=(0.7, 1.0))
+    inputs["draft_len"].zero_()
+    gpu = P.run_gpu(env["ctx"], inputs, 0, 0, 1)
+    P.compare(env["oracle"], gpu, P.to_np_inputs(inputs), 0, 0, 1, P.TOL[inputs["h_llm"].dtype])
+    assert (gpu["accept_len"] == 0).all() and (gpu["n_out"] == 1).all() and (gpu["rec_token"] >= 0).all()
