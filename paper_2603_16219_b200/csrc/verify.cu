@@ -677,6 +677,7 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
     if (BULK) {
       if (lane == 0) {  // one elected thread issues the bulk copies
         int issued = 0;
+        const uint64_t stream_once = l2_policy_evict_first();   // the logits pass through L2 once and need not stay
         for (int j = pw, g = g0; g < total_tiles; j += NPW, g += gstep) {
           const int stage = j % STAGES;
           const uint32_t phase = (uint32_t)((j / STAGES) & 1);
@@ -707,9 +708,9 @@ __global__ void __launch_bounds__((NCW + NPW) * 32, 1) verify_kernel(const Round
             if (ref_bytes) bulk_g2s(mt->ref, p.row_ref + 4ll * (b * K1 + t), 16u, &full[stage]);
           }
           if (bytes) {
-            bulk_g2s(dst, hl + off, bytes, &full[stage]);
-            if (kPlus) bulk_g2s(dst + TILE, hp + off, bytes, &full[stage]);
-            bulk_g2s(dst + MSLOT * TILE, hm + off, bytes, &full[stage]);
+            bulk_g2s(dst, hl + off, bytes, &full[stage], stream_once);
+            if (kPlus) bulk_g2s(dst + TILE, hp + off, bytes, &full[stage], stream_once);
+            bulk_g2s(dst + MSLOT * TILE, hm + off, bytes, &full[stage], stream_once);
           } else if (!ref_bytes) {
             mbar_arrive(&full[stage]);
           }
