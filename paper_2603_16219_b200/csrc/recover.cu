@@ -114,17 +114,24 @@ __global__ void __launch_bounds__(kRecThreads) recover_residual_kernel(const Rou
 template <typename T> struct Vec8;
 template <> struct Vec8<float> {
   static __device__ __forceinline__ void load(const float* p, long long i, float (&x)[8]) {
-    const float4 a = __ldg(reinterpret_cast<const float4*>(p + i)), b = __ldg(reinterpret_cast<const float4*>(p + i + 4));
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p + i)), b = __ldcs(reinterpret_cast<const float4*>(p + i + 4));   // read once: streaming loads
     x[0] = a.x; x[1] = a.y; x[2] = a.z; x[3] = a.w; x[4] = b.x; x[5] = b.y; x[6] = b.z; x[7] = b.w;
   }
 };
 template <> struct Vec8<uint16_t> {
   static __device__ __forceinline__ void load(const uint16_t* p, long long i, float (&x)[8]) {
-    const uint4 a = __ldg(reinterpret_cast<const uint4*>(p + i));
+    const uint4 a = __ldcs(reinterpret_cast<const uint4*>(p + i));
     x[0] = bf16lo(a.x); x[1] = bf16hi(a.x); x[2] = bf16lo(a.y); x[3] = bf16hi(a.y);
     x[4] = bf16lo(a.z); x[5] = bf16hi(a.z); x[6] = bf16lo(a.w); x[7] = bf16hi(a.w);
   }
 };
+
+// max that hands a NaN on: the running maxima of the three streams then show a NaN or +inf entry by themselves
+__device__ __forceinline__ float fmax_nan(float a, float b) {
+  float d;
+  asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(a), "f"(b));
+  return d;
+}
 
 // An online (maximum, sum of 2^(x - maximum)) pair and its merge; empty = (-inf, 0).
 struct OnlineLse {
@@ -177,8 +184,8 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   float best_r = 0.f;   // the thread walks its entries in ascending id order, so "strictly larger" keeps the lowest id
   int best_v = -1;
   OnlineLse acc = {kNegInf, 0.f};
-  float mx[3] = {kNegInf, kNegInf, kNegInf};   // largest entry of each stream
-  bool bad = false;                            // a NaN or +inf entry
+  float mx[3] = {kNegInf, kNegInf, kNegInf};   // largest entry of each stream; NaN once the stream held a NaN
+#pragma unroll 2   // two iterations' loads in flight: 16-bit rows otherwise keep too few bytes outstanding per SM
   for (int v = v0 + tid * 8; v < v1; v += kRecThreads * 8) {
     float l[8], q[8], m[8], r[8];
     int n = 8;
@@ -204,8 +211,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
       for (int i = 0; i < 8; ++i) {
         x[i] = r[i] * c;
         if (i < n) {
-          bad = bad || !(l[i] < -kNegInf) || !(q[i] < -kNegInf) || !(m[i] < -kNegInf);
-          mx[0] = fmaxf(mx[0], l[i]); mx[1] = fmaxf(mx[1], q[i]); mx[2] = fmaxf(mx[2], m[i]);
+          mx[0] = fmax_nan(mx[0], l[i]); mx[1] = fmax_nan(mx[1], q[i]); mx[2] = fmax_nan(mx[2], m[i]);
         } else {
           x[i] = kNegInf;
         }
@@ -232,10 +238,9 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
       t.s = __shfl_xor_sync(kFullMask, acc.s, o);
       acc = lse_merge(acc, t);
 #pragma unroll
-      for (int q = 0; q < 3; ++q) mx[q] = fmaxf(mx[q], __shfl_xor_sync(kFullMask, mx[q], o));
+      for (int q = 0; q < 3; ++q) mx[q] = fmax_nan(mx[q], __shfl_xor_sync(kFullMask, mx[q], o));
     }
   }
-  if (LSE && __any_sync(kFullMask, bad)) acc.s = __int_as_float(0x7fc00000);
   if (lane == 0) {
     wbest[warp] = best;
     if (LSE) { wlse[warp] = acc; wmax[warp][0] = mx[0]; wmax[warp][1] = mx[1]; wmax[warp][2] = mx[2]; }
@@ -246,7 +251,7 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
     best = wbest[w] > best ? wbest[w] : best;
     if (LSE) {
       acc = lse_merge(acc, wlse[w]);
-      for (int q = 0; q < 3; ++q) mx[q] = fmaxf(mx[q], wmax[w][q]);
+      for (int q = 0; q < 3; ++q) mx[q] = fmax_nan(mx[q], wmax[w][q]);
     }
   }
   // workspace of the request: [0, 16) keys, [16, 32) {maximum, sum}, [32, 48) {max h_LLM, max h_SLM+}, [48, 64) max h_SLM-
@@ -269,9 +274,9 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
         const u64 a = __ldcg(mine + 16 + j), b2 = __ldcg(mine + 32 + j), c2 = __ldcg(mine + 48 + j);
         OnlineLse t = {__uint_as_float((uint32_t)(a >> 32)), __uint_as_float((uint32_t)a)};
         acc = lse_merge(acc, t);
-        mx[0] = fmaxf(mx[0], __uint_as_float((uint32_t)(b2 >> 32)));
-        mx[1] = fmaxf(mx[1], __uint_as_float((uint32_t)b2));
-        mx[2] = fmaxf(mx[2], __uint_as_float((uint32_t)(c2 >> 32)));
+        mx[0] = fmax_nan(mx[0], __uint_as_float((uint32_t)(b2 >> 32)));
+        mx[1] = fmax_nan(mx[1], __uint_as_float((uint32_t)b2));
+        mx[2] = fmax_nan(mx[2], __uint_as_float((uint32_t)(c2 >> 32)));
       }
     }
     count_ws[b] = 0;
@@ -286,7 +291,8 @@ __global__ void __launch_bounds__(kRecThreads) recover_argmax_kernel(const Round
   bool fin = best != 0;
   if (LSE) {
     lseR = (double)acc.m + log2((double)acc.s);
-    fin = fin && isfinite(lseR) && mx[0] > kNegInf && mx[1] > kNegInf && mx[2] > kNegInf;
+    // every stream's largest entry finite: no NaN, no +inf, and not -inf throughout
+    fin = fin && isfinite(lseR) && isfinite(mx[0]) && isfinite(mx[1]) && isfinite(mx[2]);
     if (!fin) {
       p.status_ws[b] = st.status | SPECSTEER_REQ_NONFINITE;
       if (p.req_status) p.req_status[b] = st.status | SPECSTEER_REQ_NONFINITE;
